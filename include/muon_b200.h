@@ -1,0 +1,202 @@
+/*
+ * muon_b200.h -- C ABI of the B200-native layout-driven Muon step.
+ *
+ * The library implements the local compute core of the paper's distributed Muon
+ * (Section 6, Algorithm 2): whole matrices are materialised from a padded flat
+ * FSDP-style shard buffer, every 2-D matrix receives one Muon update
+ * (momentum -> Frobenius normalisation -> Newton-Schulz iteration of Eq. 1 ->
+ * shape-scaled, weight-decayed update), and results are scattered back.
+ *
+ * Conventions (all entry points)
+ *  - Every call returns MUON_OK (0) or a negative MUON_ERR_* code.  Nothing is
+ *    launched when validation fails.  No exception crosses this boundary.
+ *  - "device pointer" = address in the current CUDA device's global memory, owned by
+ *    the caller; "host pointer" = ordinary process memory, read during the call only
+ *    unless stated otherwise.
+ *  - Arrays of matrix pointers (params, grads, ...) are HOST arrays of DEVICE pointers.
+ *  - Matrices are dense row-major with leading dimension == cols.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *    All device work is enqueued on it; calls do not synchronise the stream, except
+ *    that the library may wait on the host for one of its OWN earlier pointer-table
+ *    uploads before re-using a staging slot.
+ *  - The library allocates only small device tables (layout chunk tables, per-plan
+ *    descriptors).  The Newton-Schulz workspace is caller-owned (muon_set_workspace).
+ *  - A context is bound to the device that was current in muon_create and must be used
+ *    with that device current; calls on one context must not overlap in time on the
+ *    host (one thread at a time), and device work of consecutive calls must be ordered
+ *    by the caller (same stream or events) because they share the workspace.
+ */
+#ifndef MUON_B200_H_
+#define MUON_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ------------------------------------------------------------------ status codes */
+#define MUON_OK                      0
+#define MUON_ERR_INVALID_ARG        -1   /* null pointer, negative count, bad enum, misaligned buffer      */
+#define MUON_ERR_BAD_LAYOUT         -2   /* segment table does not describe a valid flat-shard layout      */
+#define MUON_ERR_UNSUPPORTED        -3   /* legal request the library does not implement                   */
+#define MUON_ERR_WORKSPACE_TOO_SMALL -4  /* muon_set_workspace not called, or buffer smaller than required  */
+#define MUON_ERR_CUDA               -5   /* a CUDA runtime/driver call failed (no usable device, launch...) */
+#define MUON_ERR_DEVICE_TIMEOUT     -6   /* a bounded device-side wait gave up (see muon_last_device_status) */
+
+/* ------------------------------------------------------------------ enums */
+#define MUON_DTYPE_BF16 0
+#define MUON_DTYPE_FP32 1
+
+#define MUON_NS_BF16 0   /* bf16 operands, fp32 accumulation on the tensor cores (Section 6.3: "bf16 arithmetic") */
+#define MUON_NS_FP32 1   /* every product and intermediate in fp32 (no counterpart in the paper; accuracy anchor)  */
+
+#define MUON_ENGINE_TENSOR    0
+#define MUON_ENGINE_CUDA_CORE 1
+
+/* flags of muon_orthogonalize_batched */
+#define MUON_ORTHO_NO_NORMALIZE 1u  /* treat the input as X_0 already (r = 1); used for single-step checks */
+
+typedef struct muon_ctx    muon_ctx_t;
+typedef struct muon_layout muon_layout_t;
+
+/* Shape of one dense row-major matrix (Section 2.3: W in R^{m x n}). */
+typedef struct { int32_t rows, cols; } muon_shape_t;
+
+/* One contiguous piece of a matrix inside the flat buffer: elements
+ * [elem_begin, elem_begin+elem_count) of the row-major linearisation of matrix
+ * `matrix` live at flat[flat_offset, flat_offset+elem_count).  Units: elements. */
+typedef struct {
+  int32_t matrix;
+  int32_t reserved;      /* must be 0 */
+  int64_t elem_begin;
+  int64_t elem_count;
+  int64_t flat_offset;
+} muon_segment_t;
+
+/* Flat FSDP-style shard buffer (Sections 5.2-5.3 buffer conventions, Section 6.2 step 1:
+ * "aligned staging buffer (bf16, uneven splits supported)"): num_shards consecutive
+ * shards of shard_len elements each; segment starts are multiples of align_elems;
+ * everything not covered by a segment is padding that is never read nor written. */
+typedef struct {
+  int32_t elem_size;              /* 2 (bf16) or 4 (fp32) bytes per element                */
+  int32_t align_elems;            /* > 0; every flat_offset must be a multiple of it        */
+  int32_t num_shards;             /* >= 1                                                   */
+  int32_t num_matrices;           /* >= 0                                                   */
+  int64_t shard_len;              /* elements per shard, multiple of align_elems            */
+  const muon_shape_t*   shapes;   /* host, num_matrices entries                             */
+  int64_t num_segments;
+  const muon_segment_t* segments; /* host, num_segments entries; copied by muon_layout_create */
+} muon_layout_desc_t;
+
+typedef struct {
+  int32_t grad_dtype;      /* MUON_DTYPE_BF16 | MUON_DTYPE_FP32: element type of `grads`                     */
+  int32_t ns_precision;    /* MUON_NS_BF16 | MUON_NS_FP32                                                    */
+  int32_t nesterov;        /* 1: u = G + mu*M' (Section 7 set-up), 0: u = M'                                 */
+  int32_t coeffs_per_step; /* 0: coeffs[3] used at every step; 1: coeffs[3*ns_steps], (a_k,b_k,c_k) per step */
+  float   eps;             /* epsilon of Eq. 1, added to the Frobenius norm; default 1e-7                    */
+  int32_t engine;          /* MUON_ENGINE_TENSOR (default) | MUON_ENGINE_CUDA_CORE (bf16 products on CUDA cores;   */
+                           /* slow cross-check of the tensor-core engine; fp32 NS always runs on CUDA cores)        */
+  int64_t chunk_elems;     /* batching cap in elements per batched NS invocation; default 1<<29 (Section 6.3) */
+} muon_options_t;
+
+/* Fills *opt with the defaults: bf16 grads, bf16 NS, Nesterov, constant coefficients, eps 1e-7, cap 2^29. */
+int muon_default_options(muon_options_t* opt);
+
+/* Creates a context on the current CUDA device.  MUON_ERR_CUDA when no device is usable
+ * (the library never falls back to the CPU). */
+int  muon_create(muon_ctx_t** ctx, const muon_options_t* opt);
+void muon_destroy(muon_ctx_t* ctx);
+
+/* Bytes of device workspace that muon_step_batched / muon_orthogonalize_batched need for
+ * this list of shapes under these options ("workspace allocated once per batched
+ * invocation", Section 6.3).  Pure host arithmetic; needs no device. */
+int muon_workspace_bytes(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count, size_t* bytes);
+
+/* Hands the library a caller-owned device buffer (256-byte aligned) used as workspace by
+ * every later call on this context until replaced.  The caller keeps ownership. */
+int muon_set_workspace(muon_ctx_t* ctx, void* dev_ptr, size_t bytes);
+
+/* Host-only description of how a shape list is batched: matrices are grouped by core
+ * shape (min(m,n), max(m,n)) -- the paper's shape-fused batching, Section 6.3 -- and each
+ * group is cut into chunks of at most chunk_elems elements (at least one matrix).
+ * chunk_of[i] receives the chunk index of matrix i (may be NULL); *num_chunks the count. */
+int muon_plan_describe(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count,
+                       int32_t* num_chunks, int32_t* chunk_of);
+
+/* Validates a layout description on the host (no device needed): every element of every
+ * matrix covered exactly once; segments inside one shard, pairwise disjoint in the flat
+ * buffer, starts aligned; reserved fields zero.  MUON_ERR_BAD_LAYOUT otherwise. */
+int muon_layout_validate(const muon_layout_desc_t* desc);
+
+/* Validates and uploads a layout; the handle is immutable and may be used by any number of
+ * materialize/scatter calls.  `desc` and what it points to may be freed afterwards. */
+int  muon_layout_create(muon_ctx_t* ctx, const muon_layout_desc_t* desc, muon_layout_t** out);
+void muon_layout_destroy(muon_layout_t* layout);
+
+/* muon_materialize: unpack the flat shard buffer into whole matrices -- the copy-out half
+ * of a fused gather (Section 6.2 step 1; the pack/unpack passes of Section 5.2).
+ *   flat_buf : device, num_shards*shard_len elements of elem_size bytes, 16-byte aligned
+ *   matrices : host array [num_matrices] of device pointers, each rows*cols elements
+ * Bit-exact byte movement; padding is never read. */
+int muon_materialize(muon_ctx_t* ctx, const void* flat_buf, const muon_layout_t* layout,
+                     void* const* matrices, void* stream);
+
+/* muon_scatter: the inverse -- pack whole matrices into the flat shard buffer (the pack
+ * before the relay broadcast, Section 6.2 step 3).  Padding elements of flat_buf are
+ * never written. */
+int muon_scatter(muon_ctx_t* ctx, void* flat_buf, const muon_layout_t* layout,
+                 const void* const* matrices, void* stream);
+
+/* muon_step_batched: one Muon update of `count` independent matrices (Section 2.3, Eq. 1;
+ * Algorithm 2 "momentum update -> batched NS -> apply"):
+ *     M <- mu*M + G;  u = G + mu*M (Nesterov) or M;  U = cast(u)
+ *     X_0 = U / (||U||_F + eps), run on U^T when rows > cols (transpose-first, Section 6.3)
+ *     X_{k+1} = a_k X_k + (b_k A + c_k A^2) X_k,  A = X_k X_k^T,  k = 0..ns_steps-1
+ *     W <- W (1 - lr*wd) - lr * 0.2 sqrt(max(rows, cols)) * X_ns
+ *   params, momenta : host arrays [count] of device pointers to fp32 matrices (in/out)
+ *   grads           : host array  [count] of device pointers, element type opt.grad_dtype
+ *   shapes          : host, [count]; a matrix with rows==0 or cols==0 is skipped
+ *   coeffs          : host, 3 floats (or 3*ns_steps when opt.coeffs_per_step)
+ * All matrix pointers must be 16-byte aligned.  Matrices are batched by core shape; the
+ * results do not depend on how they are batched (bit-identical run to run). */
+int muon_step_batched(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
+                      const muon_shape_t* shapes, int32_t count, float lr, float mu, float wd,
+                      int32_t ns_steps, const float* coeffs, void* stream);
+
+/* muon_orthogonalize_batched: only the Newton-Schulz part of the step (Eq. 1) on given
+ * inputs -- for per-kernel parity checks and timing.  Element type of in/out is bf16 under
+ * MUON_NS_BF16 and fp32 under MUON_NS_FP32; out[i] has the shape of in[i]; in and out may
+ * not alias. */
+int muon_orthogonalize_batched(muon_ctx_t* ctx, const void* const* in, void* const* out,
+                               const muon_shape_t* shapes, int32_t count,
+                               int32_t ns_steps, const float* coeffs, uint32_t flags, void* stream);
+
+/* Device-side status word: the tensor-core pipeline bounds every wait on a barrier; a wait
+ * that gives up records a non-zero code here and the kernel exits cleanly.  Reads the word
+ * after synchronising `stream`; 0 = no bounded wait ever expired on this context. */
+int muon_last_device_status(muon_ctx_t* ctx, void* stream, int32_t* status);
+
+/* Phase timing (off by default).  When on, the library brackets each phase with CUDA
+ * events on the caller's stream; muon_profile_read synchronises those events and adds up,
+ * per phase, device milliseconds and kernel launches since the last muon_profile_reset. */
+#define MUON_PHASE_MOMENTUM 0   /* fused momentum + Nesterov + cast + sum of squares, and the norm finalise */
+#define MUON_PHASE_NS       1   /* the Newton-Schulz product kernels                                      */
+#define MUON_PHASE_UPDATE   2   /* fused scaled, weight-decayed update                                    */
+#define MUON_PHASE_GATHER   3   /* muon_materialize                                                       */
+#define MUON_PHASE_SCATTER  4   /* muon_scatter                                                           */
+#define MUON_NUM_PHASES     5
+int muon_profile_enable(muon_ctx_t* ctx, int32_t on);
+int muon_profile_reset(muon_ctx_t* ctx);
+int muon_profile_read(muon_ctx_t* ctx, int32_t phase, double* ms, int64_t* launches);
+
+/* Total kernels this context has launched since creation. */
+int64_t muon_launch_count(const muon_ctx_t* ctx);
+
+const char* muon_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MUON_B200_H_ */

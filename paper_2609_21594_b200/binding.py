@@ -1,0 +1,254 @@
+"""ctypes binding of libmuon_b200.so: argument marshalling only.
+
+Every function mirrors one entry point of include/muon_b200.h under the same name.  Tensors
+are torch CUDA tensors used purely as device memory; no arithmetic happens here.  If the
+shared library is missing the import of this module fails loudly -- there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence, Tuple
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmuon_b200.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_21594_b200.build` "
+                      "(there is no CPU or PyTorch fallback)")
+
+lib = C.CDLL(LIB_PATH)
+
+OK, ERR_INVALID_ARG, ERR_BAD_LAYOUT, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_DEVICE_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
+DTYPE_BF16, DTYPE_FP32 = 0, 1
+NS_BF16, NS_FP32 = 0, 1
+ENGINE_TENSOR, ENGINE_CUDA_CORE = 0, 1
+ORTHO_NO_NORMALIZE = 1
+PHASE_MOMENTUM, PHASE_NS, PHASE_UPDATE, PHASE_GATHER, PHASE_SCATTER = range(5)
+PHASE_NAMES = ("momentum", "ns", "update", "gather", "scatter")
+
+
+class Shape(C.Structure):
+    _fields_ = [("rows", C.c_int32), ("cols", C.c_int32)]
+
+
+class Segment(C.Structure):
+    _fields_ = [("matrix", C.c_int32), ("reserved", C.c_int32), ("elem_begin", C.c_int64),
+                ("elem_count", C.c_int64), ("flat_offset", C.c_int64)]
+
+
+class LayoutDesc(C.Structure):
+    _fields_ = [("elem_size", C.c_int32), ("align_elems", C.c_int32), ("num_shards", C.c_int32),
+                ("num_matrices", C.c_int32), ("shard_len", C.c_int64), ("shapes", C.POINTER(Shape)),
+                ("num_segments", C.c_int64), ("segments", C.POINTER(Segment))]
+
+
+class Options(C.Structure):
+    _fields_ = [("grad_dtype", C.c_int32), ("ns_precision", C.c_int32), ("nesterov", C.c_int32),
+                ("coeffs_per_step", C.c_int32), ("eps", C.c_float), ("engine", C.c_int32),
+                ("chunk_elems", C.c_int64)]
+
+
+_vp = C.c_void_p
+_sig = {
+    "muon_default_options": (C.c_int, [C.POINTER(Options)]),
+    "muon_create": (C.c_int, [C.POINTER(_vp), C.POINTER(Options)]),
+    "muon_destroy": (None, [_vp]),
+    "muon_workspace_bytes": (C.c_int, [C.POINTER(Options), C.POINTER(Shape), C.c_int32, C.POINTER(C.c_size_t)]),
+    "muon_set_workspace": (C.c_int, [_vp, _vp, C.c_size_t]),
+    "muon_plan_describe": (C.c_int, [C.POINTER(Options), C.POINTER(Shape), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
+    "muon_layout_validate": (C.c_int, [C.POINTER(LayoutDesc)]),
+    "muon_layout_create": (C.c_int, [_vp, C.POINTER(LayoutDesc), C.POINTER(_vp)]),
+    "muon_layout_destroy": (None, [_vp]),
+    "muon_materialize": (C.c_int, [_vp, _vp, _vp, C.POINTER(_vp), _vp]),
+    "muon_scatter": (C.c_int, [_vp, _vp, _vp, C.POINTER(_vp), _vp]),
+    "muon_step_batched": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(Shape), C.c_int32,
+                                    C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
+    "muon_orthogonalize_batched": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(Shape), C.c_int32,
+                                             C.c_int32, C.POINTER(C.c_float), C.c_uint32, _vp]),
+    "muon_last_device_status": (C.c_int, [_vp, _vp, C.POINTER(C.c_int32)]),
+    "muon_profile_enable": (C.c_int, [_vp, C.c_int32]),
+    "muon_profile_reset": (C.c_int, [_vp]),
+    "muon_profile_read": (C.c_int, [_vp, C.c_int32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
+    "muon_launch_count": (C.c_int64, [_vp]),
+    "muon_status_string": (C.c_char_p, [C.c_int]),
+}
+EXPORTED = tuple(_sig)
+for _name, (_res, _args) in _sig.items():
+    _f = getattr(lib, _name)
+    _f.restype = _res
+    _f.argtypes = _args
+
+
+class MuonError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {lib.muon_status_string(code).decode()} ({code})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise MuonError(code, where)
+
+
+def _shapes(shapes: Sequence[Tuple[int, int]]):
+    arr = (Shape * max(1, len(shapes)))()
+    for i, (r, c) in enumerate(shapes):
+        arr[i].rows, arr[i].cols = int(r), int(c)
+    return arr
+
+
+def _ptrs(tensors) -> "C.Array":
+    arr = (_vp * max(1, len(tensors)))()
+    for i, t in enumerate(tensors):
+        arr[i] = None if t is None else (t if isinstance(t, int) else t.data_ptr())
+    return arr
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+def muon_default_options(**over) -> Options:
+    o = Options()
+    _check(lib.muon_default_options(C.byref(o)), "muon_default_options")
+    for k, v in over.items():
+        setattr(o, k, v)
+    return o
+
+
+def muon_workspace_bytes(opt: Options, shapes) -> int:
+    out = C.c_size_t(0)
+    _check(lib.muon_workspace_bytes(C.byref(opt), _shapes(shapes), len(shapes), C.byref(out)), "muon_workspace_bytes")
+    return int(out.value)
+
+
+def muon_plan_describe(opt: Options, shapes) -> Tuple[int, List[int]]:
+    n = C.c_int32(0)
+    chunk_of = (C.c_int32 * max(1, len(shapes)))()
+    _check(lib.muon_plan_describe(C.byref(opt), _shapes(shapes), len(shapes), C.byref(n), chunk_of), "muon_plan_describe")
+    return int(n.value), [int(chunk_of[i]) for i in range(len(shapes))]
+
+
+def make_layout_desc(layout, elem_size: int):
+    """Builds a LayoutDesc (plus the arrays it points to) from a workloads.Layout."""
+    shapes = _shapes(layout.shapes)
+    segs = (Segment * max(1, len(layout.segments)))()
+    for i, s in enumerate(layout.segments):
+        segs[i].matrix, segs[i].reserved = s.matrix, 0
+        segs[i].elem_begin, segs[i].elem_count, segs[i].flat_offset = s.elem_begin, s.elem_count, s.flat_offset
+    d = LayoutDesc(elem_size, layout.align, layout.num_shards, len(layout.shapes), layout.shard_len,
+                   shapes, len(layout.segments), segs)
+    d._keep = (shapes, segs)
+    return d
+
+
+def muon_layout_validate(desc: LayoutDesc) -> int:
+    return int(lib.muon_layout_validate(C.byref(desc)))
+
+
+class Layout:
+    """Owner of a muon_layout_t handle."""
+
+    def __init__(self, ctx: "Context", layout, elem_size: int):
+        self.desc = make_layout_desc(layout, elem_size)
+        self.handle = _vp()
+        _check(lib.muon_layout_create(ctx.handle, C.byref(self.desc), C.byref(self.handle)), "muon_layout_create")
+
+    def close(self):
+        if self.handle:
+            lib.muon_layout_destroy(self.handle)
+            self.handle = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Context:
+    """Owner of a muon_ctx_t handle and (optionally) of a torch-allocated workspace."""
+
+    def __init__(self, opt: Optional[Options] = None):
+        self.opt = opt if opt is not None else muon_default_options()
+        self.handle = _vp()
+        _check(lib.muon_create(C.byref(self.handle), C.byref(self.opt)), "muon_create")
+        self._ws = None
+
+    def close(self):
+        if self.handle:
+            lib.muon_destroy(self.handle)
+            self.handle = _vp()
+            self._ws = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- workspace
+    def muon_set_workspace(self, tensor) -> None:
+        self._ws = tensor
+        _check(lib.muon_set_workspace(self.handle, tensor.data_ptr(), tensor.numel() * tensor.element_size()),
+               "muon_set_workspace")
+
+    def ensure_workspace(self, shapes) -> int:
+        """Allocates (through torch) a workspace large enough for `shapes`; returns its size."""
+        import torch
+
+        need = muon_workspace_bytes(self.opt, shapes)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = None
+            self.muon_set_workspace(torch.empty(max(need, 256), dtype=torch.uint8, device="cuda"))
+        return need
+
+    # -- layout path
+    def muon_materialize(self, flat, layout: Layout, matrices, stream=None) -> None:
+        _check(lib.muon_materialize(self.handle, flat.data_ptr(), layout.handle, _ptrs(matrices), _stream(stream)),
+               "muon_materialize")
+
+    def muon_scatter(self, flat, layout: Layout, matrices, stream=None) -> None:
+        _check(lib.muon_scatter(self.handle, flat.data_ptr(), layout.handle, _ptrs(matrices), _stream(stream)),
+               "muon_scatter")
+
+    # -- compute
+    def muon_step_batched(self, params, grads, momenta, shapes, lr, mu, wd, ns_steps, coeffs, stream=None) -> None:
+        co = (C.c_float * len(coeffs))(*[float(c) for c in coeffs])
+        _check(lib.muon_step_batched(self.handle, _ptrs(params), _ptrs(grads), _ptrs(momenta), _shapes(shapes),
+                                     len(shapes), lr, mu, wd, ns_steps, co, _stream(stream)), "muon_step_batched")
+
+    def muon_orthogonalize_batched(self, inputs, outputs, shapes, ns_steps, coeffs, flags=0, stream=None) -> None:
+        co = (C.c_float * len(coeffs))(*[float(c) for c in coeffs])
+        _check(lib.muon_orthogonalize_batched(self.handle, _ptrs(inputs), _ptrs(outputs), _shapes(shapes), len(shapes),
+                                              ns_steps, co, flags, _stream(stream)), "muon_orthogonalize_batched")
+
+    def muon_last_device_status(self, stream=None) -> int:
+        v = C.c_int32(0)
+        _check(lib.muon_last_device_status(self.handle, _stream(stream), C.byref(v)), "muon_last_device_status")
+        return int(v.value)
+
+    # -- profiling
+    def muon_profile_enable(self, on: bool) -> None:
+        _check(lib.muon_profile_enable(self.handle, 1 if on else 0), "muon_profile_enable")
+
+    def muon_profile_reset(self) -> None:
+        _check(lib.muon_profile_reset(self.handle), "muon_profile_reset")
+
+    def muon_profile_read(self):
+        out = {}
+        for ph, name in enumerate(PHASE_NAMES):
+            ms, n = C.c_double(0), C.c_int64(0)
+            _check(lib.muon_profile_read(self.handle, ph, C.byref(ms), C.byref(n)), "muon_profile_read")
+            out[name] = (float(ms.value), int(n.value))
+        return out
+
+    def muon_launch_count(self) -> int:
+        return int(lib.muon_launch_count(self.handle))

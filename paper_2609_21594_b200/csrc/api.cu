@@ -1,0 +1,516 @@
+// extern "C" entry points of libmuon_b200: argument validation, plan lookup, kernel sequencing.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+
+using namespace muon;
+
+namespace {
+
+struct DeviceGuardCheck {
+  static bool ok(const muon_ctx* ctx) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == ctx->device;
+  }
+};
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+bool valid_options(const muon_options_t& o) {
+  if (o.grad_dtype != MUON_DTYPE_BF16 && o.grad_dtype != MUON_DTYPE_FP32) return false;
+  if (o.ns_precision != MUON_NS_BF16 && o.ns_precision != MUON_NS_FP32) return false;
+  if (o.engine != MUON_ENGINE_TENSOR && o.engine != MUON_ENGINE_CUDA_CORE) return false;
+  if (o.nesterov != 0 && o.nesterov != 1) return false;
+  if (o.coeffs_per_step != 0 && o.coeffs_per_step != 1) return false;
+  if (!(o.eps >= 0.f) || !std::isfinite(o.eps)) return false;
+  if (o.chunk_elems < 0) return false;
+  return true;
+}
+
+// Stream-ordered upload of a small host table through a ring of pinned staging slots.
+int upload(muon_ctx* ctx, const void* src, size_t bytes, cudaStream_t st, void** dev_out) {
+  StagingSlot& s = ctx->slots[ctx->next_slot];
+  ctx->next_slot = (ctx->next_slot + 1) % 4;
+  if (s.used && cudaEventSynchronize(s.ev) != cudaSuccess) return MUON_ERR_CUDA;
+  if (s.cap < bytes) {
+    // a kernel of an earlier call may still read the old device table: drain before freeing it
+    if (s.dev && cudaDeviceSynchronize() != cudaSuccess) return MUON_ERR_CUDA;
+    if (s.host) cudaFreeHost(s.host);
+    if (s.dev) cudaFree(s.dev);
+    s.host = s.dev = nullptr;
+    s.cap = 0;
+    const size_t cap = (bytes + 4095) / 4096 * 4096;
+    if (cudaMallocHost(&s.host, cap) != cudaSuccess) return MUON_ERR_CUDA;
+    if (cudaMalloc(&s.dev, cap) != cudaSuccess) return MUON_ERR_CUDA;
+    s.cap = cap;
+  }
+  if (!s.ev && cudaEventCreateWithFlags(&s.ev, cudaEventDisableTiming) != cudaSuccess) return MUON_ERR_CUDA;
+  std::memcpy(s.host, src, bytes);
+  if (cudaMemcpyAsync(s.dev, s.host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return MUON_ERR_CUDA;
+  if (cudaEventRecord(s.ev, st) != cudaSuccess) return MUON_ERR_CUDA;
+  s.used = true;
+  *dev_out = s.dev;
+  return MUON_OK;
+}
+
+cudaEvent_t get_event(muon_ctx* ctx) {
+  if (!ctx->event_pool.empty()) {
+    cudaEvent_t e = ctx->event_pool.back();
+    ctx->event_pool.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+struct Span {
+  muon_ctx* ctx;
+  int idx = -1;
+  cudaStream_t st;
+  Span(muon_ctx* c, int phase, cudaStream_t s) : ctx(c), st(s) {
+    if (!c->profiling) return;
+    PhaseSpan ps{phase, get_event(c), get_event(c), 0};
+    if (!ps.a || !ps.b) return;
+    cudaEventRecord(ps.a, st);
+    c->spans.push_back(ps);
+    idx = int(c->spans.size()) - 1;
+  }
+  void end(int64_t launches) {
+    if (idx < 0) return;
+    cudaEventRecord(ctx->spans[size_t(idx)].b, st);
+    ctx->spans[size_t(idx)].launches = launches;
+    idx = -1;
+  }
+};
+
+Plan* get_plan(muon_ctx* ctx, const muon_shape_t* shapes, int32_t count, int* status) {
+  std::string key(reinterpret_cast<const char*>(shapes), size_t(count) * sizeof(muon_shape_t));
+  auto it = ctx->plans.find(key);
+  if (it != ctx->plans.end()) {
+    *status = MUON_OK;
+    return &it->second;
+  }
+  Plan p;
+  *status = build_plan(ctx->opt, shapes, count, &p);
+  if (*status != MUON_OK) return nullptr;
+  if (ctx->plans.size() > 64) ctx->plans.clear();
+  return &ctx->plans.emplace(std::move(key), std::move(p)).first->second;
+}
+
+int run_gemm(muon_ctx* ctx, const GemmArgs& g, cudaStream_t st) {
+  if (ctx->opt.ns_precision == MUON_NS_BF16 && ctx->opt.engine == MUON_ENGINE_TENSOR && tc_supported(g))
+    return launch_gemm_tc(ctx, g, st);
+  return launch_gemm_simt(g, ctx->opt.ns_precision, st);
+}
+
+struct ChunkRun {
+  int32_t momentum;     // 1: optimizer step, 0: orthogonalize only
+  int32_t normalize;
+  float lr, mu, wd;
+  int32_t ns_steps;
+  const float* coeffs;
+};
+
+int run_chunk(muon_ctx* ctx, const Chunk& ch, const MatDesc* d_descs, const ChunkRun& r, cudaStream_t st) {
+  const WsCarve w = carve_chunk(ctx->opt, ch);
+  char* base = static_cast<char*>(ctx->ws);
+  void* x0 = base + w.x0;
+  void* x1 = base + w.x1;
+  void* A = base + w.a;
+  void* B = base + w.b;
+  float* partials = reinterpret_cast<float*>(base + w.partials);
+  float* rnorm = reinterpret_cast<float*>(base + w.rnorm);
+  int n;
+  {
+    Span sp(ctx, MUON_PHASE_MOMENTUM, st);
+    StageArgs sa;
+    sa.descs = d_descs + ch.desc_begin;
+    sa.x = x0;
+    sa.partials = partials;
+    sa.rnorm = rnorm;
+    sa.count = ch.count;
+    sa.tiles_per_mat = ch.tiles_per_mat;
+    sa.s = ch.s; sa.l = ch.l; sa.ldx = ch.ldx;
+    sa.mu = r.mu; sa.eps = ctx->opt.eps;
+    sa.nesterov = ctx->opt.nesterov;
+    sa.grad_dtype = ctx->opt.grad_dtype;
+    sa.ns_precision = ctx->opt.ns_precision;
+    sa.momentum = r.momentum;
+    sa.normalize = r.normalize;
+    n = launch_stage(sa, st);
+    if (n < 0) return n;
+    ctx->launches += n;
+    sp.end(n);
+  }
+  void* cur = x0;
+  void* nxt = x1;
+  {
+    Span sp(ctx, MUON_PHASE_NS, st);
+    int64_t total = 0;
+    const int64_t sx = int64_t(ch.s) * ch.ldx, sa_ = int64_t(ch.s) * ch.lda;
+    for (int k = 0; k < r.ns_steps; ++k) {
+      const float* co = r.coeffs + (ctx->opt.coeffs_per_step ? 3 * k : 0);
+      GemmArgs g{};
+      // A = gamma * X X^T
+      g.p = cur; g.q = cur; g.d = nullptr; g.c = A;
+      g.m = ch.s; g.n = ch.s; g.kdim = ch.l;
+      g.ldp = ch.ldx; g.ldq = ch.ldx; g.ldc = ch.lda;
+      g.stride_p = sx; g.stride_q = sx; g.stride_c = sa_;
+      g.batch = ch.count; g.rnorm = rnorm; g.gamma_mode = (k == 0) ? 2 : 0;
+      g.alpha = 1.f; g.beta = 0.f; g.nn = 0; g.symmetric = 1;
+      if ((n = run_gemm(ctx, g, st)) < 0) return n;
+      total += n;
+      // B = b A + c A A^T   (A symmetric, so A A^T = A^2)
+      g.p = A; g.q = A; g.d = A; g.c = B;
+      g.kdim = ch.s; g.ldp = ch.lda; g.ldq = ch.lda;
+      g.stride_p = sa_; g.stride_q = sa_;
+      g.gamma_mode = 0; g.alpha = co[2]; g.beta = co[1];
+      if ((n = run_gemm(ctx, g, st)) < 0) return n;
+      total += n;
+      // X' = gamma * (a X + B X)
+      g.p = B; g.q = cur; g.d = cur; g.c = nxt;
+      g.m = ch.s; g.n = ch.l; g.kdim = ch.s;
+      g.ldp = ch.lda; g.ldq = ch.ldx; g.ldc = ch.ldx;
+      g.stride_p = sa_; g.stride_q = sx; g.stride_c = sx;
+      g.gamma_mode = (k == 0) ? 1 : 0; g.alpha = 1.f; g.beta = co[0]; g.nn = 1; g.symmetric = 0;
+      if ((n = run_gemm(ctx, g, st)) < 0) return n;
+      total += n;
+      void* t = cur; cur = nxt; nxt = t;
+    }
+    ctx->launches += total;
+    sp.end(total);
+  }
+  {
+    Span sp(ctx, MUON_PHASE_UPDATE, st);
+    ApplyArgs aa;
+    aa.descs = d_descs + ch.desc_begin;
+    aa.x = cur;
+    aa.count = ch.count;
+    aa.tiles_per_mat = ch.tiles_per_mat;
+    aa.s = ch.s; aa.l = ch.l; aa.ldx = ch.ldx;
+    aa.lr = r.lr; aa.wd = r.wd;
+    aa.ns_precision = ctx->opt.ns_precision;
+    aa.update = r.momentum;
+    n = launch_apply(aa, st);
+    if (n < 0) return n;
+    ctx->launches += n;
+    sp.end(n);
+  }
+  return MUON_OK;
+}
+
+int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const* m, const muon_shape_t* shapes,
+                int32_t count, const ChunkRun& r, cudaStream_t st) {
+  int status;
+  Plan* plan = get_plan(ctx, shapes, count, &status);
+  if (!plan) return status;
+  if (plan->live == 0) return MUON_OK;
+  if (!ctx->ws || ctx->ws_bytes < plan->ws_bytes) return MUON_ERR_WORKSPACE_TOO_SMALL;
+  std::vector<MatDesc> descs(size_t(plan->live));
+  for (const Chunk& ch : plan->chunks) {
+    for (int32_t j = 0; j < ch.count; ++j) {
+      const int32_t i = ch.mats[size_t(j)];
+      MatDesc& d = descs[size_t(ch.desc_begin + j)];
+      d.w = w[i];
+      d.g = g[i];
+      d.m = m ? m[i] : nullptr;
+      if (!d.w || !d.g || (r.momentum && !d.m)) return MUON_ERR_INVALID_ARG;
+      if (!aligned(d.w, 16) || !aligned(d.g, 16) || (d.m && !aligned(d.m, 16))) return MUON_ERR_INVALID_ARG;
+      d.rows = shapes[i].rows;
+      d.cols = shapes[i].cols;
+      d.transposed = d.rows > d.cols ? 1 : 0;
+      d.scale = float(0.2 * std::sqrt(double(std::max(d.rows, d.cols))));
+    }
+  }
+  void* d_descs = nullptr;
+  status = upload(ctx, descs.data(), descs.size() * sizeof(MatDesc), st, &d_descs);
+  if (status != MUON_OK) return status;
+  for (const Chunk& ch : plan->chunks) {
+    status = run_chunk(ctx, ch, static_cast<const MatDesc*>(d_descs), r, st);
+    if (status != MUON_OK) return status;
+  }
+  return MUON_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int muon_default_options(muon_options_t* opt) {
+  if (!opt) return MUON_ERR_INVALID_ARG;
+  opt->grad_dtype = MUON_DTYPE_BF16;
+  opt->ns_precision = MUON_NS_BF16;
+  opt->nesterov = 1;
+  opt->coeffs_per_step = 0;
+  opt->eps = 1e-7f;
+  opt->engine = MUON_ENGINE_TENSOR;
+  opt->chunk_elems = int64_t(1) << 29;
+  return MUON_OK;
+}
+
+int muon_create(muon_ctx_t** out, const muon_options_t* opt) {
+  if (!out) return MUON_ERR_INVALID_ARG;
+  *out = nullptr;
+  muon_options_t o;
+  muon_default_options(&o);
+  if (opt) o = *opt;
+  if (!valid_options(o)) return MUON_ERR_INVALID_ARG;
+  if (o.chunk_elems == 0) o.chunk_elems = int64_t(1) << 29;
+  int ndev = 0, dev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev <= 0) return MUON_ERR_CUDA;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MUON_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return MUON_ERR_CUDA;
+  if (prop.major != 10) return MUON_ERR_UNSUPPORTED;   // built for sm_100a only
+  muon_ctx* ctx = new (std::nothrow) muon_ctx();
+  if (!ctx) return MUON_ERR_CUDA;
+  ctx->opt = o;
+  ctx->device = dev;
+  if (cudaMalloc(&ctx->d_status, 256) != cudaSuccess || cudaMemset(ctx->d_status, 0, 256) != cudaSuccess) {
+    delete ctx;
+    return MUON_ERR_CUDA;
+  }
+  cudaDriverEntryPointQueryResult qres;
+  void* fn = nullptr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+      qres == cudaDriverEntryPointSuccess)
+    ctx->tmap_encode = fn;
+  *out = ctx;
+  return MUON_OK;
+}
+
+void muon_destroy(muon_ctx_t* ctx) {
+  if (!ctx) return;
+  cudaDeviceSynchronize();
+  for (StagingSlot& s : ctx->slots) {
+    if (s.host) cudaFreeHost(s.host);
+    if (s.dev) cudaFree(s.dev);
+    if (s.ev) cudaEventDestroy(s.ev);
+  }
+  for (PhaseSpan& p : ctx->spans) {
+    cudaEventDestroy(p.a);
+    cudaEventDestroy(p.b);
+  }
+  for (cudaEvent_t e : ctx->event_pool) cudaEventDestroy(e);
+  if (ctx->d_status) cudaFree(ctx->d_status);
+  delete ctx;
+}
+
+int muon_workspace_bytes(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count, size_t* bytes) {
+  if (!opt || !bytes || count < 0 || (count > 0 && !shapes)) return MUON_ERR_INVALID_ARG;
+  if (!valid_options(*opt)) return MUON_ERR_INVALID_ARG;
+  Plan p;
+  const int st = build_plan(*opt, shapes, count, &p);
+  if (st != MUON_OK) return st;
+  *bytes = p.ws_bytes;
+  return MUON_OK;
+}
+
+int muon_plan_describe(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count, int32_t* num_chunks,
+                       int32_t* chunk_of) {
+  if (!opt || !num_chunks || count < 0 || (count > 0 && !shapes)) return MUON_ERR_INVALID_ARG;
+  if (!valid_options(*opt)) return MUON_ERR_INVALID_ARG;
+  Plan p;
+  const int st = build_plan(*opt, shapes, count, &p);
+  if (st != MUON_OK) return st;
+  *num_chunks = int32_t(p.chunks.size());
+  if (chunk_of) {
+    for (int32_t i = 0; i < count; ++i) chunk_of[i] = -1;
+    for (size_t c = 0; c < p.chunks.size(); ++c)
+      for (int32_t i : p.chunks[c].mats) chunk_of[i] = int32_t(c);
+  }
+  return MUON_OK;
+}
+
+int muon_set_workspace(muon_ctx_t* ctx, void* dev_ptr, size_t bytes) {
+  if (!ctx) return MUON_ERR_INVALID_ARG;
+  if (bytes > 0 && (!dev_ptr || !aligned(dev_ptr, 256))) return MUON_ERR_INVALID_ARG;
+  ctx->ws = dev_ptr;
+  ctx->ws_bytes = bytes;
+  return MUON_OK;
+}
+
+int muon_layout_validate(const muon_layout_desc_t* desc) { return validate_layout_host(desc); }
+
+int muon_layout_create(muon_ctx_t* ctx, const muon_layout_desc_t* desc, muon_layout_t** out) {
+  if (!ctx || !out) return MUON_ERR_INVALID_ARG;
+  *out = nullptr;
+  const int st = validate_layout_host(desc);
+  if (st != MUON_OK) return st;
+  if (!DeviceGuardCheck::ok(ctx)) return MUON_ERR_CUDA;
+  std::vector<CopyItem> items;
+  for (int64_t k = 0; k < desc->num_segments; ++k) {
+    const muon_segment_t& s = desc->segments[k];
+    for (int64_t done = 0; done < s.elem_count; done += kCopyChunk) {
+      CopyItem it;
+      it.flat_offset = s.flat_offset + done;
+      it.elem_begin = s.elem_begin + done;
+      it.matrix = s.matrix;
+      it.count = int32_t(std::min<int64_t>(kCopyChunk, s.elem_count - done));
+      items.push_back(it);
+    }
+  }
+  muon_layout* L = new (std::nothrow) muon_layout();
+  if (!L) return MUON_ERR_CUDA;
+  L->desc = *desc;
+  L->shapes.assign(desc->shapes, desc->shapes + desc->num_matrices);
+  L->desc.shapes = nullptr;
+  L->desc.segments = nullptr;
+  L->num_items = int64_t(items.size());
+  L->device = ctx->device;
+  if (!items.empty()) {
+    if (cudaMalloc(&L->d_items, items.size() * sizeof(CopyItem)) != cudaSuccess ||
+        cudaMemcpy(L->d_items, items.data(), items.size() * sizeof(CopyItem), cudaMemcpyHostToDevice) != cudaSuccess) {
+      if (L->d_items) cudaFree(L->d_items);
+      delete L;
+      return MUON_ERR_CUDA;
+    }
+  }
+  *out = L;
+  return MUON_OK;
+}
+
+void muon_layout_destroy(muon_layout_t* L) {
+  if (!L) return;
+  if (L->d_items) {
+    cudaDeviceSynchronize();
+    cudaFree(L->d_items);
+  }
+  delete L;
+}
+
+static int copy_common(muon_ctx_t* ctx, void* flat, const muon_layout_t* L, void* const* mats, bool scatter, void* stream) {
+  if (!ctx || !L) return MUON_ERR_INVALID_ARG;
+  if (L->num_items == 0) return MUON_OK;
+  if (!flat || !mats || !aligned(flat, 16)) return MUON_ERR_INVALID_ARG;
+  if (!DeviceGuardCheck::ok(ctx) || L->device != ctx->device) return MUON_ERR_CUDA;
+  const size_t es = size_t(L->desc.elem_size);
+  for (int32_t i = 0; i < L->desc.num_matrices; ++i) {
+    const bool empty = L->shapes[size_t(i)].rows == 0 || L->shapes[size_t(i)].cols == 0;
+    if (!empty && (!mats[i] || !aligned(mats[i], es))) return MUON_ERR_INVALID_ARG;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  void* d_mats = nullptr;
+  int status = upload(ctx, mats, size_t(L->desc.num_matrices) * sizeof(void*), st, &d_mats);
+  if (status != MUON_OK) return status;
+  Span sp(ctx, scatter ? MUON_PHASE_SCATTER : MUON_PHASE_GATHER, st);
+  const int n = launch_copy(L->d_items, L->num_items, flat, static_cast<void* const*>(d_mats), int(es), scatter, st);
+  if (n < 0) return n;
+  ctx->launches += n;
+  sp.end(n);
+  return MUON_OK;
+}
+
+int muon_materialize(muon_ctx_t* ctx, const void* flat_buf, const muon_layout_t* layout, void* const* matrices,
+                     void* stream) {
+  return copy_common(ctx, const_cast<void*>(flat_buf), layout, matrices, false, stream);
+}
+
+int muon_scatter(muon_ctx_t* ctx, void* flat_buf, const muon_layout_t* layout, const void* const* matrices,
+                 void* stream) {
+  return copy_common(ctx, flat_buf, layout, const_cast<void* const*>(matrices), true, stream);
+}
+
+static int check_common(muon_ctx_t* ctx, const muon_shape_t* shapes, int32_t count, int32_t ns_steps, const float* coeffs) {
+  if (!ctx || count < 0) return MUON_ERR_INVALID_ARG;
+  if (count > 0 && !shapes) return MUON_ERR_INVALID_ARG;
+  if (ns_steps < 1 || ns_steps > 64 || !coeffs) return MUON_ERR_INVALID_ARG;
+  const int nco = ctx->opt.coeffs_per_step ? 3 * ns_steps : 3;
+  for (int i = 0; i < nco; ++i)
+    if (!std::isfinite(coeffs[i])) return MUON_ERR_INVALID_ARG;
+  if (!DeviceGuardCheck::ok(ctx)) return MUON_ERR_CUDA;
+  return MUON_OK;
+}
+
+int muon_step_batched(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
+                      const muon_shape_t* shapes, int32_t count, float lr, float mu, float wd, int32_t ns_steps,
+                      const float* coeffs, void* stream) {
+  int st = check_common(ctx, shapes, count, ns_steps, coeffs);
+  if (st != MUON_OK) return st;
+  if (count == 0) return MUON_OK;
+  if (!params || !grads || !momenta) return MUON_ERR_INVALID_ARG;
+  if (!std::isfinite(lr) || !std::isfinite(mu) || !std::isfinite(wd)) return MUON_ERR_INVALID_ARG;
+  ChunkRun r{1, 1, lr, mu, wd, ns_steps, coeffs};
+  return run_batched(ctx, params, grads, momenta, shapes, count, r, static_cast<cudaStream_t>(stream));
+}
+
+int muon_orthogonalize_batched(muon_ctx_t* ctx, const void* const* in, void* const* out, const muon_shape_t* shapes,
+                               int32_t count, int32_t ns_steps, const float* coeffs, uint32_t flags, void* stream) {
+  int st = check_common(ctx, shapes, count, ns_steps, coeffs);
+  if (st != MUON_OK) return st;
+  if (count == 0) return MUON_OK;
+  if (!in || !out || (flags & ~MUON_ORTHO_NO_NORMALIZE)) return MUON_ERR_INVALID_ARG;
+  for (int32_t i = 0; i < count; ++i)
+    if (shapes[i].rows > 0 && shapes[i].cols > 0 && in[i] == out[i]) return MUON_ERR_INVALID_ARG;
+  ChunkRun r{0, (flags & MUON_ORTHO_NO_NORMALIZE) ? 0 : 1, 0.f, 0.f, 0.f, ns_steps, coeffs};
+  return run_batched(ctx, out, in, nullptr, shapes, count, r, static_cast<cudaStream_t>(stream));
+}
+
+int muon_last_device_status(muon_ctx_t* ctx, void* stream, int32_t* status) {
+  if (!ctx || !status) return MUON_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t v = 0;
+  if (cudaMemcpyAsync(&v, ctx->d_status, sizeof(v), cudaMemcpyDeviceToHost, st) != cudaSuccess) return MUON_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return MUON_ERR_CUDA;
+  *status = v;
+  return MUON_OK;
+}
+
+int muon_profile_enable(muon_ctx_t* ctx, int32_t on) {
+  if (!ctx) return MUON_ERR_INVALID_ARG;
+  ctx->profiling = on != 0;
+  return MUON_OK;
+}
+
+static int drain_spans(muon_ctx_t* ctx) {
+  for (PhaseSpan& p : ctx->spans) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(p.b) != cudaSuccess || cudaEventElapsedTime(&ms, p.a, p.b) != cudaSuccess) return MUON_ERR_CUDA;
+    ctx->phase_ms[p.phase] += double(ms);
+    ctx->phase_launches[p.phase] += p.launches;
+    ctx->event_pool.push_back(p.a);
+    ctx->event_pool.push_back(p.b);
+  }
+  ctx->spans.clear();
+  return MUON_OK;
+}
+
+int muon_profile_reset(muon_ctx_t* ctx) {
+  if (!ctx) return MUON_ERR_INVALID_ARG;
+  const int st = drain_spans(ctx);
+  for (int i = 0; i < MUON_NUM_PHASES; ++i) {
+    ctx->phase_ms[i] = 0.0;
+    ctx->phase_launches[i] = 0;
+  }
+  return st;
+}
+
+int muon_profile_read(muon_ctx_t* ctx, int32_t phase, double* ms, int64_t* launches) {
+  if (!ctx || phase < 0 || phase >= MUON_NUM_PHASES) return MUON_ERR_INVALID_ARG;
+  const int st = drain_spans(ctx);
+  if (st != MUON_OK) return st;
+  if (ms) *ms = ctx->phase_ms[phase];
+  if (launches) *launches = ctx->phase_launches[phase];
+  return MUON_OK;
+}
+
+int64_t muon_launch_count(const muon_ctx_t* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* muon_status_string(int status) {
+  switch (status) {
+    case MUON_OK: return "ok";
+    case MUON_ERR_INVALID_ARG: return "invalid argument";
+    case MUON_ERR_BAD_LAYOUT: return "bad flat-shard layout";
+    case MUON_ERR_UNSUPPORTED: return "unsupported";
+    case MUON_ERR_WORKSPACE_TOO_SMALL: return "workspace missing or too small";
+    case MUON_ERR_CUDA: return "CUDA error or no usable sm_100 device";
+    case MUON_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,291 @@
+// Fused elementwise kernels around the Newton-Schulz engine.
+//   stage : M <- mu*M + G, u = G + mu*M (Nesterov), U = cast(u) written into the NS workspace in
+//           wide orientation (transposed through shared memory when rows > cols: the
+//           transpose-first rule of Section 6.3), plus per-tile sums of U^2
+//   norm  : r = 1 / (sqrt(sum U^2) + eps) per matrix, fixed-order reduction (Eq. 1, second line)
+//   apply : W <- W (1 - lr*wd) - lr * 0.2 sqrt(max(m,n)) * O, O read back through the transpose
+// All three are HBM-bound.  Reductions use a fixed shuffle/shared-memory tree and per-tile
+// partial sums, never floating-point atomics, so results are bit-identical run to run.
+#include "internal.h"
+
+namespace muon {
+
+namespace {
+
+constexpr int T = kElemTile;       // 64
+constexpr int PADT = T + 2;        // shared tile row pitch (elements)
+
+template <typename XT> struct XConv;
+template <> struct XConv<__nv_bfloat16> {
+  static __device__ __forceinline__ __nv_bfloat16 from(float v) { return __float2bfloat16_rn(v); }
+  static __device__ __forceinline__ float to(__nv_bfloat16 v) { return __bfloat162float(v); }
+};
+template <> struct XConv<float> {
+  static __device__ __forceinline__ float from(float v) { return v; }
+  static __device__ __forceinline__ float to(float v) { return v; }
+};
+
+template <typename GT> __device__ __forceinline__ float load_g(const GT* p);
+template <> __device__ __forceinline__ float load_g<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+template <> __device__ __forceinline__ float load_g<float>(const float* p) { return *p; }
+
+__device__ __forceinline__ float block_sum_256(float v, float* red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  const int w = threadIdx.x >> 5;
+  if ((threadIdx.x & 31) == 0) red[w] = v;
+  __syncthreads();
+  float t = 0.f;
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) t += red[i];
+  }
+  return t;  // valid in thread 0
+}
+
+// GT: gradient/input element type; XT: NS element type; MOM: momentum rule on/off.
+// Thread (ty = tid/16, tx = tid%16) handles 4 consecutive columns tx*4.. of rows ty, ty+16, ty+32, ty+48.
+template <typename GT, typename XT, bool MOM>
+__global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
+  __shared__ XT tile[T][PADT];
+  __shared__ float red[8];
+  const int mat = blockIdx.x / a.tiles_per_mat;
+  const int t = blockIdx.x - mat * a.tiles_per_mat;
+  const MatDesc d = a.descs[mat];
+  const int tiles_c = (d.cols + T - 1) / T;
+  const int r0 = (t / tiles_c) * T, c0 = (t % tiles_c) * T;
+  const GT* __restrict__ G = static_cast<const GT*>(d.g);
+  float* __restrict__ M = static_cast<float*>(d.m);
+  XT* __restrict__ X = static_cast<XT*>(a.x) + size_t(mat) * a.s * a.ldx;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const bool vec = (d.cols & 3) == 0;
+  float sum = 0.f;
+#pragma unroll
+  for (int pass = 0; pass < 4; ++pass) {
+    const int rr = ty + pass * 16, cc = tx * 4;
+    const int r = r0 + rr, c = c0 + cc;
+    float u[4] = {0.f, 0.f, 0.f, 0.f};
+    if (r < d.rows && c < d.cols) {
+      const size_t off = size_t(r) * d.cols + c;
+      float g[4], m[4] = {0.f, 0.f, 0.f, 0.f};
+      const int nv = min(4, d.cols - c);
+      if (vec) {
+        if (sizeof(GT) == 2) {
+          const uint2 raw = __ldcs(reinterpret_cast<const uint2*>(G + off));
+          const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+          const __nv_bfloat162 p1 = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+          g[0] = __low2float(p0); g[1] = __high2float(p0); g[2] = __low2float(p1); g[3] = __high2float(p1);
+        } else {
+          const float4 raw = __ldcs(reinterpret_cast<const float4*>(G + off));
+          g[0] = raw.x; g[1] = raw.y; g[2] = raw.z; g[3] = raw.w;
+        }
+        if (MOM) {
+          const float4 mv = __ldcs(reinterpret_cast<const float4*>(M + off));
+          m[0] = mv.x; m[1] = mv.y; m[2] = mv.z; m[3] = mv.w;
+        }
+      } else {
+        for (int i = 0; i < 4; ++i) {
+          g[i] = i < nv ? load_g<GT>(G + off + i) : 0.f;
+          if (MOM) m[i] = i < nv ? M[off + i] : 0.f;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (MOM) {
+          m[i] = a.mu * m[i] + g[i];
+          u[i] = a.nesterov ? g[i] + a.mu * m[i] : m[i];
+        } else {
+          u[i] = g[i];
+        }
+      }
+      if (MOM) {
+        if (vec) {
+          __stcs(reinterpret_cast<float4*>(M + off), make_float4(m[0], m[1], m[2], m[3]));
+        } else {
+          for (int i = 0; i < nv; ++i) M[off + i] = m[i];
+        }
+      }
+      alignas(16) XT xv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        xv[i] = XConv<XT>::from(u[i]);
+        const float q = XConv<XT>::to(xv[i]);
+        if (i < nv) sum += q * q;
+      }
+      if (!d.transposed) {
+        XT* dst = X + size_t(r) * a.ldx + c;   // ldx % 8 == 0 and c % 4 == 0: 8/16-byte aligned
+        if (nv == 4) {
+          if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(xv);
+          else *reinterpret_cast<float4*>(dst) = *reinterpret_cast<const float4*>(xv);
+        } else {
+          for (int i = 0; i < nv; ++i) dst[i] = xv[i];
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) tile[rr][cc + i] = xv[i];
+      }
+    }
+  }
+  if (d.transposed) {
+    __syncthreads();
+    // X holds the transpose: X[c][r].  Thread writes 4 consecutive r for one c.
+#pragma unroll
+    for (int pass = 0; pass < 4; ++pass) {
+      const int cc = ty + pass * 16, rr = tx * 4;
+      const int c = c0 + cc, r = r0 + rr;
+      if (c < d.cols && r < d.rows) {
+        alignas(16) XT xv[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) xv[i] = tile[rr + i][cc];
+        XT* dst = X + size_t(c) * a.ldx + r;
+        const int nv = min(4, d.rows - r);
+        if (nv == 4) {
+          if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(xv);
+          else *reinterpret_cast<float4*>(dst) = *reinterpret_cast<const float4*>(xv);
+        } else {
+          for (int i = 0; i < nv; ++i) dst[i] = xv[i];
+        }
+      }
+    }
+  }
+  const float tot = block_sum_256(sum, red);
+  if (threadIdx.x == 0) a.partials[blockIdx.x] = tot;
+}
+
+// One block per matrix: fixed-order sum of the tile partials in double, then r = 1/(sqrt(.)+eps).
+__global__ void __launch_bounds__(256) norm_kernel(const float* __restrict__ partials, float* __restrict__ rnorm,
+                                                   int tiles_per_mat, float eps, int normalize) {
+  __shared__ double red[256];
+  const float* p = partials + size_t(blockIdx.x) * tiles_per_mat;
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < tiles_per_mat; i += 256) acc += double(p[i]);
+  red[threadIdx.x] = acc;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (int(threadIdx.x) < o) red[threadIdx.x] += red[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) rnorm[blockIdx.x] = normalize ? float(1.0 / (sqrt(red[0]) + double(eps))) : 1.0f;
+}
+
+// XT: NS element type; UPD: 1 = weight update, 0 = plain store of O into d.w (element type XT).
+template <typename XT, bool UPD>
+__global__ void __launch_bounds__(256) apply_kernel(ApplyArgs a) {
+  __shared__ XT tile[T][PADT];
+  const int mat = blockIdx.x / a.tiles_per_mat;
+  const int t = blockIdx.x - mat * a.tiles_per_mat;
+  const MatDesc d = a.descs[mat];
+  const int tiles_c = (d.cols + T - 1) / T;
+  const int r0 = (t / tiles_c) * T, c0 = (t % tiles_c) * T;
+  const XT* __restrict__ X = static_cast<const XT*>(a.x) + size_t(mat) * a.s * a.ldx;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  if (d.transposed) {
+    // load X[c][r] coalesced along r, then read it back transposed
+#pragma unroll
+    for (int pass = 0; pass < 4; ++pass) {
+      const int cc = ty + pass * 16, rr = tx * 4;
+      const int c = c0 + cc, r = r0 + rr;
+      if (c < d.cols && r < d.rows) {
+        const XT* src = X + size_t(c) * a.ldx + r;
+        const int nv = min(4, d.rows - r);
+        alignas(16) XT xv[4];
+        if (nv == 4) {
+          if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(xv) = *reinterpret_cast<const uint2*>(src);
+          else *reinterpret_cast<float4*>(xv) = *reinterpret_cast<const float4*>(src);
+        } else {
+          for (int i = 0; i < 4; ++i) xv[i] = i < nv ? src[i] : XConv<XT>::from(0.f);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) tile[rr + i][cc] = xv[i];
+      }
+    }
+    __syncthreads();
+  }
+  const float decay = 1.0f - a.lr * a.wd;
+  const float step = a.lr * d.scale;
+  const bool vec = (d.cols & 3) == 0;
+#pragma unroll
+  for (int pass = 0; pass < 4; ++pass) {
+    const int rr = ty + pass * 16, cc = tx * 4;
+    const int r = r0 + rr, c = c0 + cc;
+    if (r < d.rows && c < d.cols) {
+      const int nv = min(4, d.cols - c);
+      alignas(16) XT xv[4];
+      if (d.transposed) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) xv[i] = tile[rr][cc + i];
+      } else {
+        const XT* src = X + size_t(r) * a.ldx + c;
+        if (nv == 4) {
+          if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(xv) = *reinterpret_cast<const uint2*>(src);
+          else *reinterpret_cast<float4*>(xv) = *reinterpret_cast<const float4*>(src);
+        } else {
+          for (int i = 0; i < 4; ++i) xv[i] = i < nv ? src[i] : XConv<XT>::from(0.f);
+        }
+      }
+      const size_t off = size_t(r) * d.cols + c;
+      if (UPD) {
+        float* W = static_cast<float*>(d.w);
+        if (vec) {
+          float4 w = __ldcs(reinterpret_cast<const float4*>(W + off));
+          w.x = w.x * decay - step * XConv<XT>::to(xv[0]);
+          w.y = w.y * decay - step * XConv<XT>::to(xv[1]);
+          w.z = w.z * decay - step * XConv<XT>::to(xv[2]);
+          w.w = w.w * decay - step * XConv<XT>::to(xv[3]);
+          __stcs(reinterpret_cast<float4*>(W + off), w);
+        } else {
+          for (int i = 0; i < nv; ++i) W[off + i] = W[off + i] * decay - step * XConv<XT>::to(xv[i]);
+        }
+      } else {
+        XT* O = static_cast<XT*>(d.w);
+        if (vec) {
+          if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(O + off) = *reinterpret_cast<const uint2*>(xv);
+          else *reinterpret_cast<float4*>(O + off) = *reinterpret_cast<const float4*>(xv);
+        } else {
+          for (int i = 0; i < nv; ++i) O[off + i] = xv[i];
+        }
+      }
+    }
+  }
+}
+
+}  // namespace
+
+int launch_stage(const StageArgs& a, cudaStream_t st) {
+  const int64_t blocks = int64_t(a.count) * a.tiles_per_mat;
+  if (blocks == 0) return 0;
+  if (blocks > 0x7fffffffLL) return MUON_ERR_UNSUPPORTED;
+  const unsigned g = unsigned(blocks);
+  const bool xbf = a.ns_precision == MUON_NS_BF16;
+  if (a.momentum) {
+    const bool gbf = a.grad_dtype == MUON_DTYPE_BF16;
+    if (gbf && xbf) stage_kernel<__nv_bfloat16, __nv_bfloat16, true><<<g, 256, 0, st>>>(a);
+    else if (gbf && !xbf) stage_kernel<__nv_bfloat16, float, true><<<g, 256, 0, st>>>(a);
+    else if (!gbf && xbf) stage_kernel<float, __nv_bfloat16, true><<<g, 256, 0, st>>>(a);
+    else stage_kernel<float, float, true><<<g, 256, 0, st>>>(a);
+  } else {
+    if (xbf) stage_kernel<__nv_bfloat16, __nv_bfloat16, false><<<g, 256, 0, st>>>(a);
+    else stage_kernel<float, float, false><<<g, 256, 0, st>>>(a);
+  }
+  if (cudaGetLastError() != cudaSuccess) return MUON_ERR_CUDA;
+  norm_kernel<<<unsigned(a.count), 256, 0, st>>>(a.partials, a.rnorm, a.tiles_per_mat, a.eps, a.normalize);
+  return cudaGetLastError() == cudaSuccess ? 2 : MUON_ERR_CUDA;
+}
+
+int launch_apply(const ApplyArgs& a, cudaStream_t st) {
+  const int64_t blocks = int64_t(a.count) * a.tiles_per_mat;
+  if (blocks == 0) return 0;
+  if (blocks > 0x7fffffffLL) return MUON_ERR_UNSUPPORTED;
+  const unsigned g = unsigned(blocks);
+  const bool xbf = a.ns_precision == MUON_NS_BF16;
+  if (a.update) {
+    if (xbf) apply_kernel<__nv_bfloat16, true><<<g, 256, 0, st>>>(a);
+    else apply_kernel<float, true><<<g, 256, 0, st>>>(a);
+  } else {
+    if (xbf) apply_kernel<__nv_bfloat16, false><<<g, 256, 0, st>>>(a);
+    else apply_kernel<float, false><<<g, 256, 0, st>>>(a);
+  }
+  return cudaGetLastError() == cudaSuccess ? 1 : MUON_ERR_CUDA;
+}
+
+}  // namespace muon

@@ -1,0 +1,296 @@
+"""GPU parity of the Muon step against the CPU oracle, element by element, through the C ABI.
+
+Tolerances (relative Frobenius error per matrix): bf16 Newton-Schulz vs the bf16-emulating oracle
+<= 1e-2; fp32 mode vs the fp64 oracle <= 1e-4; a single teacher-forced NS step <= 2e-3; momentum
+and the update are compared in fp32 precision (1e-6).  Parity is measured on O (the NS output),
+on the stored momentum M' and on dW = W' - W, never only on W'.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import muon_oracle as orc
+from paper_2609_21594_b200 import workloads as wl
+from gpu_util import QUINTIC, bf16_input, dev_f32, host_f64, rel
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 1e-2
+TOL_FP32 = 1e-4
+TOL_SINGLE_STEP = 2e-3
+ENGINES = ["tensor", "cuda_core"]
+
+
+def _ctx(mb, precision="bf16", engine="tensor", grad="bf16", **kw):
+    opt = mb.muon_default_options(
+        ns_precision=mb.NS_BF16 if precision == "bf16" else mb.NS_FP32,
+        engine=mb.ENGINE_TENSOR if engine == "tensor" else mb.ENGINE_CUDA_CORE,
+        grad_dtype=mb.DTYPE_BF16 if grad == "bf16" else mb.DTYPE_FP32, **kw)
+    return mb.Context(opt)
+
+
+def _ortho(mb, ctx, mats_np, steps=5, coeffs=QUINTIC, flags=0):
+    """Runs muon_orthogonalize_batched; returns (outputs as float64, inputs as float64 of the device values)."""
+    bf = ctx.opt.ns_precision == mb.NS_BF16
+    ins, vals = [], []
+    for x in mats_np:
+        if bf:
+            t, v = bf16_input(x.astype(np.float32))
+        else:
+            t, v = dev_f32(x), x.astype(np.float32).astype(np.float64)
+        ins.append(t)
+        vals.append(v)
+    outs = [torch.full_like(t, float("nan")) for t in ins]
+    shapes = [tuple(x.shape) for x in mats_np]
+    ctx.ensure_workspace(shapes)
+    ctx.muon_orthogonalize_batched(ins, outs, shapes, steps, coeffs, flags)
+    torch.cuda.synchronize()
+    assert ctx.muon_last_device_status() == 0
+    return [host_f64(o) for o in outs], vals
+
+
+# ----------------------------------------------------------------------------- Newton-Schulz alone
+@pytest.mark.parametrize("engine", ENGINES)
+def test_ns_bf16_tiny_config_vs_oracle(engine):
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "bf16", engine)
+    shapes = wl.shapes_tiny()
+    mats = [wl.grad_np("tiny", 0, i, s) for i, s in enumerate(shapes)]
+    outs, vals = _ortho(mb, ctx, mats)
+    for i, (o, v) in enumerate(zip(outs, vals)):
+        ref = orc.newton_schulz(v, 5, QUINTIC, 1e-7, "bf16")
+        assert rel(o, ref) <= TOL_BF16, (i, shapes[i], rel(o, ref))
+        hi = orc.newton_schulz(v, 5, QUINTIC, 1e-7, "fp64")
+        assert rel(o, hi) <= 1.5 * rel(ref, hi) + 2e-3
+    ctx.close()
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_ns_bf16_ragged_shapes_vs_oracle(engine):
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "bf16", engine)
+    shapes = [(37, 53), (130, 7), (5, 1000), (1, 1), (300, 129), (129, 300), (200, 264), (8, 8), (1, 77), (77, 1)]
+    mats = [wl.grad_np("ragged", 0, i, s) for i, s in enumerate(shapes)]
+    outs, vals = _ortho(mb, ctx, mats)
+    for i, (o, v) in enumerate(zip(outs, vals)):
+        assert np.isfinite(o).all()
+        ref = orc.newton_schulz(v, 5, QUINTIC, 1e-7, "bf16")
+        assert rel(o, ref) <= TOL_BF16, (i, shapes[i], rel(o, ref))
+    ctx.close()
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+@pytest.mark.parametrize("shape", [(256, 256), (256, 1024), (1024, 256), (384, 640), (200, 264)])
+def test_ns_single_step_teacher_forced(engine, shape):
+    """Feed the oracle's bf16 X_k to one device NS step and compare with the oracle's X_{k+1}: the sharp,
+    chaos-free check of every product and epilogue."""
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "bf16", engine)
+    G = orc.bf16_rne(wl.grad_np("teacher", 0, shape[0], shape).astype(np.float64))
+    trace = []
+    orc.newton_schulz(G, 3, QUINTIC, 1e-7, "bf16", trace=trace)
+    for k in (0, 2):
+        Xk = trace[k][2]                       # working orientation (wide)
+        Xk = Xk.T if shape[0] > shape[1] else Xk
+        outs, vals = _ortho(mb, ctx, [Xk.astype(np.float32)], steps=1, flags=mb.ORTHO_NO_NORMALIZE)
+        assert np.array_equal(vals[0], Xk)
+        wide = vals[0].T if shape[0] > shape[1] else vals[0]
+        ref = orc.ns_single_step(wide, *QUINTIC, mode="bf16")
+        ref = ref.T if shape[0] > shape[1] else ref
+        e = rel(outs[0], ref)
+        assert e <= TOL_SINGLE_STEP, (k, e)
+        assert np.mean(outs[0] != ref) < 0.10
+    ctx.close()
+
+
+def test_ns_fp32_mode_vs_fp64_oracle():
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "fp32")
+    shapes = wl.shapes_tiny() + [(37, 53), (130, 7), (300, 129)]
+    mats = [wl.grad_np("fp32", 0, i, s) for i, s in enumerate(shapes)]
+    outs, vals = _ortho(mb, ctx, mats)
+    for i, (o, v) in enumerate(zip(outs, vals)):
+        ref = orc.newton_schulz(v, 5, QUINTIC, 1e-7, "fp64")
+        assert rel(o, ref) <= TOL_FP32, (i, shapes[i], rel(o, ref))
+    ctx.close()
+
+
+def test_ns_fp32_cubic_converges_to_polar_factor_on_device():
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "fp32")
+    rng = np.random.default_rng(4)
+    U, _ = np.linalg.qr(rng.standard_normal((48, 48)))
+    V, _ = np.linalg.qr(rng.standard_normal((80, 48)))
+    G = (U * np.linspace(1, 3, 48)) @ V.T
+    outs, _ = _ortho(mb, ctx, [G.astype(np.float32)], steps=40, coeffs=(1.5, -0.5, 0.0))
+    assert rel(outs[0], U @ V.T) < 1e-4
+    ctx.close()
+
+
+def test_ns_per_step_coefficients():
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "fp32", coeffs_per_step=1)
+    co = [3.0, -3.2, 1.2, 3.4445, -4.7750, 2.0315, 2.0, -1.5, 0.5]
+    G = wl.grad_np("perstep", 0, 0, (40, 72))
+    outs, vals = _ortho(mb, ctx, [G], steps=3, coeffs=co)
+    assert rel(outs[0], orc.newton_schulz(vals[0], 3, co, 1e-7, "fp64")) <= TOL_FP32
+    ctx.close()
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_zero_gradient_and_scaling(engine):
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "bf16", engine)
+    Z = np.zeros((64, 96), dtype=np.float32)
+    G = wl.grad_np("scale", 0, 0, (64, 96), std=1.0)
+    outs, vals = _ortho(mb, ctx, [Z, G, G * np.float32(2.0 ** 40), G * np.float32(2.0 ** 20)])
+    assert np.array_equal(outs[0], np.zeros((64, 96)))
+    assert np.isfinite(outs[1]).all()
+    # powers of two commute with every rounding and eps is negligible at these norms
+    assert rel(outs[2], outs[1]) < 1e-3 and rel(outs[3], outs[1]) < 1e-3
+    ctx.close()
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_batched_equals_alone_and_rerun_bit_exact(engine):
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "bf16", engine)
+    shapes = [(256, 256)] * 3 + [(1024, 256), (256, 1024), (130, 200)]
+    mats = [wl.grad_np("batch", 0, i, s) for i, s in enumerate(shapes)]
+    together, _ = _ortho(mb, ctx, mats)
+    again, _ = _ortho(mb, ctx, mats)
+    for a, b in zip(together, again):
+        assert np.array_equal(a, b)
+    for i, m in enumerate(mats):
+        alone, _ = _ortho(mb, ctx, [m])
+        assert np.array_equal(alone[0], together[i]), i
+    # a small chunk cap changes the batching but not the numbers
+    ctx2 = _ctx(mb, "bf16", engine, chunk_elems=70000)
+    capped, _ = _ortho(mb, ctx2, mats)
+    for a, b in zip(together, capped):
+        assert np.array_equal(a, b)
+    ctx.close()
+    ctx2.close()
+
+
+# ----------------------------------------------------------------------------- the full step
+def _run_steps(mb, ctx, config, shapes, n_steps, grad_bf16, row_scaled=False, lr=0.02, mu=0.95, wd=0.01):
+    Ws = [wl.param_np(config, i, s) for i, s in enumerate(shapes)]
+    dW, dM = [dev_f32(w) for w in Ws], [torch.zeros(s, dtype=torch.float32, device="cuda") for s in shapes]
+    ctx.ensure_workspace(shapes)
+    Gs_all, hist = [], []
+    for t in range(n_steps):
+        Gs_dev, Gs_val = [], []
+        for i, s in enumerate(shapes):
+            g = wl.grad_np(config, t, i, s, row_scaled=row_scaled)
+            if grad_bf16:
+                d, v = bf16_input(g)
+            else:
+                d, v = dev_f32(g), g.astype(np.float64)
+            Gs_dev.append(d)
+            Gs_val.append(v)
+        Gs_all.append(Gs_val)
+        ctx.muon_step_batched(dW, Gs_dev, dM, shapes, lr, mu, wd, 5, QUINTIC)
+        torch.cuda.synchronize()
+        hist.append(([host_f64(w) for w in dW], [host_f64(m) for m in dM]))
+    assert ctx.muon_last_device_status() == 0
+    return Ws, Gs_all, hist
+
+
+@pytest.mark.parametrize("precision,engine,grad", [("fp32", "tensor", "fp32"), ("bf16", "tensor", "fp32"),
+                                                   ("bf16", "cuda_core", "fp32"), ("bf16", "tensor", "bf16")])
+def test_tiny_config_three_steps(precision, engine, grad):
+    """d=256 one-layer matrix set, 3 consecutive optimizer steps from seed 0 (mu 0.95 Nesterov, lr 0.02, wd 0.01)."""
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, precision, engine, grad)
+    shapes = wl.shapes_tiny()
+    lr, mu, wd = 0.02, 0.95, 0.01
+    Ws, Gs_all, hist = _run_steps(mb, ctx, "tiny", shapes, 3, grad == "bf16")
+    mode = "bf16" if precision == "bf16" else "fp64"
+    tol = TOL_BF16 if precision == "bf16" else TOL_FP32
+    W = [w.astype(np.float64) for w in Ws]
+    M = [np.zeros(s) for s in shapes]
+    for t in range(3):
+        gotW, gotM = hist[t]
+        for i in range(len(shapes)):
+            # teacher-forced per optimizer step: the oracle continues from the device's own state
+            Wprev = W[i]
+            Wn, Mn, O = orc.muon_step(Wprev, Gs_all[t][i], M[i], lr, mu, wd, 5, QUINTIC, 1e-7, True, mode)
+            assert rel(gotM[i], Mn) <= 1e-6, (t, i)
+            e = rel(gotW[i] - Wprev, Wn - Wprev)
+            assert e <= tol, (t, i, shapes[i], e)
+            O_dev = (Wprev * (1 - lr * wd) - gotW[i]) / (lr * orc.update_scale(*shapes[i]))
+            assert rel(O_dev, O) <= tol + 1e-4, (t, i)
+            W[i], M[i] = gotW[i], gotM[i]
+    ctx.close()
+
+
+def test_update_limits_and_snapshot_resume():
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "bf16", "tensor", "bf16")
+    shapes = [(256, 256), (320, 192)]
+    ctx.ensure_workspace(shapes)
+    Ws = [dev_f32(wl.param_np("lim", i, s)) for i, s in enumerate(shapes)]
+    Ms = [torch.zeros(s, dtype=torch.float32, device="cuda") for s in shapes]
+    Gs = [bf16_input(wl.grad_np("lim", 0, i, s))[0] for i, s in enumerate(shapes)]
+    W0 = [w.clone() for w in Ws]
+    ctx.muon_step_batched(Ws, Gs, Ms, shapes, 0.0, 0.95, 0.3, 5, QUINTIC)     # lr = 0: weights untouched, momentum moves
+    torch.cuda.synchronize()
+    for w, w0, m, g in zip(Ws, W0, Ms, Gs):
+        assert torch.equal(w, w0)
+        assert torch.equal(m, g.float())                                     # M0 = 0: M' = G exactly
+    # 3 steps == 2 steps + snapshot/restore + 1 step, bit for bit (all state is caller-owned)
+    def run(n, Wi, Mi):
+        for t in range(n[0], n[1]):
+            G = [bf16_input(wl.grad_np("lim", t, i, s))[0] for i, s in enumerate(shapes)]
+            ctx.muon_step_batched(Wi, G, Mi, shapes, 0.02, 0.95, 0.01, 5, QUINTIC)
+        torch.cuda.synchronize()
+    Wa, Ma = [w.clone() for w in W0], [torch.zeros_like(m) for m in Ms]
+    run((0, 3), Wa, Ma)
+    Wb, Mb = [w.clone() for w in W0], [torch.zeros_like(m) for m in Ms]
+    run((0, 2), Wb, Mb)
+    Wc, Mc = [w.cpu().cuda() for w in Wb], [m.cpu().cuda() for m in Mb]
+    run((2, 3), Wc, Mc)
+    for a, c in zip(Wa + Ma, Wc + Mc):
+        assert torch.equal(a, c)
+    ctx.close()
+
+
+def test_step_argument_errors_launch_nothing():
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "bf16", "tensor", "bf16")
+    shapes = [(64, 64)]
+    W = [torch.zeros(64, 64, device="cuda")]
+    M = [torch.zeros(64, 64, device="cuda")]
+    G = [torch.zeros(64, 64, device="cuda", dtype=torch.bfloat16)]
+    before = ctx.muon_launch_count()
+    with pytest.raises(mb.MuonError) as e:
+        ctx.muon_step_batched(W, G, M, shapes, 0.02, 0.95, 0.01, 5, QUINTIC)
+    assert e.value.code == mb.ERR_WORKSPACE_TOO_SMALL
+    ctx.ensure_workspace(shapes)
+    for bad in ([None], [W[0].view(-1)[1:]]):
+        with pytest.raises(mb.MuonError) as e:
+            ctx.muon_step_batched(bad, G, M, shapes, 0.02, 0.95, 0.01, 5, QUINTIC)
+        assert e.value.code == mb.ERR_INVALID_ARG
+    with pytest.raises(mb.MuonError):
+        ctx.muon_step_batched(W, G, M, shapes, 0.02, 0.95, 0.01, 0, QUINTIC)
+    with pytest.raises(mb.MuonError):
+        ctx.muon_step_batched(W, G, M, shapes, float("nan"), 0.95, 0.01, 5, QUINTIC)
+    with pytest.raises(mb.MuonError):
+        ctx.muon_step_batched(W, G, M, [(-1, 4)], 0.02, 0.95, 0.01, 5, QUINTIC)
+    assert ctx.muon_launch_count() == before
+    ctx.muon_step_batched([], [], [], [], 0.02, 0.95, 0.01, 5, QUINTIC)       # count == 0: a no-op
+    ctx.muon_step_batched([None], [None], [None], [(0, 7)], 0.02, 0.95, 0.01, 5, QUINTIC)
+    assert ctx.muon_launch_count() == before
+    ctx.close()
