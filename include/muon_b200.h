@@ -173,6 +173,22 @@ int muon_orthogonalize_batched(muon_ctx_t* ctx, const void* const* in, void* con
                                const muon_shape_t* shapes, int32_t count,
                                int32_t ns_steps, const float* coeffs, uint32_t flags, void* stream);
 
+/* muon_ns_product: the batched product primitive the Newton-Schulz iteration is built from (the
+ * three products of one step of Eq. 1), exposed for per-kernel parity checks and timing:
+ *     C[i] = gamma_i * (beta * D[i] + alpha * P[i] Q[i]^T)        nn = 0, P: m x k, Q: n x k
+ *     C[i] = gamma_i * (beta * D[i] + alpha * P[i] Q[i])          nn = 1, P: m x k, Q: k x n
+ * for i < batch.  All operands are device pointers to row-major matrices of the NS element type
+ * (bf16 under MUON_NS_BF16, fp32 under MUON_NS_FP32) with leading dimensions ldp, ldq, ldc in
+ * elements (D shares ldc and stride_c; d may be NULL) and stride_* elements between consecutive
+ * matrices.  gamma_i = 1 when gamma is NULL, else gamma[i] (gamma_mode 1) or gamma[i]^2
+ * (gamma_mode 2), gamma being a device array of `batch` floats.  For the tensor-core engine bases
+ * must be 16-byte aligned and every ld/stride a multiple of 8 elements; other cases run on CUDA
+ * cores.  C must not alias P, Q or D. */
+int muon_ns_product(muon_ctx_t* ctx, const void* p, const void* q, const void* d, void* c,
+                    int32_t m, int32_t n, int32_t k, int32_t ldp, int32_t ldq, int32_t ldc,
+                    int64_t stride_p, int64_t stride_q, int64_t stride_c, int32_t batch, int32_t nn,
+                    float alpha, float beta, const float* gamma, int32_t gamma_mode, void* stream);
+
 /* Device-side status word: the tensor-core pipeline bounds every wait on a barrier; a wait
  * that gives up records a non-zero code here and the kernel exits cleanly.  Reads the word
  * after synchronising `stream`; 0 = no bounded wait ever expired on this context. */

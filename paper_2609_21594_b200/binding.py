@@ -66,6 +66,9 @@ _sig = {
                                     C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
     "muon_orthogonalize_batched": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(Shape), C.c_int32,
                                              C.c_int32, C.POINTER(C.c_float), C.c_uint32, _vp]),
+    "muon_ns_product": (C.c_int, [_vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                  C.c_int64, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_float, C.c_float, _vp,
+                                  C.c_int32, _vp]),
     "muon_last_device_status": (C.c_int, [_vp, _vp, C.POINTER(C.c_int32)]),
     "muon_profile_enable": (C.c_int, [_vp, C.c_int32]),
     "muon_profile_reset": (C.c_int, [_vp]),
@@ -229,6 +232,13 @@ class Context:
         co = (C.c_float * len(coeffs))(*[float(c) for c in coeffs])
         _check(lib.muon_orthogonalize_batched(self.handle, _ptrs(inputs), _ptrs(outputs), _shapes(shapes), len(shapes),
                                               ns_steps, co, flags, _stream(stream)), "muon_orthogonalize_batched")
+
+    def muon_ns_product(self, p, q, d, c, m, n, k, ldp, ldq, ldc, stride_p, stride_q, stride_c, batch, nn,
+                        alpha=1.0, beta=0.0, gamma=None, gamma_mode=0, stream=None) -> None:
+        _check(lib.muon_ns_product(self.handle, p.data_ptr(), q.data_ptr(), None if d is None else d.data_ptr(),
+                                   c.data_ptr(), m, n, k, ldp, ldq, ldc, stride_p, stride_q, stride_c, batch, nn,
+                                   alpha, beta, None if gamma is None else gamma.data_ptr(), gamma_mode,
+                                   _stream(stream)), "muon_ns_product")
 
     def muon_last_device_status(self, stream=None) -> int:
         v = C.c_int32(0)

@@ -450,6 +450,36 @@ int muon_orthogonalize_batched(muon_ctx_t* ctx, const void* const* in, void* con
   return run_batched(ctx, out, in, nullptr, shapes, count, r, static_cast<cudaStream_t>(stream));
 }
 
+int muon_ns_product(muon_ctx_t* ctx, const void* p, const void* q, const void* d, void* c, int32_t m, int32_t n,
+                    int32_t k, int32_t ldp, int32_t ldq, int32_t ldc, int64_t stride_p, int64_t stride_q,
+                    int64_t stride_c, int32_t batch, int32_t nn, float alpha, float beta, const float* gamma,
+                    int32_t gamma_mode, void* stream) {
+  if (!ctx || m < 0 || n < 0 || k < 0 || batch < 0) return MUON_ERR_INVALID_ARG;
+  if (m == 0 || n == 0 || batch == 0) return MUON_OK;
+  if (!p || !q || !c || k < 1) return MUON_ERR_INVALID_ARG;
+  if (nn != 0 && nn != 1) return MUON_ERR_INVALID_ARG;
+  if (gamma_mode < 0 || gamma_mode > 2 || (gamma_mode && !gamma)) return MUON_ERR_INVALID_ARG;
+  if (ldp < k || ldc < n || ldq < (nn ? n : k)) return MUON_ERR_INVALID_ARG;
+  if (c == p || c == q || c == d) return MUON_ERR_INVALID_ARG;
+  if (!DeviceGuardCheck::ok(ctx)) return MUON_ERR_CUDA;
+  GemmArgs g{};
+  g.p = p; g.q = q; g.d = d; g.c = c;
+  g.m = m; g.n = n; g.kdim = k;
+  g.ldp = ldp; g.ldq = ldq; g.ldc = ldc;
+  g.stride_p = stride_p; g.stride_q = stride_q; g.stride_c = stride_c;
+  g.batch = batch;
+  g.rnorm = gamma;
+  g.gamma_mode = gamma ? gamma_mode : 0;
+  g.alpha = alpha; g.beta = beta; g.nn = nn; g.symmetric = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Span sp(ctx, MUON_PHASE_NS, st);
+  const int nl = run_gemm(ctx, g, st);
+  if (nl < 0) return nl;
+  ctx->launches += nl;
+  sp.end(nl);
+  return MUON_OK;
+}
+
 int muon_last_device_status(muon_ctx_t* ctx, void* stream, int32_t* status) {
   if (!ctx || !status) return MUON_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

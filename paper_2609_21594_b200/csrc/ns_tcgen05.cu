@@ -1,7 +1,424 @@
-// Tensor-core Newton-Schulz engine (placeholder translation unit: filled in by the tcgen05 kernels).
+// Tensor-core Newton-Schulz engine for sm_100a: batched products of Eq. 1 with bf16 operands and
+// fp32 accumulation in tensor memory.
+//
+//   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k]^T)     nn = 0   (A = X X^T,  B = bA + cA A^T)
+//   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k])       nn = 1   (X' = aX + B X)
+//
+// One persistent CTA per SM, 192 threads, warp-specialised:
+//   warp 0      TMA producer: cp.async.bulk.tensor loads of 128B-swizzled operand tiles into a
+//               4-stage shared-memory ring (one mbarrier pair per stage)
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (M128 x N256 x K16, kind::f16) on shared-memory
+//               descriptors; accumulators live in TMEM, double-buffered (2 x 256 columns)
+//   warps 2..5  epilogue: tcgen05.ld of the accumulator, fused gamma*(beta*D + alpha*acc), one bf16
+//               rounding, 16-byte global stores; overlaps the next tile's main loop
+// P tiles are K-major.  Q tiles are K-major for nn = 0 and MN-major for nn = 1 (X is read as stored,
+// row-major s x l, so no transposed copy of X is ever made).
+// Every wait on an mbarrier is bounded: on expiry the CTA records a code in the context's status
+// word, stops issuing work, waits (bounded) for its own TMA copies, frees its TMEM and returns.
+#include <cuda.h>
+
+#include <cstring>
+
 #include "internal.h"
 
 namespace muon {
-bool tc_supported(const GemmArgs&) { return false; }
-int launch_gemm_tc(muon_ctx*, const GemmArgs&, cudaStream_t) { return MUON_ERR_UNSUPPORTED; }
+namespace {
+
+constexpr int BM = 128;          // tile rows   (UMMA M)
+constexpr int BN = 256;          // tile cols   (UMMA N)
+constexpr int BK = 64;           // k per stage (one 128-byte swizzle atom of bf16)
+constexpr int UK = 16;           // k per tcgen05.mma for 16-bit inputs
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;          // 16 KiB
+constexpr int B_BYTES = BN * BK * 2;          // 32 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int TMEM_COLS = 512;
+constexpr int NUM_THREADS = 192;
+constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2 s at 1.9 GHz: far beyond any legitimate wait
+
+struct TcArgs {
+  const __nv_bfloat16* d;   // aux matrix (may be null)
+  __nv_bfloat16* c;
+  int32_t m, n, kdim, ldc;
+  int64_t stride_c;
+  int32_t batch, tiles_m, tiles_n;
+  const float* rnorm;
+  int32_t gamma_mode;
+  float alpha, beta;
+  int32_t* status;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the deadline passed or (honor_abort) another role gave up;
+// the caller must then abandon the pipeline.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          bool honor_abort = true, long long limit = WAIT_CYCLES) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++spins & 255u) == 0) {
+      if (honor_abort && *abort_flag) return false;
+      if (clock64() - t0 > limit) return false;
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
+// lbo/sbo in bytes.  K-major: lbo is unused by the hardware for swizzled layouts (set to 16),
+// sbo = distance between 8-row groups.  MN-major: lbo = distance between 64-element column
+// chunks, sbo = distance between groups of 8 k-rows.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= uint64_t((saddr & 0x3FFFFu) >> 4);
+  d |= uint64_t((lbo >> 4) & 0x3FFFu) << 16;
+  d |= uint64_t((sbo >> 4) & 0x3FFFu) << 32;
+  d |= uint64_t(1) << 46;
+  d |= uint64_t(2) << 61;
+  return d;
+}
+
+// Instruction descriptor for kind::f16: fp32 accumulator, bf16 A and B, A K-major, B K- or MN-major.
+__host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(b_mn_major ? 1 : 0) << 16) | (uint32_t(BN >> 3) << 17) |
+         (uint32_t(BM >> 4) << 24);
+}
+
+struct Tile {
+  int mat, m0, n0;
+};
+__device__ __forceinline__ Tile decode_tile(int t, const TcArgs& a) {
+  const int per = a.tiles_m * a.tiles_n;
+  Tile r;
+  r.mat = t / per;
+  const int u = t - r.mat * per;
+  r.n0 = (u / a.tiles_m) * BN;     // row blocks vary fastest: concurrent CTAs share the Q tile
+  r.m0 = (u % a.tiles_m) * BM;
+  return r;
+}
+
+template <bool NN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q, const TcArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;            // swizzled tiles need 1024-byte alignment
+  uint8_t* gen_base = smem_raw + (base - raw);
+  const uint32_t bars = base + STAGES * STAGE_BYTES;        // barrier block follows the tiles
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + STAGES * STAGE_BYTES + 128);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + STAGES * STAGE_BYTES + 136);
+  auto full_bar = [&](int s) { return bars + uint32_t(s) * 8u; };
+  auto empty_bar = [&](int s) { return bars + uint32_t(STAGES + s) * 8u; };
+  auto tfull_bar = [&](int i) { return bars + uint32_t(2 * STAGES + i) * 8u; };
+  auto tempty_bar = [&](int i) { return bars + uint32_t(2 * STAGES + 2 + i) * 8u; };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_tiles = a.batch * a.tiles_m * a.tiles_n;
+  const int num_kb = (a.kdim + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(tfull_bar(i), 1);
+      mbar_init(tempty_bar(i), 4);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const Tile tl = decode_tile(t, a);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = int(it % STAGES);
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t sa = base + uint32_t(s) * STAGE_BYTES, sb = sa + A_BYTES;
+          mbar_expect_tx(full_bar(s), STAGE_BYTES);
+          const int k0 = kb * BK;
+          tma_load_3d(sa, &map_p, full_bar(s), k0, tl.m0, tl.mat);                   // P rows m0.., k0..k0+63
+          if (!NN) {
+            tma_load_3d(sb, &map_q, full_bar(s), k0, tl.n0, tl.mat);                 // Q rows n0..n0+127
+            tma_load_3d(sb + A_BYTES, &map_q, full_bar(s), k0, tl.n0 + 128, tl.mat); // Q rows n0+128..n0+255
+          } else {
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j)                                        // Q[k0..k0+63][n0+64j..+63]
+              tma_load_3d(sb + uint32_t(j) * (64 * BK * 2), &map_q, full_bar(s), tl.n0 + 64 * j, k0, tl.mat);
+          }
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicExch(a.status, 1);
+      }
+      // Drain: every armed stage must have landed before this CTA's shared memory is released.
+      const uint32_t issued = it;
+      for (uint32_t j = (issued > STAGES ? issued - STAGES : 0); j < issued; ++j) {
+        const int s = int(j % STAGES);
+        const uint32_t ph = (j / STAGES) & 1u;
+        if (!mbar_wait(full_bar(s), ph, abort_flag, false, WAIT_CYCLES / 8)) atomicExch(a.status, 2);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(NN);
+      uint32_t it = 0, tile_it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_it) {
+        const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(int(acc)), aph ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * uint32_t(BN);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = int(it % STAGES);
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + uint32_t(s) * STAGE_BYTES, sb = sa + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UK; ++k) {
+            const uint64_t ad = make_desc(sa + uint32_t(k) * (UK * 2), 16, 1024);
+            const uint64_t bd = NN ? make_desc(sb + uint32_t(k) * (UK * 128), 64 * BK * 2, 1024)
+                                   : make_desc(sb + uint32_t(k) * (UK * 2), 16, 1024);
+            tc_mma(d_tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          tc_commit(empty_bar(s));             // stage reusable once these MMAs have read it
+        }
+        if (ok) tc_commit(tfull_bar(int(acc)));  // accumulator complete
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicExch(a.status, 3);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps
+    const int quad = warp & 3;                     // TMEM lane quadrant this warp may read
+    uint32_t tile_it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_it) {
+      const Tile tl = decode_tile(t, a);
+      const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+      if (!mbar_wait(tfull_bar(int(acc)), aph, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      float gamma = 1.f;
+      if (a.gamma_mode) {
+        const float r = a.rnorm[tl.mat];
+        gamma = a.gamma_mode == 1 ? r : r * r;
+      }
+      const int row = tl.m0 + quad * 32 + lane;
+      const bool row_ok = row < a.m;
+      const size_t row_off = size_t(tl.mat) * a.stride_c + size_t(row_ok ? row : 0) * a.ldc;
+      const __nv_bfloat16* drow = a.d ? a.d + row_off : nullptr;
+      __nv_bfloat16* crow = a.c + row_off;
+      const uint32_t taddr = tmem_base + acc * uint32_t(BN) + (uint32_t(quad * 32) << 16);
+#pragma unroll 1
+      for (int cb = 0; cb < BN / 32; ++cb) {
+        const int c0 = tl.n0 + cb * 32;
+        if (c0 >= a.n) break;                       // warp-uniform
+        uint32_t v[32];
+        tc_ld32(taddr + uint32_t(cb * 32), v);
+        tc_wait_ld();
+        if (row_ok) {
+          if (c0 + 32 <= a.n) {
+            alignas(16) __nv_bfloat16 dv[32];
+            if (drow) {
+#pragma unroll
+              for (int q = 0; q < 4; ++q) reinterpret_cast<uint4*>(dv)[q] = reinterpret_cast<const uint4*>(drow + c0)[q];
+            }
+            alignas(16) __nv_bfloat162 out[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              float x0 = a.alpha * __uint_as_float(v[2 * j]), x1 = a.alpha * __uint_as_float(v[2 * j + 1]);
+              if (drow) {
+                x0 += a.beta * __bfloat162float(dv[2 * j]);
+                x1 += a.beta * __bfloat162float(dv[2 * j + 1]);
+              }
+              out[j] = __floats2bfloat162_rn(gamma * x0, gamma * x1);
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) reinterpret_cast<uint4*>(crow + c0)[q] = reinterpret_cast<const uint4*>(out)[q];
+          } else {
+            for (int j = 0; j < 32; ++j) {
+              const int c = c0 + j;
+              if (c < a.n) {
+                float x = a.alpha * __uint_as_float(v[j]);
+                if (drow) x += a.beta * __bfloat162float(drow[c]);
+                crow[c] = __float2bfloat16_rn(gamma * x);
+              }
+            }
+          }
+        }
+        __syncwarp();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(int(acc)));
+    }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      atomicExch(a.status, 4);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 3-D map over a batch of row-major matrices: dims (cols, rows, batch), box (64, box_rows, 1), 128B swizzle.
+bool encode_map(void* fn, CUtensorMap* map, const void* ptr, int cols, int rows, int batch, int ld, int64_t stride,
+                int box_rows) {
+  const cuuint64_t dims[3] = {cuuint64_t(cols), cuuint64_t(rows), cuuint64_t(batch)};
+  const cuuint64_t strides[2] = {cuuint64_t(ld) * 2u, cuuint64_t(stride) * 2u};
+  const cuuint32_t box[3] = {64u, cuuint32_t(box_rows), 1u};
+  const cuuint32_t estr[3] = {1u, 1u, 1u};
+  const CUresult r = reinterpret_cast<EncodeFn>(fn)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims,
+                                                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+int g_num_sms = 0;
+bool g_attr_set = false;
+
+}  // namespace
+
+bool tc_supported(const GemmArgs& a) {
+  if (a.m < 1 || a.n < 1 || a.kdim < 1 || a.batch < 1) return false;
+  // tensor-map strides must be multiples of 16 bytes, bases 16-byte aligned
+  if ((a.ldp % 8) || (a.ldq % 8) || (a.ldc % 8) || (a.stride_p % 8) || (a.stride_q % 8) || (a.stride_c % 8)) return false;
+  if ((reinterpret_cast<uintptr_t>(a.p) | reinterpret_cast<uintptr_t>(a.q) | reinterpret_cast<uintptr_t>(a.c) |
+       reinterpret_cast<uintptr_t>(a.d)) & 15u)
+    return false;
+  const int64_t tiles = int64_t((a.m + BM - 1) / BM) * ((a.n + BN - 1) / BN) * a.batch;
+  return tiles < (int64_t(1) << 30);
+}
+
+int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st) {
+  if (!ctx->tmap_encode) return MUON_ERR_CUDA;
+  if (!g_attr_set) {
+    if (cudaFuncSetAttribute(ns_product_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(ns_product_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+      return MUON_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, ctx->device) != cudaSuccess) return MUON_ERR_CUDA;
+    g_num_sms = prop.multiProcessorCount;
+    g_attr_set = true;
+  }
+  CUtensorMap map_p, map_q;
+  // P: rows = m, cols = kdim
+  if (!encode_map(ctx->tmap_encode, &map_p, a.p, a.kdim, a.m, a.batch, a.ldp, a.stride_p, BM)) return MUON_ERR_CUDA;
+  if (!a.nn) {  // Q: rows = n, cols = kdim; two 128-row boxes per stage
+    if (!encode_map(ctx->tmap_encode, &map_q, a.q, a.kdim, a.n, a.batch, a.ldq, a.stride_q, 128)) return MUON_ERR_CUDA;
+  } else {      // Q: rows = kdim, cols = n; four 64(k) x 64(n) boxes per stage
+    if (!encode_map(ctx->tmap_encode, &map_q, a.q, a.n, a.kdim, a.batch, a.ldq, a.stride_q, BK)) return MUON_ERR_CUDA;
+  }
+  TcArgs t;
+  t.d = static_cast<const __nv_bfloat16*>(a.d);
+  t.c = static_cast<__nv_bfloat16*>(a.c);
+  t.m = a.m; t.n = a.n; t.kdim = a.kdim; t.ldc = a.ldc;
+  t.stride_c = a.stride_c;
+  t.batch = a.batch;
+  t.tiles_m = (a.m + BM - 1) / BM;
+  t.tiles_n = (a.n + BN - 1) / BN;
+  t.rnorm = a.rnorm;
+  t.gamma_mode = a.gamma_mode;
+  t.alpha = a.alpha; t.beta = a.beta;
+  t.status = ctx->d_status;
+  const int64_t tiles = int64_t(t.tiles_m) * t.tiles_n * t.batch;
+  const unsigned grid = unsigned(tiles < g_num_sms ? tiles : g_num_sms);
+  if (a.nn) ns_product_tc_kernel<true><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, t);
+  else ns_product_tc_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, t);
+  return cudaGetLastError() == cudaSuccess ? 1 : MUON_ERR_CUDA;
+}
+
 }  // namespace muon
