@@ -165,6 +165,27 @@ int muon_step_batched(muon_ctx_t* ctx, void* const* params, const void* const* g
                       const muon_shape_t* shapes, int32_t count, float lr, float mu, float wd,
                       int32_t ns_steps, const float* coeffs, void* stream);
 
+/* muon_step_batched_out: muon_step_batched that additionally writes each matrix's orthogonalised
+ * update O = X_ns (shape rows x cols, element type of the NS precision) to updates[i] -- the payload
+ * owners pack for the relay broadcast (Section 6.2 step 3).  updates may be NULL (then identical to
+ * muon_step_batched); otherwise a host array [count] of 16-byte-aligned device pointers. */
+int muon_step_batched_out(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
+                          void* const* updates, const muon_shape_t* shapes, int32_t count, float lr, float mu,
+                          float wd, int32_t ns_steps, const float* coeffs, void* stream);
+
+/* muon_step_flat_host: the whole path on HOST flat buffers, for end-to-end use and timing:
+ * copy host_flat_grads (host; pinned memory makes the copies asynchronous) to dev_flat, materialise it
+ * into grads[], run muon_step_batched_out on the layout's shapes, scatter updates[] into dev_flat and
+ * copy dev_flat to host_flat_updates (host).  dev_flat: device staging buffer of
+ * num_shards*shard_len elements; grads/updates: host arrays of device pointers to whole-matrix
+ * scratch the caller owns.  The layout's element size must equal both the gradient and the NS
+ * element size (bf16/bf16 or fp32/fp32).  Everything is enqueued on `stream` in order; the host
+ * buffers may be touched again once the stream has been synchronised. */
+int muon_step_flat_host(muon_ctx_t* ctx, const void* host_flat_grads, void* host_flat_updates, void* dev_flat,
+                        const muon_layout_t* layout, void* const* params, void* const* grads, void* const* momenta,
+                        void* const* updates, float lr, float mu, float wd, int32_t ns_steps, const float* coeffs,
+                        void* stream);
+
 /* muon_orthogonalize_batched: only the Newton-Schulz part of the step (Eq. 1) on given
  * inputs -- for per-kernel parity checks and timing.  Element type of in/out is bf16 under
  * MUON_NS_BF16 and fp32 under MUON_NS_FP32; out[i] has the shape of in[i]; in and out may

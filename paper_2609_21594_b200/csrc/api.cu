@@ -203,8 +203,8 @@ int run_chunk(muon_ctx* ctx, const Chunk& ch, const MatDesc* d_descs, const Chun
   return MUON_OK;
 }
 
-int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const* m, const muon_shape_t* shapes,
-                int32_t count, const ChunkRun& r, cudaStream_t st) {
+int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const* m, void* const* o,
+                const muon_shape_t* shapes, int32_t count, const ChunkRun& r, cudaStream_t st) {
   int status;
   Plan* plan = get_plan(ctx, shapes, count, &status);
   if (!plan) return status;
@@ -218,8 +218,10 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
       d.w = w[i];
       d.g = g[i];
       d.m = m ? m[i] : nullptr;
-      if (!d.w || !d.g || (r.momentum && !d.m)) return MUON_ERR_INVALID_ARG;
-      if (!aligned(d.w, 16) || !aligned(d.g, 16) || (d.m && !aligned(d.m, 16))) return MUON_ERR_INVALID_ARG;
+      d.o = o ? o[i] : nullptr;
+      if (!d.w || !d.g || (r.momentum && !d.m) || (o && !d.o)) return MUON_ERR_INVALID_ARG;
+      if (!aligned(d.w, 16) || !aligned(d.g, 16) || (d.m && !aligned(d.m, 16)) || (d.o && !aligned(d.o, 16)))
+        return MUON_ERR_INVALID_ARG;
       d.rows = shapes[i].rows;
       d.cols = shapes[i].cols;
       d.transposed = d.rows > d.cols ? 1 : 0;
@@ -426,16 +428,47 @@ static int check_common(muon_ctx_t* ctx, const muon_shape_t* shapes, int32_t cou
   return MUON_OK;
 }
 
-int muon_step_batched(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
-                      const muon_shape_t* shapes, int32_t count, float lr, float mu, float wd, int32_t ns_steps,
-                      const float* coeffs, void* stream) {
+int muon_step_batched_out(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
+                          void* const* updates, const muon_shape_t* shapes, int32_t count, float lr, float mu, float wd,
+                          int32_t ns_steps, const float* coeffs, void* stream) {
   int st = check_common(ctx, shapes, count, ns_steps, coeffs);
   if (st != MUON_OK) return st;
   if (count == 0) return MUON_OK;
   if (!params || !grads || !momenta) return MUON_ERR_INVALID_ARG;
   if (!std::isfinite(lr) || !std::isfinite(mu) || !std::isfinite(wd)) return MUON_ERR_INVALID_ARG;
   ChunkRun r{1, 1, lr, mu, wd, ns_steps, coeffs};
-  return run_batched(ctx, params, grads, momenta, shapes, count, r, static_cast<cudaStream_t>(stream));
+  return run_batched(ctx, params, grads, momenta, updates, shapes, count, r, static_cast<cudaStream_t>(stream));
+}
+
+int muon_step_batched(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
+                      const muon_shape_t* shapes, int32_t count, float lr, float mu, float wd, int32_t ns_steps,
+                      const float* coeffs, void* stream) {
+  return muon_step_batched_out(ctx, params, grads, momenta, nullptr, shapes, count, lr, mu, wd, ns_steps, coeffs, stream);
+}
+
+int muon_step_flat_host(muon_ctx_t* ctx, const void* host_flat_grads, void* host_flat_updates, void* dev_flat,
+                        const muon_layout_t* layout, void* const* params, void* const* grads, void* const* momenta,
+                        void* const* updates, float lr, float mu, float wd, int32_t ns_steps, const float* coeffs,
+                        void* stream) {
+  if (!ctx || !layout || !host_flat_grads || !host_flat_updates || !dev_flat || !updates) return MUON_ERR_INVALID_ARG;
+  const int want = ctx->opt.grad_dtype == MUON_DTYPE_BF16 ? 2 : 4;
+  const int ns_es = ctx->opt.ns_precision == MUON_NS_BF16 ? 2 : 4;
+  if (layout->desc.elem_size != want || ns_es != want) return MUON_ERR_INVALID_ARG;   // one flat buffer carries both ways
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = size_t(layout->desc.num_shards) * size_t(layout->desc.shard_len) * size_t(want);
+  const int32_t count = layout->desc.num_matrices;
+  int rc = check_common(ctx, layout->shapes.data(), count, ns_steps, coeffs);
+  if (rc != MUON_OK) return rc;
+  if (cudaMemcpyAsync(dev_flat, host_flat_grads, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return MUON_ERR_CUDA;
+  rc = muon_materialize(ctx, dev_flat, layout, grads, stream);
+  if (rc != MUON_OK) return rc;
+  rc = muon_step_batched_out(ctx, params, const_cast<const void* const*>(grads), momenta, updates, layout->shapes.data(),
+                             count, lr, mu, wd, ns_steps, coeffs, stream);
+  if (rc != MUON_OK) return rc;
+  rc = muon_scatter(ctx, dev_flat, layout, const_cast<const void* const*>(updates), stream);
+  if (rc != MUON_OK) return rc;
+  if (cudaMemcpyAsync(host_flat_updates, dev_flat, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MUON_ERR_CUDA;
+  return MUON_OK;
 }
 
 int muon_orthogonalize_batched(muon_ctx_t* ctx, const void* const* in, void* const* out, const muon_shape_t* shapes,
@@ -447,7 +480,7 @@ int muon_orthogonalize_batched(muon_ctx_t* ctx, const void* const* in, void* con
   for (int32_t i = 0; i < count; ++i)
     if (shapes[i].rows > 0 && shapes[i].cols > 0 && in[i] == out[i]) return MUON_ERR_INVALID_ARG;
   ChunkRun r{0, (flags & MUON_ORTHO_NO_NORMALIZE) ? 0 : 1, 0.f, 0.f, 0.f, ns_steps, coeffs};
-  return run_batched(ctx, out, in, nullptr, shapes, count, r, static_cast<cudaStream_t>(stream));
+  return run_batched(ctx, out, in, nullptr, nullptr, shapes, count, r, static_cast<cudaStream_t>(stream));
 }
 
 int muon_ns_product(muon_ctx_t* ctx, const void* p, const void* q, const void* d, void* c, int32_t m, int32_t n,

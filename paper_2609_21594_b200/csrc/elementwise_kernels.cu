@@ -236,6 +236,15 @@ __global__ void __launch_bounds__(256) apply_kernel(ApplyArgs a) {
         } else {
           for (int i = 0; i < nv; ++i) W[off + i] = W[off + i] * decay - step * XConv<XT>::to(xv[i]);
         }
+        if (d.o) {   // the update itself, for the pack that follows (relay broadcast payload)
+          XT* O = static_cast<XT*>(d.o);
+          if (vec) {
+            if (sizeof(XT) == 2) __stcs(reinterpret_cast<uint2*>(O + off), *reinterpret_cast<const uint2*>(xv));
+            else __stcs(reinterpret_cast<float4*>(O + off), *reinterpret_cast<const float4*>(xv));
+          } else {
+            for (int i = 0; i < nv; ++i) O[off + i] = xv[i];
+          }
+        }
       } else {
         XT* O = static_cast<XT*>(d.w);
         if (vec) {
