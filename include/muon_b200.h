@@ -44,6 +44,7 @@ extern "C" {
 #define MUON_ERR_WORKSPACE_TOO_SMALL -4  /* muon_set_workspace not called, or buffer smaller than required  */
 #define MUON_ERR_CUDA               -5   /* a CUDA runtime/driver call failed (no usable device, launch...) */
 #define MUON_ERR_DEVICE_TIMEOUT     -6   /* a bounded device-side wait gave up (see muon_last_device_status) */
+#define MUON_ERR_TOO_LARGE          -7   /* the matrix needs more than the fixed built-in scratch (muon_orthogonalize_static) */
 
 /* ------------------------------------------------------------------ enums */
 #define MUON_DTYPE_BF16 0
@@ -209,6 +210,37 @@ int muon_ns_product(muon_ctx_t* ctx, const void* p, const void* q, const void* d
                     int32_t m, int32_t n, int32_t k, int32_t ldp, int32_t ldq, int32_t ldc,
                     int64_t stride_p, int64_t stride_q, int64_t stride_c, int32_t batch, int32_t nn,
                     float alpha, float beta, const float* gamma, int32_t gamma_mode, void* stream);
+
+/* muon_orthogonalize_static: muon_orthogonalize_batched for ONE matrix, for callers that cannot
+ * allocate device memory.  (The paper has no counterpart; it exists for integration reasons only.)
+ *
+ * Who needs it: code that runs where cudaMalloc is forbidden or unavailable -- inside a memory
+ * pool or allocator callback, in a process whose device memory is fully pre-assigned by another
+ * runtime, or in a latency-critical section where an allocation's implicit synchronisation is not
+ * acceptable.  Such a caller can create no muon_ctx_t (creation allocates) and own no workspace.
+ * This entry point therefore takes no context and allocates nothing: it calls neither cudaMalloc
+ * nor cudaFree nor any allocating library routine, on the device or for pinned host memory.  All
+ * scratch (the two X iterates, A, B, the norm partial sums and a small descriptor) lives in one
+ * fixed array of MUON_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that loads
+ * the library holds that much memory until the process exits.
+ *
+ *   in, out : device, rows x cols row-major, bf16 under MUON_NS_BF16 / fp32 under MUON_NS_FP32,
+ *             16-byte aligned, not aliased; the caller owns them
+ *   status  : optional device int32 the caller has zeroed; a bounded device-side wait that expires
+ *             writes a non-zero code there (NULL: such a code is dropped)
+ *   flags   : MUON_ORTHO_NO_NORMALIZE or 0;  coeffs: host, 3 floats
+ * Limits: a matrix whose Newton-Schulz workspace exceeds the array (for bf16 roughly
+ * 4*rows*cols + 4*min(rows,cols)^2 bytes; 1024 x 1024 fits, 2048 x 2048 does not) is rejected
+ * with MUON_ERR_TOO_LARGE and nothing is launched.
+ * Set-up: the first call on each device resolves the array's device address and the driver's
+ * tensor-map encoder; make that first call outside any stream capture.
+ * Sharing: all calls on a device use the same array, which keeps whatever the previous call left;
+ * the entry point rewrites every element it later reads, so no clearing by the caller is needed,
+ * but two calls whose device work overlaps in time (different streams without ordering) race. */
+#define MUON_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u + 4096u)
+int muon_orthogonalize_static(const void* in, void* out, int32_t rows, int32_t cols, int32_t ns_precision,
+                              int32_t ns_steps, const float* coeffs, float eps, uint32_t flags,
+                              int32_t* status, void* stream);
 
 /* Device-side status word: the tensor-core pipeline bounds every wait on a barrier; a wait
  * that gives up records a non-zero code here and the kernel exits cleanly.  Reads the word

@@ -20,6 +20,8 @@ if not os.path.exists(LIB_PATH):
 lib = C.CDLL(LIB_PATH)
 
 OK, ERR_INVALID_ARG, ERR_BAD_LAYOUT, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_DEVICE_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
+ERR_TOO_LARGE = -7
+STATIC_SCRATCH_BYTES = 16 * 1024 * 1024 + 4096
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 NS_BF16, NS_FP32 = 0, 1
 ENGINE_TENSOR, ENGINE_CUDA_CORE = 0, 1
@@ -73,6 +75,8 @@ _sig = {
     "muon_ns_product": (C.c_int, [_vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                   C.c_int64, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_float, C.c_float, _vp,
                                   C.c_int32, _vp]),
+    "muon_orthogonalize_static": (C.c_int, [_vp, _vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_float),
+                                            C.c_float, C.c_uint32, _vp, _vp]),
     "muon_last_device_status": (C.c_int, [_vp, _vp, C.POINTER(C.c_int32)]),
     "muon_profile_enable": (C.c_int, [_vp, C.c_int32]),
     "muon_profile_reset": (C.c_int, [_vp]),
@@ -158,6 +162,16 @@ def make_layout_desc(layout, elem_size: int):
 
 def muon_layout_validate(desc: LayoutDesc) -> int:
     return int(lib.muon_layout_validate(C.byref(desc)))
+
+
+def muon_orthogonalize_static(inp, out, rows, cols, ns_precision, ns_steps, coeffs, eps=1e-7, flags=0, status=None,
+                              stream=None) -> None:
+    """One-matrix Newton-Schulz with the library's built-in scratch: needs no Context and allocates nothing.
+    `inp`, `out` (and the optional zeroed int32 `status`) are CUDA tensors the caller owns."""
+    co = (C.c_float * 3)(*[float(c) for c in coeffs[:3]])
+    _check(lib.muon_orthogonalize_static(inp.data_ptr(), out.data_ptr(), rows, cols, ns_precision, ns_steps, co, eps, flags,
+                                         None if status is None else status.data_ptr(), _stream(stream)),
+           "muon_orthogonalize_static")
 
 
 class Layout:

@@ -572,8 +572,104 @@ const char* muon_status_string(int status) {
     case MUON_ERR_WORKSPACE_TOO_SMALL: return "workspace missing or too small";
     case MUON_ERR_CUDA: return "CUDA error or no usable sm_100 device";
     case MUON_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    case MUON_ERR_TOO_LARGE: return "matrix too large for the fixed built-in scratch";
     default: return "unknown status";
   }
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant: one matrix, all scratch in a fixed device array that ships with the
+// library image.  The array's name is only a host-side handle here; kernels need its device
+// address, which differs per GPU, so it is looked up once per device with that device current.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[MUON_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+constexpr size_t kStaticHeader = 4096;      // [0,256): spare status word, [256,512): matrix descriptor
+void* g_static_ptr[kMaxDevices] = {};       // device address of g_static_scratch, per device ordinal
+void* g_static_encode = nullptr;            // cuTensorMapEncodeTiled
+
+int static_setup(int dev, void** ptr_out) {
+  if (dev < 0 || dev >= kMaxDevices) return MUON_ERR_UNSUPPORTED;
+  if (!g_static_ptr[dev]) {
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return MUON_ERR_CUDA;
+    if (prop.major != 10) return MUON_ERR_UNSUPPORTED;
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return MUON_ERR_CUDA;
+    if (!g_static_encode) {
+      cudaDriverEntryPointQueryResult qres;
+      void* fn = nullptr;
+      if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+          qres != cudaDriverEntryPointSuccess || !fn)
+        return MUON_ERR_CUDA;
+      g_static_encode = fn;
+    }
+    g_static_ptr[dev] = p;
+  }
+  *ptr_out = g_static_ptr[dev];
+  return MUON_OK;
+}
+
+}  // namespace
+
+extern "C" int muon_orthogonalize_static(const void* in, void* out, int32_t rows, int32_t cols, int32_t ns_precision,
+                                         int32_t ns_steps, const float* coeffs, float eps, uint32_t flags,
+                                         int32_t* status, void* stream) {
+  if (rows < 0 || cols < 0 || ns_steps < 1 || ns_steps > 64 || !coeffs) return MUON_ERR_INVALID_ARG;
+  if (ns_precision != MUON_NS_BF16 && ns_precision != MUON_NS_FP32) return MUON_ERR_INVALID_ARG;
+  if (flags & ~MUON_ORTHO_NO_NORMALIZE) return MUON_ERR_INVALID_ARG;
+  if (!(eps >= 0.f) || !std::isfinite(eps)) return MUON_ERR_INVALID_ARG;
+  for (int i = 0; i < 3; ++i)
+    if (!std::isfinite(coeffs[i])) return MUON_ERR_INVALID_ARG;
+  if (rows == 0 || cols == 0) return MUON_OK;
+  if (!in || !out || in == out || !aligned(in, 16) || !aligned(out, 16)) return MUON_ERR_INVALID_ARG;
+
+  // A stack context: it only carries options and pointers into the fixed array; nothing is allocated.
+  muon_ctx ctx;
+  muon_default_options(&ctx.opt);
+  ctx.opt.ns_precision = ns_precision;
+  ctx.opt.eps = eps;
+  Chunk ch;                                    // one matrix, one chunk, described on the stack
+  ch.s = std::min(rows, cols);
+  ch.l = std::max(rows, cols);
+  ch.ldx = (ch.l + 7) / 8 * 8;
+  ch.lda = (ch.s + 7) / 8 * 8;
+  ch.count = 1;
+  ch.tiles_per_mat = ((ch.s + kElemTile - 1) / kElemTile) * ((ch.l + kElemTile - 1) / kElemTile);
+  ch.desc_begin = 0;
+  const WsCarve carve = carve_chunk(ctx.opt, ch);
+  if (carve.total + kStaticHeader > size_t(MUON_STATIC_SCRATCH_BYTES)) return MUON_ERR_TOO_LARGE;
+
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MUON_ERR_CUDA;
+  void* base = nullptr;
+  const int rc = static_setup(dev, &base);
+  if (rc != MUON_OK) return rc;
+  char* sb = static_cast<char*>(base);
+  ctx.device = dev;
+  ctx.tmap_encode = g_static_encode;
+  ctx.d_status = status ? status : reinterpret_cast<int32_t*>(sb);
+  ctx.ws = sb + kStaticHeader;
+  ctx.ws_bytes = size_t(MUON_STATIC_SCRATCH_BYTES) - kStaticHeader;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  MatDesc d;
+  std::memset(&d, 0, sizeof(d));
+  d.w = out;
+  d.g = in;
+  d.rows = rows;
+  d.cols = cols;
+  d.transposed = rows > cols ? 1 : 0;
+  d.scale = 0.f;
+  MatDesc* d_desc = reinterpret_cast<MatDesc*>(sb + 256);
+  // Pageable source: the runtime stages the 48 bytes before returning, so `d` may go out of scope.
+  if (cudaMemcpyAsync(d_desc, &d, sizeof(d), cudaMemcpyHostToDevice, st) != cudaSuccess) return MUON_ERR_CUDA;
+  ChunkRun r{0, (flags & MUON_ORTHO_NO_NORMALIZE) ? 0 : 1, 0.f, 0.f, 0.f, ns_steps, coeffs};
+  return run_chunk(&ctx, ch, d_desc, r, st);
+}
+
