@@ -199,6 +199,9 @@ int muon_orthogonalize_batched(muon_ctx_t* ctx, const void* const* in, void* con
  * three products of one step of Eq. 1), exposed for per-kernel parity checks and timing:
  *     C[i] = gamma_i * (beta * D[i] + alpha * P[i] Q[i]^T)        nn = 0, P: m x k, Q: n x k
  *     C[i] = gamma_i * (beta * D[i] + alpha * P[i] Q[i])          nn = 1, P: m x k, Q: k x n
+ *     C[i] = gamma_i * (beta * D[i] + alpha * P[i] P[i]^T)        nn = 2, symmetric rank-k form: q == p,
+ *            m == n, D symmetric (or NULL); only tiles touching the upper triangle are computed and
+ *            the strictly upper ones are mirrored, so C is exactly symmetric
  * for i < batch.  All operands are device pointers to row-major matrices of the NS element type
  * (bf16 under MUON_NS_BF16, fp32 under MUON_NS_FP32) with leading dimensions ldp, ldq, ldc in
  * elements (D shares ldc and stride_c; d may be NULL) and stride_* elements between consecutive

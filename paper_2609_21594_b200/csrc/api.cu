@@ -490,9 +490,10 @@ int muon_ns_product(muon_ctx_t* ctx, const void* p, const void* q, const void* d
   if (!ctx || m < 0 || n < 0 || k < 0 || batch < 0) return MUON_ERR_INVALID_ARG;
   if (m == 0 || n == 0 || batch == 0) return MUON_OK;
   if (!p || !q || !c || k < 1) return MUON_ERR_INVALID_ARG;
-  if (nn != 0 && nn != 1) return MUON_ERR_INVALID_ARG;
+  if (nn < 0 || nn > 2) return MUON_ERR_INVALID_ARG;
+  if (nn == 2 && (m != n || p != q || ldp != ldq || stride_p != stride_q)) return MUON_ERR_INVALID_ARG;
   if (gamma_mode < 0 || gamma_mode > 2 || (gamma_mode && !gamma)) return MUON_ERR_INVALID_ARG;
-  if (ldp < k || ldc < n || ldq < (nn ? n : k)) return MUON_ERR_INVALID_ARG;
+  if (ldp < k || ldc < n || ldq < (nn == 1 ? n : k)) return MUON_ERR_INVALID_ARG;
   if (c == p || c == q || c == d) return MUON_ERR_INVALID_ARG;
   if (!DeviceGuardCheck::ok(ctx)) return MUON_ERR_CUDA;
   GemmArgs g{};
@@ -503,7 +504,7 @@ int muon_ns_product(muon_ctx_t* ctx, const void* p, const void* q, const void* d
   g.batch = batch;
   g.rnorm = gamma;
   g.gamma_mode = gamma ? gamma_mode : 0;
-  g.alpha = alpha; g.beta = beta; g.nn = nn; g.symmetric = 0;
+  g.alpha = alpha; g.beta = beta; g.nn = nn == 1 ? 1 : 0; g.symmetric = nn == 2 ? 1 : 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   Span sp(ctx, MUON_PHASE_NS, st);
   const int nl = run_gemm(ctx, g, st);

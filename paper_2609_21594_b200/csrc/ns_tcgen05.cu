@@ -43,6 +43,8 @@ struct TcArgs {
   int32_t m, n, kdim, ldc;
   int64_t stride_c;
   int32_t batch, tiles_m, tiles_n;
+  int32_t tiles_per_mat;    // tiles_m*tiles_n, or the number of tiles on/above the diagonal when symmetric
+  int32_t symmetric;        // C = C^T: compute tiles that touch the upper triangle, mirror the strictly upper ones
   const float* rnorm;
   int32_t gamma_mode;
   float alpha, beta;
@@ -148,13 +150,30 @@ __host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major) {
 struct Tile {
   int mat, m0, n0;
 };
+// Dense: row blocks vary fastest, so concurrent CTAs share the Q tile.
+// Symmetric (m == n): row block i (128 rows) needs column blocks j >= i/2 (256 columns): the tile then holds
+// at least one element on or above the diagonal.  Rows 2q and 2q+1 both start at column block q; the pair
+// owns 2*(tiles_n - q) tiles, so the pairs before q own 2*q*tiles_n - q*(q-1).
 __device__ __forceinline__ Tile decode_tile(int t, const TcArgs& a) {
-  const int per = a.tiles_m * a.tiles_n;
   Tile r;
-  r.mat = t / per;
-  const int u = t - r.mat * per;
-  r.n0 = (u / a.tiles_m) * BN;     // row blocks vary fastest: concurrent CTAs share the Q tile
-  r.m0 = (u % a.tiles_m) * BM;
+  r.mat = t / a.tiles_per_mat;
+  int u = t - r.mat * a.tiles_per_mat;
+  if (!a.symmetric) {
+    r.n0 = (u / a.tiles_m) * BN;
+    r.m0 = (u % a.tiles_m) * BM;
+    return r;
+  }
+  int q = 0;
+  while (true) {
+    const int rows_in_pair = (2 * q + 1 < a.tiles_m) ? 2 : 1;
+    const int cnt = rows_in_pair * (a.tiles_n - q);
+    if (u < cnt) break;
+    u -= cnt;
+    ++q;
+  }
+  const int w = a.tiles_n - q;
+  r.m0 = (2 * q + u / w) * BM;
+  r.n0 = (q + u % w) * BN;
   return r;
 }
 
@@ -174,7 +193,7 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
   auto tempty_bar = [&](int i) { return bars + uint32_t(2 * STAGES + 2 + i) * 8u; };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_tiles = a.batch * a.tiles_m * a.tiles_n;
+  const int total_tiles = a.batch * a.tiles_per_mat;
   const int num_kb = (a.kdim + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
@@ -290,6 +309,8 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
       const size_t row_off = size_t(tl.mat) * a.stride_c + size_t(row_ok ? row : 0) * a.ldc;
       const __nv_bfloat16* drow = a.d ? a.d + row_off : nullptr;
       __nv_bfloat16* crow = a.c + row_off;
+      __nv_bfloat16* cmat = a.c + size_t(tl.mat) * a.stride_c;
+      const bool mirror = a.symmetric && tl.n0 >= tl.m0 + BM;   // tile lies strictly above the diagonal
       const uint32_t taddr = tmem_base + acc * uint32_t(BN) + (uint32_t(quad * 32) << 16);
 #pragma unroll 1
       for (int cb = 0; cb < BN / 32; ++cb) {
@@ -317,13 +338,20 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
             }
 #pragma unroll
             for (int q = 0; q < 4; ++q) reinterpret_cast<uint4*>(crow + c0)[q] = reinterpret_cast<const uint4*>(out)[q];
+            if (mirror) {   // C[c][row] = C[row][c]: for a fixed c the 32 lanes write 64 contiguous bytes
+              const __nv_bfloat16* oe = reinterpret_cast<const __nv_bfloat16*>(out);
+#pragma unroll
+              for (int j = 0; j < 32; ++j) cmat[size_t(c0 + j) * a.ldc + row] = oe[j];
+            }
           } else {
             for (int j = 0; j < 32; ++j) {
               const int c = c0 + j;
               if (c < a.n) {
                 float x = a.alpha * __uint_as_float(v[j]);
                 if (drow) x += a.beta * __bfloat162float(drow[c]);
-                crow[c] = __float2bfloat16_rn(gamma * x);
+                const __nv_bfloat16 o = __float2bfloat16_rn(gamma * x);
+                crow[c] = o;
+                if (mirror) cmat[size_t(c) * a.ldc + row] = o;
               }
             }
           }
@@ -379,6 +407,7 @@ bool tc_supported(const GemmArgs& a) {
   if ((reinterpret_cast<uintptr_t>(a.p) | reinterpret_cast<uintptr_t>(a.q) | reinterpret_cast<uintptr_t>(a.c) |
        reinterpret_cast<uintptr_t>(a.d)) & 15u)
     return false;
+  if (a.symmetric && (a.nn || a.m != a.n || a.p != a.q || a.ldp != a.ldq || a.stride_p != a.stride_q)) return false;
   const int64_t tiles = int64_t((a.m + BM - 1) / BM) * ((a.n + BN - 1) / BN) * a.batch;
   return tiles < (int64_t(1) << 30);
 }
@@ -410,11 +439,18 @@ int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st) {
   t.batch = a.batch;
   t.tiles_m = (a.m + BM - 1) / BM;
   t.tiles_n = (a.n + BN - 1) / BN;
+  t.symmetric = a.symmetric ? 1 : 0;
+  t.tiles_per_mat = t.tiles_m * t.tiles_n;
+  if (t.symmetric) {
+    int cnt = 0;
+    for (int i = 0; i < t.tiles_m; ++i) cnt += t.tiles_n - i / 2;
+    t.tiles_per_mat = cnt;
+  }
   t.rnorm = a.rnorm;
   t.gamma_mode = a.gamma_mode;
   t.alpha = a.alpha; t.beta = a.beta;
   t.status = ctx->d_status;
-  const int64_t tiles = int64_t(t.tiles_m) * t.tiles_n * t.batch;
+  const int64_t tiles = int64_t(t.tiles_per_mat) * t.batch;
   const unsigned grid = unsigned(tiles < g_num_sms ? tiles : g_num_sms);
   if (a.nn) ns_product_tc_kernel<true><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, t);
   else ns_product_tc_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, t);

@@ -30,26 +30,30 @@ def _run(mb, engine, m, n, k, batch, nn, with_d, gamma_mode, seed):
     ctx = mb.Context(opt)
     rng = np.random.default_rng(seed)
     up8 = lambda x: (x + 7) // 8 * 8
+    sym = nn == 2
     P = [rng.standard_normal((m, k)) for _ in range(batch)]
-    Q = [rng.standard_normal((k, n) if nn else (n, k)) for _ in range(batch)]
+    Q = [rng.standard_normal((k, n) if nn == 1 else (n, k)) for _ in range(batch)]
     D = [rng.standard_normal((m, n)) for _ in range(batch)]
-    ldp, ldq, ldc = up8(k), up8(n if nn else k), up8(n)
+    if sym:
+        assert m == n
+        D = [(d + d.T) / 2 for d in D]
+    ldp, ldq, ldc = up8(k), up8(n if nn == 1 else k), up8(n)
     tP, hP = _padded(P, ldp)
-    tQ, hQ = _padded(Q, ldq)
+    tQ, hQ = (tP, hP) if sym else _padded(Q, ldq)
     tD, hD = _padded(D, ldc)
     tC = torch.full((batch, m, ldc), -7.0, dtype=torch.bfloat16, device="cuda")
     gam = rng.uniform(0.5, 2.0, size=batch).astype(np.float32)
     tG = torch.from_numpy(gam).cuda()
     alpha, beta = 2.0315, -4.775
     ctx.muon_ns_product(tP, tQ, tD if with_d else None, tC, m, n, k, ldp, ldq, ldc, m * ldp, tQ.shape[1] * ldq, m * ldc,
-                        batch, 1 if nn else 0, alpha, beta, tG if gamma_mode else None, gamma_mode)
+                        batch, nn, alpha, beta, tG if gamma_mode else None, gamma_mode)
     torch.cuda.synchronize()
     assert ctx.muon_last_device_status() == 0
     got = host_f64(tC)
     a32, b32 = float(np.float32(alpha)), float(np.float32(beta))
     worst = 0.0
     for i in range(batch):
-        acc = hP[i] @ (hQ[i] if nn else hQ[i].T)
+        acc = hP[i] @ (hQ[i] if nn == 1 else hQ[i].T)
         v = a32 * acc + (b32 * hD[i] if with_d else 0.0)
         g = 1.0 if not gamma_mode else (float(gam[i]) if gamma_mode == 1 else float(gam[i]) ** 2)
         ref = orc.bf16_rne(g * v)
@@ -58,10 +62,12 @@ def _run(mb, engine, m, n, k, batch, nn, with_d, gamma_mode, seed):
         worst = max(worst, rel(out, ref))
         # at most one bf16 ulp apart anywhere (fp32 vs fp64 accumulation can flip a rounding), plus the
         # absolute fp32 accumulation error where the sum cancels
-        mag = np.abs(hP[i]) @ np.abs(hQ[i] if nn else hQ[i].T)
+        mag = np.abs(hP[i]) @ np.abs(hQ[i] if nn == 1 else hQ[i].T)
         slack = abs(g) * (abs(a32) * mag + (abs(b32) * np.abs(hD[i]) if with_d else 0.0)) * 2.0 ** -20
         assert np.all(np.abs(out - ref) <= np.abs(ref) * 2.0 ** -7 + slack)
         assert np.all(got[i, :, n:] == -7.0)          # pad columns of C untouched
+        if sym:
+            assert np.array_equal(out, out.T)         # mirrored stores make the result exactly symmetric
     ctx.close()
     return worst
 
@@ -105,3 +111,17 @@ def test_product_many_tiles_persistent_loop():
 
     assert _run(mb, "tensor", 1024, 1024, 512, 6, 0, True, 1, seed=3) < 3e-3
     assert _run(mb, "tensor", 1024, 2048, 1024, 3, 1, True, 2, seed=4) < 3e-3
+
+
+SYM_CASES = [(128, 64, 1), (256, 320, 2), (384, 136, 3), (200, 1000, 2), (1024, 512, 2), (1408, 256, 1), (37, 53, 2)]
+
+
+@pytest.mark.parametrize("engine", ["tensor", "cuda_core"])
+@pytest.mark.parametrize("case", SYM_CASES)
+def test_symmetric_product(engine, case):
+    """C = gamma (beta D + alpha P P^T): triangular tile schedule with mirrored stores on the tensor engine."""
+    from paper_2609_21594_b200 import binding as mb
+
+    s, k, batch = case
+    assert _run(mb, engine, s, s, k, batch, 2, False, 0, seed=s + k) < 3e-3
+    assert _run(mb, engine, s, s, k, batch, 2, True, 2, seed=s + k + 1) < 3e-3
