@@ -208,7 +208,8 @@ int muon_orthogonalize_batched(muon_ctx_t* ctx, const void* const* in, void* con
  * matrices.  gamma_i = 1 when gamma is NULL, else gamma[i] (gamma_mode 1) or gamma[i]^2
  * (gamma_mode 2), gamma being a device array of `batch` floats.  For the tensor-core engine bases
  * must be 16-byte aligned and every ld/stride a multiple of 8 elements; other cases run on CUDA
- * cores.  C must not alias P, Q or D. */
+ * cores.  C must not alias P, Q or D.  The tensor engine stores C in 16-byte pieces: the padding
+ * columns [n, ldc) of a row may be overwritten up to the next multiple of 8 elements. */
 int muon_ns_product(muon_ctx_t* ctx, const void* p, const void* q, const void* d, void* c,
                     int32_t m, int32_t n, int32_t k, int32_t ldp, int32_t ldq, int32_t ldc,
                     int64_t stride_p, int64_t stride_q, int64_t stride_c, int32_t batch, int32_t nn,

@@ -32,7 +32,9 @@ constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;          // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;          // 32 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int EPI_COLS = 64;                         // columns per epilogue chunk (one 128-byte swizzle row of bf16)
+constexpr int EPI_BYTES = BM * EPI_COLS * 2;         // 16 KiB staging buffer, two of them
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * EPI_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int TMEM_COLS = 512;
 constexpr int NUM_THREADS = 192;
 constexpr long long WAIT_CYCLES = 4000000000LL;   // ~2 s at 1.9 GHz: far beyond any legitimate wait
@@ -96,6 +98,18 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
+__device__ __forceinline__ void tma_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void tma_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -179,14 +193,19 @@ __device__ __forceinline__ Tile decode_tile(int t, const TcArgs& a) {
 
 template <bool NN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q, const TcArgs a) {
+ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q,
+                     const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_c, const TcArgs a) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;            // swizzled tiles need 1024-byte alignment
   uint8_t* gen_base = smem_raw + (base - raw);
-  const uint32_t bars = base + STAGES * STAGE_BYTES;        // barrier block follows the tiles
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + STAGES * STAGE_BYTES + 128);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + STAGES * STAGE_BYTES + 136);
+  const uint32_t epi_base = base + STAGES * STAGE_BYTES;    // two epilogue staging buffers follow the ring
+  constexpr int BAR_OFF = STAGES * STAGE_BYTES + 2 * EPI_BYTES;
+  const uint32_t bars = base + BAR_OFF;                     // barrier block follows the buffers
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + BAR_OFF + 128);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + BAR_OFF + 136);
+  auto dfull_bar = [&](int i) { return bars + uint32_t(2 * STAGES + 4 + i) * 8u; };
+  const uint32_t egroup_bar = bars + uint32_t(2 * STAGES + 6) * 8u;   // 128-thread rendezvous of the epilogue group
   auto full_bar = [&](int s) { return bars + uint32_t(s) * 8u; };
   auto empty_bar = [&](int s) { return bars + uint32_t(STAGES + s) * 8u; };
   auto tfull_bar = [&](int i) { return bars + uint32_t(2 * STAGES + i) * 8u; };
@@ -204,7 +223,9 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
     for (int i = 0; i < 2; ++i) {
       mbar_init(tfull_bar(i), 1);
       mbar_init(tempty_bar(i), 4);
+      mbar_init(dfull_bar(i), 1);
     }
+    mbar_init(egroup_bar, 4);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -291,77 +312,110 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps
+    // Thread = one accumulator row (TMEM lane).  The tile leaves in four 64-column chunks through two
+    // 128B-swizzled staging buffers: TMA brings the D chunk in, every thread turns its own row of D
+    // into its row of C in place, TMA stores the chunk.  All global traffic of the epilogue is
+    // therefore full-line bulk traffic; only the mirrored copy of a symmetric tile uses plain stores.
     const int quad = warp & 3;                     // TMEM lane quadrant this warp may read
-    uint32_t tile_it = 0;
+    const int etid = threadIdx.x - 64;             // 0..127 within the epilogue group
+    const bool leader = etid == 0;
+    const int lrow = quad * 32 + lane;             // row inside the tile
+    uint32_t tile_it = 0, g = 0;                   // g counts chunks across tiles (buffer = g & 1)
+    uint32_t eph = 0;                              // phase of the group rendezvous
     bool ok = true;
+    // Rendezvous of the four epilogue warps on an mbarrier (one arrival per warp), so that this wait is
+    // bounded like every other.
+    auto group_sync = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(egroup_bar);
+      const bool done = mbar_wait(egroup_bar, eph, abort_flag);
+      eph ^= 1u;
+      return done;
+    };
     for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_it) {
       const Tile tl = decode_tile(t, a);
       const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-      if (!mbar_wait(tfull_bar(int(acc)), aph, abort_flag)) { ok = false; break; }
-      tc_fence_after();
       float gamma = 1.f;
       if (a.gamma_mode) {
         const float r = a.rnorm[tl.mat];
         gamma = a.gamma_mode == 1 ? r : r * r;
       }
-      const int row = tl.m0 + quad * 32 + lane;
+      const int row = tl.m0 + lrow;
       const bool row_ok = row < a.m;
-      const size_t row_off = size_t(tl.mat) * a.stride_c + size_t(row_ok ? row : 0) * a.ldc;
-      const __nv_bfloat16* drow = a.d ? a.d + row_off : nullptr;
-      __nv_bfloat16* crow = a.c + row_off;
       __nv_bfloat16* cmat = a.c + size_t(tl.mat) * a.stride_c;
       const bool mirror = a.symmetric && tl.n0 >= tl.m0 + BM;   // tile lies strictly above the diagonal
       const uint32_t taddr = tmem_base + acc * uint32_t(BN) + (uint32_t(quad * 32) << 16);
+      bool acc_ready = false;
 #pragma unroll 1
-      for (int cb = 0; cb < BN / 32; ++cb) {
-        const int c0 = tl.n0 + cb * 32;
-        if (c0 >= a.n) break;                       // warp-uniform
-        uint32_t v[32];
-        tc_ld32(taddr + uint32_t(cb * 32), v);
+      for (int cb = 0; cb < BN / EPI_COLS; ++cb, ++g) {
+        const int c0 = tl.n0 + cb * EPI_COLS;
+        if (c0 >= a.n) break;                       // uniform over the group
+        const uint32_t b = g & 1u;
+        const uint32_t ebuf = epi_base + b * EPI_BYTES;
+        if (leader) {
+          tma_wait_read<1>();                       // the store that last used this buffer has read it
+          if (a.d) {
+            mbar_expect_tx(dfull_bar(int(b)), EPI_BYTES);
+            tma_load_3d(ebuf, &map_d, dfull_bar(int(b)), c0, tl.m0, tl.mat);
+          }
+        }
+        if (!acc_ready) {
+          if (!mbar_wait(tfull_bar(int(acc)), aph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          acc_ready = true;
+        }
+        if (a.d) {
+          if (!mbar_wait(dfull_bar(int(b)), (g >> 1) & 1u, abort_flag)) { ok = false; break; }
+        } else {
+          if (!group_sync()) { ok = false; break; }  // leader's wait_group above frees the buffer for everyone
+        }
+        uint32_t v[64];
+        tc_ld32(taddr + uint32_t(cb * EPI_COLS), *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+        tc_ld32(taddr + uint32_t(cb * EPI_COLS + 32), *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
         tc_wait_ld();
-        if (row_ok) {
-          if (c0 + 32 <= a.n) {
-            alignas(16) __nv_bfloat16 dv[32];
-            if (drow) {
+        const uint32_t srow = ebuf + uint32_t(lrow) * 128u;
 #pragma unroll
-              for (int q = 0; q < 4; ++q) reinterpret_cast<uint4*>(dv)[q] = reinterpret_cast<const uint4*>(drow + c0)[q];
+        for (int q = 0; q < 8; ++q) {               // 16-byte piece q of the row sits at piece q ^ (row & 7)
+          const uint32_t addr = srow + (uint32_t(q ^ (lrow & 7)) << 4);
+          uint32_t d0 = 0, d1 = 0, d2 = 0, d3 = 0;
+          if (a.d) asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3) : "r"(addr));
+          const uint32_t dd[4] = {d0, d1, d2, d3};
+          uint32_t oo[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float x0 = a.alpha * __uint_as_float(v[q * 8 + 2 * e]), x1 = a.alpha * __uint_as_float(v[q * 8 + 2 * e + 1]);
+            if (a.d) {
+              const __nv_bfloat162 dp = *reinterpret_cast<const __nv_bfloat162*>(&dd[e]);
+              x0 += a.beta * __low2float(dp);
+              x1 += a.beta * __high2float(dp);
             }
-            alignas(16) __nv_bfloat162 out[16];
+            const __nv_bfloat162 o = __floats2bfloat162_rn(gamma * x0, gamma * x1);
+            oo[e] = *reinterpret_cast<const uint32_t*>(&o);
+          }
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(oo[0]), "r"(oo[1]), "r"(oo[2]), "r"(oo[3]) : "memory");
+          if (mirror && row_ok) {                   // C[c][row] = C[row][c]: 32 lanes write 64 contiguous bytes per c
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              float x0 = a.alpha * __uint_as_float(v[2 * j]), x1 = a.alpha * __uint_as_float(v[2 * j + 1]);
-              if (drow) {
-                x0 += a.beta * __bfloat162float(dv[2 * j]);
-                x1 += a.beta * __bfloat162float(dv[2 * j + 1]);
-              }
-              out[j] = __floats2bfloat162_rn(gamma * x0, gamma * x1);
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) reinterpret_cast<uint4*>(crow + c0)[q] = reinterpret_cast<const uint4*>(out)[q];
-            if (mirror) {   // C[c][row] = C[row][c]: for a fixed c the 32 lanes write 64 contiguous bytes
-              const __nv_bfloat16* oe = reinterpret_cast<const __nv_bfloat16*>(out);
-#pragma unroll
-              for (int j = 0; j < 32; ++j) cmat[size_t(c0 + j) * a.ldc + row] = oe[j];
-            }
-          } else {
-            for (int j = 0; j < 32; ++j) {
-              const int c = c0 + j;
-              if (c < a.n) {
-                float x = a.alpha * __uint_as_float(v[j]);
-                if (drow) x += a.beta * __bfloat162float(drow[c]);
-                const __nv_bfloat16 o = __float2bfloat16_rn(gamma * x);
-                crow[c] = o;
-                if (mirror) cmat[size_t(c) * a.ldc + row] = o;
-              }
+            for (int e = 0; e < 4; ++e) {
+              const int c = c0 + q * 8 + 2 * e;
+              const __nv_bfloat162 o = *reinterpret_cast<const __nv_bfloat162*>(&oo[e]);
+              if (c < a.n) cmat[size_t(c) * a.ldc + row] = __low2bfloat16(o);
+              if (c + 1 < a.n) cmat[size_t(c + 1) * a.ldc + row] = __high2bfloat16(o);
             }
           }
         }
-        __syncwarp();
+        fence_async_smem();                         // generic-proxy writes -> visible to the TMA store
+        if (!group_sync()) { ok = false; break; }
+        if (leader) {
+          tma_store_3d(&map_c, ebuf, c0, tl.m0, tl.mat);   // rows/columns beyond the matrix are clipped
+          tma_commit();
+        }
       }
+      if (!ok) break;
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(int(acc)));
     }
+    if (leader) tma_wait_all();                     // every store has landed before the CTA retires
     if (!ok && lane == 0) {
       *abort_flag = 1;
       atomicExch(a.status, 4);
@@ -431,6 +485,10 @@ int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st) {
   } else {      // Q: rows = kdim, cols = n; four 64(k) x 64(n) boxes per stage
     if (!encode_map(ctx->tmap_encode, &map_q, a.q, a.n, a.kdim, a.batch, a.ldq, a.stride_q, BK)) return MUON_ERR_CUDA;
   }
+  // C (store) and D (load) chunks: 128 rows x 64 columns
+  CUtensorMap map_c, map_d;
+  if (!encode_map(ctx->tmap_encode, &map_c, a.c, a.n, a.m, a.batch, a.ldc, a.stride_c, BM)) return MUON_ERR_CUDA;
+  if (!encode_map(ctx->tmap_encode, &map_d, a.d ? a.d : a.c, a.n, a.m, a.batch, a.ldc, a.stride_c, BM)) return MUON_ERR_CUDA;
   TcArgs t;
   t.d = static_cast<const __nv_bfloat16*>(a.d);
   t.c = static_cast<__nv_bfloat16*>(a.c);
@@ -452,8 +510,8 @@ int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st) {
   t.status = ctx->d_status;
   const int64_t tiles = int64_t(t.tiles_per_mat) * t.batch;
   const unsigned grid = unsigned(tiles < g_num_sms ? tiles : g_num_sms);
-  if (a.nn) ns_product_tc_kernel<true><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, t);
-  else ns_product_tc_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, t);
+  if (a.nn) ns_product_tc_kernel<true><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, map_d, map_c, t);
+  else ns_product_tc_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, map_d, map_c, t);
   return cudaGetLastError() == cudaSuccess ? 1 : MUON_ERR_CUDA;
 }
 
