@@ -53,8 +53,9 @@ extern "C" {
 #define MUON_NS_BF16 0   /* bf16 operands, fp32 accumulation on the tensor cores (Section 6.3: "bf16 arithmetic") */
 #define MUON_NS_FP32 1   /* every product and intermediate in fp32 (no counterpart in the paper; accuracy anchor)  */
 
-#define MUON_ENGINE_TENSOR    0
-#define MUON_ENGINE_CUDA_CORE 1
+#define MUON_ENGINE_TENSOR      0   /* tensor cores; CTA pairs (cta_group::2) wherever a matrix has more than 128 rows */
+#define MUON_ENGINE_CUDA_CORE   1
+#define MUON_ENGINE_TENSOR_1CTA 2   /* tensor cores, single-CTA kernel only (cross-check of the paired kernel)        */
 
 /* flags of muon_orthogonalize_batched */
 #define MUON_ORTHO_NO_NORMALIZE 1u  /* treat the input as X_0 already (r = 1); used for single-step checks */
@@ -97,8 +98,8 @@ typedef struct {
   int32_t nesterov;        /* 1: u = G + mu*M' (Section 7 set-up), 0: u = M'                                 */
   int32_t coeffs_per_step; /* 0: coeffs[3] used at every step; 1: coeffs[3*ns_steps], (a_k,b_k,c_k) per step */
   float   eps;             /* epsilon of Eq. 1, added to the Frobenius norm; default 1e-7                    */
-  int32_t engine;          /* MUON_ENGINE_TENSOR (default) | MUON_ENGINE_CUDA_CORE (bf16 products on CUDA cores;   */
-                           /* slow cross-check of the tensor-core engine; fp32 NS always runs on CUDA cores)        */
+  int32_t engine;          /* MUON_ENGINE_TENSOR (default) | MUON_ENGINE_TENSOR_1CTA | MUON_ENGINE_CUDA_CORE (bf16  */
+                           /* products on CUDA cores; slow cross-check); fp32 NS always runs on CUDA cores          */
   int64_t chunk_elems;     /* batching cap in elements per batched NS invocation; default 1<<29 (Section 6.3) */
 } muon_options_t;
 

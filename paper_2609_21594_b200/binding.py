@@ -24,7 +24,7 @@ ERR_TOO_LARGE = -7
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024 + 4096
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 NS_BF16, NS_FP32 = 0, 1
-ENGINE_TENSOR, ENGINE_CUDA_CORE = 0, 1
+ENGINE_TENSOR, ENGINE_CUDA_CORE, ENGINE_TENSOR_1CTA = 0, 1, 2
 ORTHO_NO_NORMALIZE = 1
 PHASE_MOMENTUM, PHASE_NS, PHASE_UPDATE, PHASE_GATHER, PHASE_SCATTER = range(5)
 PHASE_NAMES = ("momentum", "ns", "update", "gather", "scatter")

@@ -22,7 +22,7 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 bool valid_options(const muon_options_t& o) {
   if (o.grad_dtype != MUON_DTYPE_BF16 && o.grad_dtype != MUON_DTYPE_FP32) return false;
   if (o.ns_precision != MUON_NS_BF16 && o.ns_precision != MUON_NS_FP32) return false;
-  if (o.engine != MUON_ENGINE_TENSOR && o.engine != MUON_ENGINE_CUDA_CORE) return false;
+  if (o.engine != MUON_ENGINE_TENSOR && o.engine != MUON_ENGINE_CUDA_CORE && o.engine != MUON_ENGINE_TENSOR_1CTA) return false;
   if (o.nesterov != 0 && o.nesterov != 1) return false;
   if (o.coeffs_per_step != 0 && o.coeffs_per_step != 1) return false;
   if (!(o.eps >= 0.f) || !std::isfinite(o.eps)) return false;
@@ -102,8 +102,10 @@ Plan* get_plan(muon_ctx* ctx, const muon_shape_t* shapes, int32_t count, int* st
 }
 
 int run_gemm(muon_ctx* ctx, const GemmArgs& g, cudaStream_t st) {
-  if (ctx->opt.ns_precision == MUON_NS_BF16 && ctx->opt.engine == MUON_ENGINE_TENSOR && tc_supported(g))
+  if (ctx->opt.ns_precision == MUON_NS_BF16 && ctx->opt.engine != MUON_ENGINE_CUDA_CORE && tc_supported(g)) {
+    if (ctx->opt.engine == MUON_ENGINE_TENSOR && tc_pair_supported(g)) return launch_gemm_tc_pair(ctx, g, st);
     return launch_gemm_tc(ctx, g, st);
+  }
   return launch_gemm_simt(g, ctx->opt.ns_precision, st);
 }
 

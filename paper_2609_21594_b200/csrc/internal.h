@@ -148,5 +148,7 @@ struct GemmArgs {
 int launch_gemm_simt(const GemmArgs& a, int ns_precision, cudaStream_t st);
 int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st);   // tcgen05 engine (bf16 only)
 bool tc_supported(const GemmArgs& a);
+int launch_gemm_tc_pair(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st);   // two-CTA (cta_group::2) variant
+bool tc_pair_supported(const GemmArgs& a);
 
 }  // namespace muon

@@ -26,7 +26,7 @@ def _padded(vals_list, ld):
 
 
 def _run(mb, engine, m, n, k, batch, nn, with_d, gamma_mode, seed):
-    opt = mb.muon_default_options(engine=mb.ENGINE_TENSOR if engine == "tensor" else mb.ENGINE_CUDA_CORE)
+    opt = mb.muon_default_options(engine={"tensor": mb.ENGINE_TENSOR, "tensor_1cta": mb.ENGINE_TENSOR_1CTA, "cuda_core": mb.ENGINE_CUDA_CORE}[engine])
     ctx = mb.Context(opt)
     rng = np.random.default_rng(seed)
     up8 = lambda x: (x + 7) // 8 * 8
@@ -88,7 +88,7 @@ CASES = [
 ]
 
 
-@pytest.mark.parametrize("engine", ["tensor", "cuda_core"])
+@pytest.mark.parametrize("engine", ["tensor", "tensor_1cta", "cuda_core"])
 @pytest.mark.parametrize("nn", [0, 1])
 @pytest.mark.parametrize("case", CASES)
 def test_product_plain(engine, nn, case):
@@ -98,7 +98,7 @@ def test_product_plain(engine, nn, case):
     assert _run(mb, engine, m, n, k, batch, nn, False, 0, seed=m * 7 + n) < 3e-3
 
 
-@pytest.mark.parametrize("engine", ["tensor", "cuda_core"])
+@pytest.mark.parametrize("engine", ["tensor", "tensor_1cta", "cuda_core"])
 @pytest.mark.parametrize("nn", [0, 1])
 @pytest.mark.parametrize("gamma_mode", [0, 1, 2])
 def test_product_fused_epilogue(engine, nn, gamma_mode):
@@ -119,7 +119,7 @@ def test_product_many_tiles_persistent_loop():
 SYM_CASES = [(128, 64, 1), (256, 320, 2), (384, 136, 3), (200, 1000, 2), (1024, 512, 2), (1408, 256, 1), (37, 53, 2)]
 
 
-@pytest.mark.parametrize("engine", ["tensor", "cuda_core"])
+@pytest.mark.parametrize("engine", ["tensor", "tensor_1cta", "cuda_core"])
 @pytest.mark.parametrize("case", SYM_CASES)
 def test_symmetric_product(engine, case):
     """C = gamma (beta D + alpha P P^T): triangular tile schedule with mirrored stores on the tensor engine."""

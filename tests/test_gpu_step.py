@@ -18,13 +18,13 @@ pytestmark = pytest.mark.gpu
 TOL_BF16 = 1e-2
 TOL_FP32 = 1e-4
 TOL_SINGLE_STEP = 2e-3
-ENGINES = ["tensor", "cuda_core"]
+ENGINES = ["tensor", "tensor_1cta", "cuda_core"]
 
 
 def _ctx(mb, precision="bf16", engine="tensor", grad="bf16", **kw):
     opt = mb.muon_default_options(
         ns_precision=mb.NS_BF16 if precision == "bf16" else mb.NS_FP32,
-        engine=mb.ENGINE_TENSOR if engine == "tensor" else mb.ENGINE_CUDA_CORE,
+        engine={"tensor": mb.ENGINE_TENSOR, "tensor_1cta": mb.ENGINE_TENSOR_1CTA, "cuda_core": mb.ENGINE_CUDA_CORE}[engine],
         grad_dtype=mb.DTYPE_BF16 if grad == "bf16" else mb.DTYPE_FP32, **kw)
     return mb.Context(opt)
 
