@@ -169,6 +169,8 @@ __global__ void __launch_bounds__(256) norm_kernel(const float* __restrict__ par
 }
 
 // XT: NS element type; UPD: 1 = weight update, 0 = plain store of O into d.w (element type XT).
+// The weights of all four passes are requested first, then the O tile (through shared memory when it has
+// to be transposed back), then the arithmetic and the stores.
 template <typename XT, bool UPD>
 __global__ void __launch_bounds__(256) apply_kernel(ApplyArgs a) {
   __shared__ XT tile[T][PADT];
@@ -178,80 +180,111 @@ __global__ void __launch_bounds__(256) apply_kernel(ApplyArgs a) {
   const int tiles_c = (d.cols + T - 1) / T;
   const int r0 = (t / tiles_c) * T, c0 = (t % tiles_c) * T;
   const XT* __restrict__ X = static_cast<const XT*>(a.x) + size_t(mat) * a.s * a.ldx;
+  float* __restrict__ W = static_cast<float*>(d.w);
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const bool vec = (d.cols & 3) == 0;
+  const int cc = tx * 4, c = c0 + cc;
+  const int nv = min(4, d.cols - c);
+  float w[4][4];
+  alignas(16) XT xv[4][4];
+  // ---- loads: W (update mode), then O
+  if (UPD) {
+#pragma unroll
+    for (int pass = 0; pass < 4; ++pass) {
+      const int r = r0 + ty + pass * 16;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) w[pass][i] = 0.f;
+      if (r < d.rows && nv > 0) {
+        const size_t off = size_t(r) * d.cols + c;
+        if (vec) {
+          const float4 wv = __ldcs(reinterpret_cast<const float4*>(W + off));
+          w[pass][0] = wv.x; w[pass][1] = wv.y; w[pass][2] = wv.z; w[pass][3] = wv.w;
+        } else {
+          for (int i = 0; i < nv; ++i) w[pass][i] = W[off + i];
+        }
+      }
+    }
+  }
   if (d.transposed) {
     // load X[c][r] coalesced along r, then read it back transposed
 #pragma unroll
     for (int pass = 0; pass < 4; ++pass) {
-      const int cc = ty + pass * 16, rr = tx * 4;
-      const int c = c0 + cc, r = r0 + rr;
-      if (c < d.cols && r < d.rows) {
-        const XT* src = X + size_t(c) * a.ldx + r;
-        const int nv = min(4, d.rows - r);
-        alignas(16) XT xv[4];
-        if (nv == 4) {
-          if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(xv) = *reinterpret_cast<const uint2*>(src);
-          else *reinterpret_cast<float4*>(xv) = *reinterpret_cast<const float4*>(src);
+      const int cc2 = ty + pass * 16, rr = tx * 4;
+      const int c2 = c0 + cc2, r = r0 + rr;
+      if (c2 < d.cols && r < d.rows) {
+        const XT* src = X + size_t(c2) * a.ldx + r;
+        const int nr = min(4, d.rows - r);
+        alignas(16) XT tv[4];
+        if (nr == 4) {
+          if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(tv) = __ldcs(reinterpret_cast<const uint2*>(src));
+          else *reinterpret_cast<float4*>(tv) = __ldcs(reinterpret_cast<const float4*>(src));
         } else {
-          for (int i = 0; i < 4; ++i) xv[i] = i < nv ? src[i] : XConv<XT>::from(0.f);
+          for (int i = 0; i < 4; ++i) tv[i] = i < nr ? src[i] : XConv<XT>::from(0.f);
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) tile[rr + i][cc] = xv[i];
+        for (int i = 0; i < 4; ++i) tile[rr + i][cc2] = tv[i];
       }
     }
     __syncthreads();
-  }
-  const float decay = 1.0f - a.lr * a.wd;
-  const float step = a.lr * d.scale;
-  const bool vec = (d.cols & 3) == 0;
 #pragma unroll
-  for (int pass = 0; pass < 4; ++pass) {
-    const int rr = ty + pass * 16, cc = tx * 4;
-    const int r = r0 + rr, c = c0 + cc;
-    if (r < d.rows && c < d.cols) {
-      const int nv = min(4, d.cols - c);
-      alignas(16) XT xv[4];
-      if (d.transposed) {
+    for (int pass = 0; pass < 4; ++pass) {
+      const int rr = ty + pass * 16;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) xv[i] = tile[rr][cc + i];
-      } else {
+      for (int i = 0; i < 4; ++i) xv[pass][i] = tile[rr][cc + i];
+    }
+  } else {
+#pragma unroll
+    for (int pass = 0; pass < 4; ++pass) {
+      const int r = r0 + ty + pass * 16;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) xv[pass][i] = XConv<XT>::from(0.f);
+      if (r < d.rows && nv > 0) {
         const XT* src = X + size_t(r) * a.ldx + c;
         if (nv == 4) {
-          if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(xv) = *reinterpret_cast<const uint2*>(src);
-          else *reinterpret_cast<float4*>(xv) = *reinterpret_cast<const float4*>(src);
+          if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(xv[pass]) = __ldcs(reinterpret_cast<const uint2*>(src));
+          else *reinterpret_cast<float4*>(xv[pass]) = __ldcs(reinterpret_cast<const float4*>(src));
         } else {
-          for (int i = 0; i < 4; ++i) xv[i] = i < nv ? src[i] : XConv<XT>::from(0.f);
+          for (int i = 0; i < nv; ++i) xv[pass][i] = src[i];
         }
       }
+    }
+  }
+  // ---- arithmetic and stores
+  const float decay = 1.0f - a.lr * a.wd;
+  const float step = a.lr * d.scale;
+#pragma unroll
+  for (int pass = 0; pass < 4; ++pass) {
+    const int r = r0 + ty + pass * 16;
+    if (r < d.rows && nv > 0) {
       const size_t off = size_t(r) * d.cols + c;
       if (UPD) {
-        float* W = static_cast<float*>(d.w);
+        float4 o;
+        o.x = w[pass][0] * decay - step * XConv<XT>::to(xv[pass][0]);
+        o.y = w[pass][1] * decay - step * XConv<XT>::to(xv[pass][1]);
+        o.z = w[pass][2] * decay - step * XConv<XT>::to(xv[pass][2]);
+        o.w = w[pass][3] * decay - step * XConv<XT>::to(xv[pass][3]);
         if (vec) {
-          float4 w = __ldcs(reinterpret_cast<const float4*>(W + off));
-          w.x = w.x * decay - step * XConv<XT>::to(xv[0]);
-          w.y = w.y * decay - step * XConv<XT>::to(xv[1]);
-          w.z = w.z * decay - step * XConv<XT>::to(xv[2]);
-          w.w = w.w * decay - step * XConv<XT>::to(xv[3]);
-          __stcs(reinterpret_cast<float4*>(W + off), w);
+          __stcs(reinterpret_cast<float4*>(W + off), o);
         } else {
-          for (int i = 0; i < nv; ++i) W[off + i] = W[off + i] * decay - step * XConv<XT>::to(xv[i]);
+          const float ov[4] = {o.x, o.y, o.z, o.w};
+          for (int i = 0; i < nv; ++i) W[off + i] = ov[i];
         }
         if (d.o) {   // the update itself, for the pack that follows (relay broadcast payload)
           XT* O = static_cast<XT*>(d.o);
           if (vec) {
-            if (sizeof(XT) == 2) __stcs(reinterpret_cast<uint2*>(O + off), *reinterpret_cast<const uint2*>(xv));
-            else __stcs(reinterpret_cast<float4*>(O + off), *reinterpret_cast<const float4*>(xv));
+            if (sizeof(XT) == 2) __stcs(reinterpret_cast<uint2*>(O + off), *reinterpret_cast<const uint2*>(xv[pass]));
+            else __stcs(reinterpret_cast<float4*>(O + off), *reinterpret_cast<const float4*>(xv[pass]));
           } else {
-            for (int i = 0; i < nv; ++i) O[off + i] = xv[i];
+            for (int i = 0; i < nv; ++i) O[off + i] = xv[pass][i];
           }
         }
       } else {
         XT* O = static_cast<XT*>(d.w);
         if (vec) {
-          if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(O + off) = *reinterpret_cast<const uint2*>(xv);
-          else *reinterpret_cast<float4*>(O + off) = *reinterpret_cast<const float4*>(xv);
+          if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(O + off) = *reinterpret_cast<const uint2*>(xv[pass]);
+          else *reinterpret_cast<float4*>(O + off) = *reinterpret_cast<const float4*>(xv[pass]);
         } else {
-          for (int i = 0; i < nv; ++i) O[off + i] = xv[i];
+          for (int i = 0; i < nv; ++i) O[off + i] = xv[pass][i];
         }
       }
     }
