@@ -274,24 +274,34 @@ def run_ours(args, world, rank, local):
     # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region
     e2e = None
     if not args.no_e2e:
-        host_in = torch.empty(layout.flat_len, dtype=torch.bfloat16).pin_memory()
-        host_out = torch.empty(layout.flat_len, dtype=torch.bfloat16).pin_memory()
-        host_in.copy_(flat_g)
-        e2e_steps = max(1, min(args.steps, args.e2e_steps))
-        for _ in range(2):
-            ctx.muon_step_flat_host(host_in, host_out, flat_o, L, W, G, M, O, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
-        torch.cuda.synchronize()
-        barrier(world)
-        e0.record(stream)
-        for _ in range(e2e_steps):
-            ctx.muon_step_flat_host(host_in, host_out, flat_o, L, W, G, M, O, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        barrier(world)
-        ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev) / e2e_steps
-        flat_bytes = layout.flat_len * 2
-        e2e = {"value": world * 1e3 / ms_e2e, "unit": UNIT, "h2d_bytes_per_step": flat_bytes, "d2h_bytes_per_step": flat_bytes,
-               "ms_per_step": ms_e2e, "steps": e2e_steps}
+        host_in = host_out = None
+        try:
+            host_in = torch.empty(layout.flat_len, dtype=torch.bfloat16).pin_memory()
+            host_out = torch.empty(layout.flat_len, dtype=torch.bfloat16).pin_memory()
+            pinned_ok = 1.0
+        except RuntimeError:
+            pinned_ok = 0.0
+        # every rank must take the same branch (the timed loop contains barriers)
+        if -max_over_ranks(-pinned_ok, world, dev) < 1.0:
+            e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                   "error": "could not pin the host flat buffers on every rank"}
+        else:
+            host_in.copy_(flat_g)
+            e2e_steps = max(1, min(args.steps, args.e2e_steps))
+            for _ in range(2):
+                ctx.muon_step_flat_host(host_in, host_out, flat_o, L, W, G, M, O, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
+            torch.cuda.synchronize()
+            barrier(world)
+            e0.record(stream)
+            for _ in range(e2e_steps):
+                ctx.muon_step_flat_host(host_in, host_out, flat_o, L, W, G, M, O, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            barrier(world)
+            ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev) / e2e_steps
+            flat_bytes = layout.flat_len * 2
+            e2e = {"value": world * 1e3 / ms_e2e, "unit": UNIT, "h2d_bytes_per_step": flat_bytes, "d2h_bytes_per_step": flat_bytes,
+                   "ms_per_step": ms_e2e, "steps": e2e_steps}
         del host_in, host_out
 
     if rank != 0:

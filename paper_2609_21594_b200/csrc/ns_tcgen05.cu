@@ -308,8 +308,9 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
 }
 
 // ------------------------------------------------------------------ host side
-int g_num_sms = 0;
-bool g_attr_set = false;
+// Per device ordinal: shared-memory attribute set and SM count looked up once.
+constexpr int kMaxDevices = 64;
+int g_num_sms[kMaxDevices] = {};
 
 }  // namespace
 
@@ -327,14 +328,14 @@ bool tc_supported(const GemmArgs& a) {
 
 int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st) {
   if (!ctx->tmap_encode) return MUON_ERR_CUDA;
-  if (!g_attr_set) {
+  if (ctx->device < 0 || ctx->device >= kMaxDevices) return MUON_ERR_UNSUPPORTED;
+  if (!g_num_sms[ctx->device]) {
     if (cudaFuncSetAttribute(ns_product_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
         cudaFuncSetAttribute(ns_product_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
       return MUON_ERR_CUDA;
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, ctx->device) != cudaSuccess) return MUON_ERR_CUDA;
-    g_num_sms = prop.multiProcessorCount;
-    g_attr_set = true;
+    g_num_sms[ctx->device] = prop.multiProcessorCount;
   }
   CUtensorMap map_p, map_q;
   // P: rows = m, cols = kdim
@@ -368,7 +369,7 @@ int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st) {
   t.alpha = a.alpha; t.beta = a.beta;
   t.status = ctx->d_status;
   const int64_t tiles = int64_t(t.tiles_per_mat) * t.batch;
-  const unsigned grid = unsigned(tiles < g_num_sms ? tiles : g_num_sms);
+  const unsigned grid = unsigned(tiles < g_num_sms[ctx->device] ? tiles : g_num_sms[ctx->device]);
   if (a.nn) ns_product_tc_kernel<true><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, map_d, map_c, t);
   else ns_product_tc_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, map_d, map_c, t);
   return cudaGetLastError() == cudaSuccess ? 1 : MUON_ERR_CUDA;

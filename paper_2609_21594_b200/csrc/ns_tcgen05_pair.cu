@@ -348,8 +348,9 @@ ns_product_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
   }
 }
 
-int g_num_sms = 0;
-bool g_attr_set = false;
+// Per device ordinal: shared-memory attribute set and SM count looked up once.
+constexpr int kMaxDevices = 64;
+int g_num_sms[kMaxDevices] = {};
 
 }  // namespace
 
@@ -360,14 +361,14 @@ bool tc_pair_supported(const GemmArgs& a) {
 
 int launch_gemm_tc_pair(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st) {
   if (!ctx->tmap_encode) return MUON_ERR_CUDA;
-  if (!g_attr_set) {
+  if (ctx->device < 0 || ctx->device >= kMaxDevices) return MUON_ERR_UNSUPPORTED;
+  if (!g_num_sms[ctx->device]) {
     if (cudaFuncSetAttribute(ns_product_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
         cudaFuncSetAttribute(ns_product_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
       return MUON_ERR_CUDA;
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, ctx->device) != cudaSuccess) return MUON_ERR_CUDA;
-    g_num_sms = prop.multiProcessorCount;
-    g_attr_set = true;
+    g_num_sms[ctx->device] = prop.multiProcessorCount;
   }
   CUtensorMap map_p, map_q, map_c, map_d;
   if (!encode_map(ctx->tmap_encode, &map_p, a.p, a.kdim, a.m, a.batch, a.ldp, a.stride_p, BM)) return MUON_ERR_CUDA;
@@ -393,7 +394,7 @@ int launch_gemm_tc_pair(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st) {
   t.alpha = a.alpha; t.beta = a.beta;
   t.status = ctx->d_status;
   const int64_t tiles = int64_t(t.tiles_per_mat) * t.batch;
-  const int64_t pairs = g_num_sms / 2;
+  const int64_t pairs = g_num_sms[ctx->device] / 2;
   const unsigned grid = unsigned(2 * (tiles < pairs ? tiles : pairs));
   if (a.nn) ns_product_pair_kernel<true><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, map_d, map_c, t);
   else ns_product_pair_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, map_d, map_c, t);

@@ -294,3 +294,53 @@ def test_step_argument_errors_launch_nothing():
     ctx.muon_step_batched([None], [None], [None], [(0, 7)], 0.02, 0.95, 0.01, 5, QUINTIC)
     assert ctx.muon_launch_count() == before
     ctx.close()
+
+
+def test_step_out_and_flat_host_path_match_the_plain_step():
+    """muon_step_batched_out emits exactly the O the update applied; muon_step_flat_host (host flat shards in,
+    host flat updates out) reproduces the device-resident sequence bit for bit."""
+    from paper_2609_21594_b200 import binding as mb
+
+    shapes = wl.shapes_tiny() + [(130, 200), (200, 130)]
+    lay = wl.layout_per_param(shapes, 8)
+    segs = [(s.matrix, s.elem_begin, s.elem_count, s.flat_offset) for s in lay.segments]
+    ctx = _ctx(mb, "bf16", "tensor", "bf16")
+    ctx.ensure_workspace(shapes)
+    L = mb.Layout(ctx, lay, 2)
+    g_bits = [wl.to_bf16_bits(wl.grad_np("flat", 0, i, s)) for i, s in enumerate(shapes)]
+    flat_np = orc.scatter(np.zeros(lay.flat_len, dtype=np.uint16), shapes, segs, g_bits)
+    W0 = [dev_f32(wl.param_np("flat", i, s)) for i, s in enumerate(shapes)]
+    # (a) device-resident reference sequence
+    Wa = [w.clone() for w in W0]
+    Ma = [torch.zeros(s, dtype=torch.float32, device="cuda") for s in shapes]
+    Ga = [torch.from_numpy(b.view(np.int16)).cuda().view(torch.bfloat16).reshape(s) for b, s in zip(g_bits, shapes)]
+    Oa = [torch.full(s, float("nan"), dtype=torch.bfloat16, device="cuda") for s in shapes]
+    ctx.muon_step_batched_out(Wa, Ga, Ma, Oa, shapes, 0.02, 0.95, 0.01, 5, QUINTIC)
+    Wp = [w.clone() for w in W0]
+    Mp = [torch.zeros_like(m) for m in Ma]
+    ctx.muon_step_batched(Wp, Ga, Mp, shapes, 0.02, 0.95, 0.01, 5, QUINTIC)
+    torch.cuda.synchronize()
+    for i, s in enumerate(shapes):
+        assert torch.equal(Wa[i], Wp[i]) and torch.equal(Ma[i], Mp[i])
+        O_from_W = (host_f64(W0[i]) * (1 - 0.02 * 0.01) - host_f64(Wa[i])) / (0.02 * orc.update_scale(*s))
+        assert rel(host_f64(Oa[i]), O_from_W) < 2e-4            # the emitted O is the O that was applied
+        ref = orc.muon_step(host_f64(W0[i]), wl.bf16_bits_to_f32(g_bits[i]).astype(np.float64).reshape(s), np.zeros(s),
+                            0.02, 0.95, 0.01, 5, QUINTIC, 1e-7, True, "bf16")[2]
+        assert rel(host_f64(Oa[i]), ref) <= TOL_BF16
+    # (b) the same step from host flat buffers
+    host_in = torch.from_numpy(flat_np.view(np.int16)).view(torch.bfloat16).pin_memory()
+    host_out = torch.zeros(lay.flat_len, dtype=torch.bfloat16).pin_memory()
+    dev_flat = torch.zeros(lay.flat_len, dtype=torch.bfloat16, device="cuda")
+    Wb = [w.clone() for w in W0]
+    Mb = [torch.zeros_like(m) for m in Ma]
+    Gb = [torch.zeros(s, dtype=torch.bfloat16, device="cuda") for s in shapes]
+    Ob = [torch.zeros(s, dtype=torch.bfloat16, device="cuda") for s in shapes]
+    ctx.muon_step_flat_host(host_in, host_out, dev_flat, L, Wb, Gb, Mb, Ob, 0.02, 0.95, 0.01, 5, QUINTIC)
+    torch.cuda.synchronize()
+    for i in range(len(shapes)):
+        assert torch.equal(Wb[i], Wa[i]) and torch.equal(Mb[i], Ma[i]) and torch.equal(Ob[i].view(torch.int16), Oa[i].view(torch.int16))
+    back = orc.materialize(host_out.view(torch.int16).numpy().view(np.uint16), shapes, segs)
+    for i in range(len(shapes)):
+        assert np.array_equal(back[i], Oa[i].view(torch.int16).cpu().numpy().view(np.uint16))
+    L.close()
+    ctx.close()
