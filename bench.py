@@ -289,12 +289,12 @@ def run_ours(args, world, rank, local):
             host_in.copy_(flat_g)
             e2e_steps = max(1, min(args.steps, args.e2e_steps))
             for _ in range(2):
-                ctx.muon_step_flat_host(host_in, host_out, flat_o, L, W, G, M, O, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
+                ctx.muon_step_flat_host(host_in, host_out, L, W, G, M, O, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
             torch.cuda.synchronize()
             barrier(world)
             e0.record(stream)
             for _ in range(e2e_steps):
-                ctx.muon_step_flat_host(host_in, host_out, flat_o, L, W, G, M, O, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
+                ctx.muon_step_flat_host(host_in, host_out, L, W, G, M, O, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
             e1.record(stream)
             torch.cuda.synchronize()
             barrier(world)

@@ -175,15 +175,20 @@ int muon_step_batched_out(muon_ctx_t* ctx, void* const* params, const void* cons
                           void* const* updates, const muon_shape_t* shapes, int32_t count, float lr, float mu,
                           float wd, int32_t ns_steps, const float* coeffs, void* stream);
 
-/* muon_step_flat_host: the whole path on HOST flat buffers, for end-to-end use and timing:
- * copy host_flat_grads (host; pinned memory makes the copies asynchronous) to dev_flat, materialise it
- * into grads[], run muon_step_batched_out on the layout's shapes, scatter updates[] into dev_flat and
- * copy dev_flat to host_flat_updates (host).  dev_flat: device staging buffer of
- * num_shards*shard_len elements; grads/updates: host arrays of device pointers to whole-matrix
- * scratch the caller owns.  The layout's element size must equal both the gradient and the NS
- * element size (bf16/bf16 or fp32/fp32).  Everything is enqueued on `stream` in order; the host
- * buffers may be touched again once the stream has been synchronised. */
-int muon_step_flat_host(muon_ctx_t* ctx, const void* host_flat_grads, void* host_flat_updates, void* dev_flat,
+/* muon_step_flat_host: the whole path on HOST flat buffers, for end-to-end use and timing.
+ * host_flat_grads / host_flat_updates are host buffers of num_shards*shard_len elements in the
+ * layout's format (pinned memory makes the copies asynchronous).  Per batch of matrices (the chunks of
+ * muon_plan_describe) the gradient segments are copied by DMA straight into grads[] -- the copy engine
+ * performs the gather of Section 6.2 step 1 -- the batch is updated as in muon_step_batched_out, and
+ * its update segments are copied from updates[] straight into host_flat_updates (the pack of step 3).
+ * Inbound copies of later batches and outbound copies of earlier ones overlap the Newton-Schulz work
+ * on two internal copy streams; padding of host_flat_updates is never written.
+ *   grads, updates : host arrays of device pointers to whole-matrix scratch the caller owns
+ * The layout's element size must equal both the gradient and the NS element size (bf16/bf16 or
+ * fp32/fp32).  Ordering: everything starts after prior work on `stream`, and later work on `stream`
+ * waits for the last outbound copy; the host buffers may be touched again once `stream` has been
+ * synchronised.  The two copy streams are created on the first call (which therefore allocates). */
+int muon_step_flat_host(muon_ctx_t* ctx, const void* host_flat_grads, void* host_flat_updates,
                         const muon_layout_t* layout, void* const* params, void* const* grads, void* const* momenta,
                         void* const* updates, float lr, float mu, float wd, int32_t ns_steps, const float* coeffs,
                         void* stream);

@@ -68,7 +68,7 @@ _sig = {
                                     C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
     "muon_step_batched_out": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(Shape),
                                         C.c_int32, C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
-    "muon_step_flat_host": (C.c_int, [_vp, _vp, _vp, _vp, _vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp),
+    "muon_step_flat_host": (C.c_int, [_vp, _vp, _vp, _vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp),
                                       C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
     "muon_orthogonalize_batched": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(Shape), C.c_int32,
                                              C.c_int32, C.POINTER(C.c_float), C.c_uint32, _vp]),
@@ -252,12 +252,12 @@ class Context:
                                          None if updates is None else _ptrs(updates), _shapes(shapes), len(shapes),
                                          lr, mu, wd, ns_steps, co, _stream(stream)), "muon_step_batched_out")
 
-    def muon_step_flat_host(self, host_flat_grads, host_flat_updates, dev_flat, layout: Layout, params, grads, momenta,
+    def muon_step_flat_host(self, host_flat_grads, host_flat_updates, layout: Layout, params, grads, momenta,
                             updates, lr, mu, wd, ns_steps, coeffs, stream=None) -> None:
-        """host_flat_*: CPU tensors (pinned for asynchronous copies); dev_flat: CUDA tensor."""
+        """host_flat_*: CPU tensors (pinned for asynchronous copies)."""
         co = (C.c_float * len(coeffs))(*[float(c) for c in coeffs])
         _check(lib.muon_step_flat_host(self.handle, host_flat_grads.data_ptr(), host_flat_updates.data_ptr(),
-                                       dev_flat.data_ptr(), layout.handle, _ptrs(params), _ptrs(grads), _ptrs(momenta),
+                                       layout.handle, _ptrs(params), _ptrs(grads), _ptrs(momenta),
                                        _ptrs(updates), lr, mu, wd, ns_steps, co, _stream(stream)), "muon_step_flat_host")
 
     def muon_orthogonalize_batched(self, inputs, outputs, shapes, ns_steps, coeffs, flags=0, stream=None) -> None:

@@ -205,8 +205,31 @@ int run_chunk(muon_ctx* ctx, const Chunk& ch, const MatDesc* d_descs, const Chun
   return MUON_OK;
 }
 
+// Host-buffer pipeline: per chunk, gradients arrive by DMA straight into the whole-matrix buffers (the
+// copy engine performs the gather) and updates leave the same way, on two copy streams that run ahead
+// of / behind the compute stream.
+struct HostPipe {
+  const char* host_in;
+  char* host_out;
+  const muon_layout* layout;
+};
+
+cudaEvent_t next_sync_event(muon_ctx* ctx) {
+  if (ctx->sync_events.size() < 1024) {
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    ctx->sync_events.push_back(e);
+    return e;
+  }
+  // a recorded event may be re-recorded: earlier waits captured its earlier state
+  cudaEvent_t e = ctx->sync_events[ctx->next_sync_event];
+  ctx->next_sync_event = (ctx->next_sync_event + 1) % ctx->sync_events.size();
+  return e;
+}
+
 int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const* m, void* const* o,
-                const muon_shape_t* shapes, int32_t count, const ChunkRun& r, cudaStream_t st) {
+                const muon_shape_t* shapes, int32_t count, const ChunkRun& r, cudaStream_t st,
+                const HostPipe* pipe = nullptr) {
   int status;
   Plan* plan = get_plan(ctx, shapes, count, &status);
   if (!plan) return status;
@@ -233,10 +256,48 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
   void* d_descs = nullptr;
   status = upload(ctx, descs.data(), descs.size() * sizeof(MatDesc), st, &d_descs);
   if (status != MUON_OK) return status;
-  for (const Chunk& ch : plan->chunks) {
+  if (!pipe) {
+    for (const Chunk& ch : plan->chunks) {
+      status = run_chunk(ctx, ch, static_cast<const MatDesc*>(d_descs), r, st);
+      if (status != MUON_OK) return status;
+    }
+    return MUON_OK;
+  }
+  // ---- pipelined host path
+  const size_t es = size_t(pipe->layout->desc.elem_size);
+  cudaEvent_t ev = next_sync_event(ctx);
+  if (!ev || cudaEventRecord(ev, st) != cudaSuccess) return MUON_ERR_CUDA;
+  if (cudaStreamWaitEvent(ctx->h2d_stream, ev, 0) != cudaSuccess || cudaStreamWaitEvent(ctx->d2h_stream, ev, 0) != cudaSuccess)
+    return MUON_ERR_CUDA;
+  std::vector<cudaEvent_t> arrived(plan->chunks.size());
+  for (size_t c = 0; c < plan->chunks.size(); ++c) {            // all inbound copies are queued up front, in chunk order
+    for (int32_t i : plan->chunks[c].mats)
+      for (const muon_segment_t& sg : pipe->layout->segs_of[size_t(i)])
+        if (cudaMemcpyAsync(static_cast<char*>(const_cast<void*>(g[i])) + size_t(sg.elem_begin) * es,
+                            pipe->host_in + size_t(sg.flat_offset) * es, size_t(sg.elem_count) * es, cudaMemcpyHostToDevice,
+                            ctx->h2d_stream) != cudaSuccess)
+          return MUON_ERR_CUDA;
+    arrived[c] = next_sync_event(ctx);
+    if (!arrived[c] || cudaEventRecord(arrived[c], ctx->h2d_stream) != cudaSuccess) return MUON_ERR_CUDA;
+  }
+  for (size_t c = 0; c < plan->chunks.size(); ++c) {
+    const Chunk& ch = plan->chunks[c];
+    if (cudaStreamWaitEvent(st, arrived[c], 0) != cudaSuccess) return MUON_ERR_CUDA;
     status = run_chunk(ctx, ch, static_cast<const MatDesc*>(d_descs), r, st);
     if (status != MUON_OK) return status;
+    cudaEvent_t done = next_sync_event(ctx);
+    if (!done || cudaEventRecord(done, st) != cudaSuccess || cudaStreamWaitEvent(ctx->d2h_stream, done, 0) != cudaSuccess)
+      return MUON_ERR_CUDA;
+    for (int32_t i : ch.mats)
+      for (const muon_segment_t& sg : pipe->layout->segs_of[size_t(i)])
+        if (cudaMemcpyAsync(pipe->host_out + size_t(sg.flat_offset) * es,
+                            static_cast<const char*>(o[i]) + size_t(sg.elem_begin) * es, size_t(sg.elem_count) * es,
+                            cudaMemcpyDeviceToHost, ctx->d2h_stream) != cudaSuccess)
+          return MUON_ERR_CUDA;
   }
+  cudaEvent_t fin = next_sync_event(ctx);
+  if (!fin || cudaEventRecord(fin, ctx->d2h_stream) != cudaSuccess || cudaStreamWaitEvent(st, fin, 0) != cudaSuccess)
+    return MUON_ERR_CUDA;
   return MUON_OK;
 }
 
@@ -300,6 +361,9 @@ void muon_destroy(muon_ctx_t* ctx) {
     cudaEventDestroy(p.b);
   }
   for (cudaEvent_t e : ctx->event_pool) cudaEventDestroy(e);
+  for (cudaEvent_t e : ctx->sync_events) cudaEventDestroy(e);
+  if (ctx->h2d_stream) cudaStreamDestroy(ctx->h2d_stream);
+  if (ctx->d2h_stream) cudaStreamDestroy(ctx->d2h_stream);
   if (ctx->d_status) cudaFree(ctx->d_status);
   delete ctx;
 }
@@ -366,6 +430,9 @@ int muon_layout_create(muon_ctx_t* ctx, const muon_layout_desc_t* desc, muon_lay
   L->desc.segments = nullptr;
   L->num_items = int64_t(items.size());
   L->device = ctx->device;
+  L->segs_of.resize(size_t(desc->num_matrices));
+  for (int64_t k = 0; k < desc->num_segments; ++k)
+    if (desc->segments[k].elem_count > 0) L->segs_of[size_t(desc->segments[k].matrix)].push_back(desc->segments[k]);
   if (!items.empty()) {
     if (cudaMalloc(&L->d_items, items.size() * sizeof(CopyItem)) != cudaSuccess ||
         cudaMemcpy(L->d_items, items.data(), items.size() * sizeof(CopyItem), cudaMemcpyHostToDevice) != cudaSuccess) {
@@ -448,29 +515,26 @@ int muon_step_batched(muon_ctx_t* ctx, void* const* params, const void* const* g
   return muon_step_batched_out(ctx, params, grads, momenta, nullptr, shapes, count, lr, mu, wd, ns_steps, coeffs, stream);
 }
 
-int muon_step_flat_host(muon_ctx_t* ctx, const void* host_flat_grads, void* host_flat_updates, void* dev_flat,
+int muon_step_flat_host(muon_ctx_t* ctx, const void* host_flat_grads, void* host_flat_updates,
                         const muon_layout_t* layout, void* const* params, void* const* grads, void* const* momenta,
                         void* const* updates, float lr, float mu, float wd, int32_t ns_steps, const float* coeffs,
                         void* stream) {
-  if (!ctx || !layout || !host_flat_grads || !host_flat_updates || !dev_flat || !updates) return MUON_ERR_INVALID_ARG;
+  if (!ctx || !layout || !host_flat_grads || !host_flat_updates || !updates) return MUON_ERR_INVALID_ARG;
   const int want = ctx->opt.grad_dtype == MUON_DTYPE_BF16 ? 2 : 4;
   const int ns_es = ctx->opt.ns_precision == MUON_NS_BF16 ? 2 : 4;
-  if (layout->desc.elem_size != want || ns_es != want) return MUON_ERR_INVALID_ARG;   // one flat buffer carries both ways
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const size_t bytes = size_t(layout->desc.num_shards) * size_t(layout->desc.shard_len) * size_t(want);
+  if (layout->desc.elem_size != want || ns_es != want) return MUON_ERR_INVALID_ARG;   // one flat format carries both ways
   const int32_t count = layout->desc.num_matrices;
   int rc = check_common(ctx, layout->shapes.data(), count, ns_steps, coeffs);
   if (rc != MUON_OK) return rc;
-  if (cudaMemcpyAsync(dev_flat, host_flat_grads, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return MUON_ERR_CUDA;
-  rc = muon_materialize(ctx, dev_flat, layout, grads, stream);
-  if (rc != MUON_OK) return rc;
-  rc = muon_step_batched_out(ctx, params, const_cast<const void* const*>(grads), momenta, updates, layout->shapes.data(),
-                             count, lr, mu, wd, ns_steps, coeffs, stream);
-  if (rc != MUON_OK) return rc;
-  rc = muon_scatter(ctx, dev_flat, layout, const_cast<const void* const*>(updates), stream);
-  if (rc != MUON_OK) return rc;
-  if (cudaMemcpyAsync(host_flat_updates, dev_flat, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MUON_ERR_CUDA;
-  return MUON_OK;
+  if (count == 0) return MUON_OK;
+  if (!params || !grads || !momenta || layout->device != ctx->device) return MUON_ERR_INVALID_ARG;
+  if (!std::isfinite(lr) || !std::isfinite(mu) || !std::isfinite(wd)) return MUON_ERR_INVALID_ARG;
+  if (!ctx->h2d_stream && cudaStreamCreateWithFlags(&ctx->h2d_stream, cudaStreamNonBlocking) != cudaSuccess) return MUON_ERR_CUDA;
+  if (!ctx->d2h_stream && cudaStreamCreateWithFlags(&ctx->d2h_stream, cudaStreamNonBlocking) != cudaSuccess) return MUON_ERR_CUDA;
+  HostPipe pipe{static_cast<const char*>(host_flat_grads), static_cast<char*>(host_flat_updates), layout};
+  ChunkRun r{1, 1, lr, mu, wd, ns_steps, coeffs};
+  return run_batched(ctx, params, const_cast<const void* const*>(grads), momenta, updates, layout->shapes.data(), count, r,
+                     static_cast<cudaStream_t>(stream), &pipe);
 }
 
 int muon_orthogonalize_batched(muon_ctx_t* ctx, const void* const* in, void* const* out, const muon_shape_t* shapes,

@@ -83,6 +83,7 @@ struct muon_layout {
   muon::CopyItem* d_items = nullptr;
   int64_t num_items = 0;
   int device = 0;
+  std::vector<std::vector<muon_segment_t>> segs_of;   // host copy of the segment table, grouped by matrix
 };
 
 struct muon_ctx {
@@ -101,6 +102,9 @@ struct muon_ctx {
   int64_t phase_launches[MUON_NUM_PHASES] = {0, 0, 0, 0, 0};
   int64_t launches = 0;
   void* tmap_encode = nullptr;                     // cuTensorMapEncodeTiled, resolved at run time
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;   // copy streams of the host-buffer path (created on first use)
+  std::vector<cudaEvent_t> sync_events;            // untimed events that order the copy streams against the caller's stream
+  size_t next_sync_event = 0;
 };
 
 namespace muon {

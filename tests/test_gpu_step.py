@@ -330,12 +330,11 @@ def test_step_out_and_flat_host_path_match_the_plain_step():
     # (b) the same step from host flat buffers
     host_in = torch.from_numpy(flat_np.view(np.int16)).view(torch.bfloat16).pin_memory()
     host_out = torch.zeros(lay.flat_len, dtype=torch.bfloat16).pin_memory()
-    dev_flat = torch.zeros(lay.flat_len, dtype=torch.bfloat16, device="cuda")
     Wb = [w.clone() for w in W0]
     Mb = [torch.zeros_like(m) for m in Ma]
     Gb = [torch.zeros(s, dtype=torch.bfloat16, device="cuda") for s in shapes]
     Ob = [torch.zeros(s, dtype=torch.bfloat16, device="cuda") for s in shapes]
-    ctx.muon_step_flat_host(host_in, host_out, dev_flat, L, Wb, Gb, Mb, Ob, 0.02, 0.95, 0.01, 5, QUINTIC)
+    ctx.muon_step_flat_host(host_in, host_out, L, Wb, Gb, Mb, Ob, 0.02, 0.95, 0.01, 5, QUINTIC)
     torch.cuda.synchronize()
     for i in range(len(shapes)):
         assert torch.equal(Wb[i], Wa[i]) and torch.equal(Mb[i], Ma[i]) and torch.equal(Ob[i].view(torch.int16), Oa[i].view(torch.int16))
