@@ -66,6 +66,12 @@ typedef struct muon_layout muon_layout_t;
 /* Shape of one dense row-major matrix (Section 2.3: W in R^{m x n}). */
 typedef struct { int32_t rows, cols; } muon_shape_t;
 
+/* A logical matrix inside a larger physical parameter (Section 6.3, "the matrix as Muon sees it":
+ * one physical parameter can hold several logical matrices -- the heads of a fused QKV projection, the
+ * gate and up halves of an MoE FC1 weight, the factors of an MLA projection, the E planes of an
+ * [E, M, N] expert tensor).  rows x cols elements, row r starting ld elements after row r-1. */
+typedef struct { int32_t rows, cols; int64_t ld; } muon_view_t;
+
 /* One contiguous piece of a matrix inside the flat buffer: elements
  * [elem_begin, elem_begin+elem_count) of the row-major linearisation of matrix
  * `matrix` live at flat[flat_offset, flat_offset+elem_count).  Units: elements. */
@@ -174,6 +180,17 @@ int muon_step_batched(muon_ctx_t* ctx, void* const* params, const void* const* g
 int muon_step_batched_out(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
                           void* const* updates, const muon_shape_t* shapes, int32_t count, float lr, float mu,
                           float wd, int32_t ns_steps, const float* coeffs, void* stream);
+
+/* muon_step_batched_views: muon_step_batched_out on strided views, so that logical matrices are
+ * updated in place inside their physical parameters without split/concatenate copies and without a
+ * restore pass (the zero-copy view and the restore mapping of the model adapter, Section 6.3).
+ * params[i], grads[i], momenta[i] and, when given, updates[i] point at element (0,0) of view i inside
+ * tensors that share the physical layout; all use views[i].ld as row stride (ld >= cols).  Pointers must
+ * be 16-byte aligned; the vectorised path also needs ld to be a multiple of 4 elements (other strides
+ * run element-wise).  Elements outside the views are never touched.  Views of one call must not overlap. */
+int muon_step_batched_views(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
+                            void* const* updates, const muon_view_t* views, int32_t count, float lr, float mu,
+                            float wd, int32_t ns_steps, const float* coeffs, void* stream);
 
 /* muon_step_flat_host: the whole path on HOST flat buffers, for end-to-end use and timing.
  * host_flat_grads / host_flat_updates are host buffers of num_shards*shard_len elements in the

@@ -34,6 +34,10 @@ class Shape(C.Structure):
     _fields_ = [("rows", C.c_int32), ("cols", C.c_int32)]
 
 
+class View(C.Structure):
+    _fields_ = [("rows", C.c_int32), ("cols", C.c_int32), ("ld", C.c_int64)]
+
+
 class Segment(C.Structure):
     _fields_ = [("matrix", C.c_int32), ("reserved", C.c_int32), ("elem_begin", C.c_int64),
                 ("elem_count", C.c_int64), ("flat_offset", C.c_int64)]
@@ -68,6 +72,8 @@ _sig = {
                                     C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
     "muon_step_batched_out": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(Shape),
                                         C.c_int32, C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
+    "muon_step_batched_views": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(View),
+                                          C.c_int32, C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
     "muon_step_flat_host": (C.c_int, [_vp, _vp, _vp, _vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp),
                                       C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
     "muon_orthogonalize_batched": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(Shape), C.c_int32,
@@ -174,6 +180,39 @@ def muon_orthogonalize_static(inp, out, rows, cols, ns_precision, ns_steps, coef
            "muon_orthogonalize_static")
 
 
+# ---- logical-matrix views: pure address arithmetic on tensors that share one physical layout
+def views_of_rows(tensor, row_counts):
+    """Row blocks of a 2-D tensor (fused QKV projections, gate/up halves stacked along rows).
+    Returns [(element offset, (rows, cols, ld))]."""
+    assert tensor.dim() == 2 and tensor.stride(1) == 1 and sum(row_counts) == tensor.shape[0]
+    ld, out, r0 = tensor.stride(0), [], 0
+    for n in row_counts:
+        out.append((r0 * ld, (n, tensor.shape[1], ld)))
+        r0 += n
+    return out
+
+
+def views_of_cols(tensor, col_counts):
+    """Column blocks of a 2-D tensor (factors packed side by side, e.g. the two parts of an MLA projection)."""
+    assert tensor.dim() == 2 and tensor.stride(1) == 1 and sum(col_counts) == tensor.shape[1]
+    ld, out, c0 = tensor.stride(0), [], 0
+    for n in col_counts:
+        out.append((c0, (tensor.shape[0], n, ld)))
+        c0 += n
+    return out
+
+
+def views_of_planes(tensor):
+    """The E matrix planes of an [E, M, N] tensor: E independent M x N matrices, never one E x MN matrix."""
+    assert tensor.dim() == 3 and tensor.stride(2) == 1
+    return [(e * tensor.stride(0), (tensor.shape[1], tensor.shape[2], tensor.stride(1))) for e in range(tensor.shape[0])]
+
+
+def view_addresses(tensor, views):
+    """Device addresses of element (0,0) of each view of `tensor`."""
+    return [tensor.data_ptr() + off * tensor.element_size() for off, _ in views]
+
+
 class Layout:
     """Owner of a muon_layout_t handle."""
 
@@ -251,6 +290,17 @@ class Context:
         _check(lib.muon_step_batched_out(self.handle, _ptrs(params), _ptrs(grads), _ptrs(momenta),
                                          None if updates is None else _ptrs(updates), _shapes(shapes), len(shapes),
                                          lr, mu, wd, ns_steps, co, _stream(stream)), "muon_step_batched_out")
+
+    def muon_step_batched_views(self, params, grads, momenta, updates, views, lr, mu, wd, ns_steps, coeffs, stream=None) -> None:
+        """params/grads/momenta/updates: lists of device addresses (ints) of element (0,0) of each view;
+        views: list of (rows, cols, ld)."""
+        co = (C.c_float * len(coeffs))(*[float(c) for c in coeffs])
+        va = (View * max(1, len(views)))()
+        for i, (r, c, ld) in enumerate(views):
+            va[i].rows, va[i].cols, va[i].ld = int(r), int(c), int(ld)
+        _check(lib.muon_step_batched_views(self.handle, _ptrs(params), _ptrs(grads), _ptrs(momenta),
+                                           None if updates is None else _ptrs(updates), va, len(views), lr, mu, wd, ns_steps,
+                                           co, _stream(stream)), "muon_step_batched_views")
 
     def muon_step_flat_host(self, host_flat_grads, host_flat_updates, layout: Layout, params, grads, momenta,
                             updates, lr, mu, wd, ns_steps, coeffs, stream=None) -> None:

@@ -229,7 +229,7 @@ cudaEvent_t next_sync_event(muon_ctx* ctx) {
 
 int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const* m, void* const* o,
                 const muon_shape_t* shapes, int32_t count, const ChunkRun& r, cudaStream_t st,
-                const HostPipe* pipe = nullptr) {
+                const HostPipe* pipe = nullptr, const int64_t* lds = nullptr) {
   int status;
   Plan* plan = get_plan(ctx, shapes, count, &status);
   if (!plan) return status;
@@ -249,6 +249,8 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
         return MUON_ERR_INVALID_ARG;
       d.rows = shapes[i].rows;
       d.cols = shapes[i].cols;
+      d.ld = lds ? lds[i] : int64_t(d.cols);
+      if (d.ld < d.cols) return MUON_ERR_INVALID_ARG;
       d.transposed = d.rows > d.cols ? 1 : 0;
       d.scale = float(0.2 * std::sqrt(double(std::max(d.rows, d.cols))));
     }
@@ -509,6 +511,27 @@ int muon_step_batched_out(muon_ctx_t* ctx, void* const* params, const void* cons
   return run_batched(ctx, params, grads, momenta, updates, shapes, count, r, static_cast<cudaStream_t>(stream));
 }
 
+int muon_step_batched_views(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
+                            void* const* updates, const muon_view_t* views, int32_t count, float lr, float mu, float wd,
+                            int32_t ns_steps, const float* coeffs, void* stream) {
+  if (!ctx || count < 0 || (count > 0 && !views)) return MUON_ERR_INVALID_ARG;
+  std::vector<muon_shape_t> shapes(static_cast<size_t>(count));
+  std::vector<int64_t> lds(static_cast<size_t>(count));
+  for (int32_t i = 0; i < count; ++i) {
+    shapes[size_t(i)].rows = views[i].rows;
+    shapes[size_t(i)].cols = views[i].cols;
+    lds[size_t(i)] = views[i].ld;
+  }
+  int st = check_common(ctx, shapes.data(), count, ns_steps, coeffs);
+  if (st != MUON_OK) return st;
+  if (count == 0) return MUON_OK;
+  if (!params || !grads || !momenta) return MUON_ERR_INVALID_ARG;
+  if (!std::isfinite(lr) || !std::isfinite(mu) || !std::isfinite(wd)) return MUON_ERR_INVALID_ARG;
+  ChunkRun r{1, 1, lr, mu, wd, ns_steps, coeffs};
+  return run_batched(ctx, params, grads, momenta, updates, shapes.data(), count, r, static_cast<cudaStream_t>(stream), nullptr,
+                     lds.data());
+}
+
 int muon_step_batched(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
                       const muon_shape_t* shapes, int32_t count, float lr, float mu, float wd, int32_t ns_steps,
                       const float* coeffs, void* stream) {
@@ -731,6 +754,7 @@ extern "C" int muon_orthogonalize_static(const void* in, void* out, int32_t rows
   d.g = in;
   d.rows = rows;
   d.cols = cols;
+  d.ld = cols;
   d.transposed = rows > cols ? 1 : 0;
   d.scale = 0.f;
   MatDesc* d_desc = reinterpret_cast<MatDesc*>(sb + 256);

@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
   float* __restrict__ M = static_cast<float*>(d.m);
   XT* __restrict__ X = static_cast<XT*>(a.x) + size_t(mat) * a.s * a.ldx;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  const bool vec = (d.cols & 3) == 0;
+  const bool vec = ((d.cols | int(d.ld)) & 3) == 0;
   float sum = 0.f;
 #pragma unroll
   for (int pass = 0; pass < 4; ++pass) {
@@ -66,7 +66,7 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
     const int r = r0 + rr, c = c0 + cc;
     float u[4] = {0.f, 0.f, 0.f, 0.f};
     if (r < d.rows && c < d.cols) {
-      const size_t off = size_t(r) * d.cols + c;
+      const size_t off = size_t(r) * size_t(d.ld) + c;
       float g[4], m[4] = {0.f, 0.f, 0.f, 0.f};
       const int nv = min(4, d.cols - c);
       if (vec) {
@@ -182,7 +182,7 @@ __global__ void __launch_bounds__(256) apply_kernel(ApplyArgs a) {
   const XT* __restrict__ X = static_cast<const XT*>(a.x) + size_t(mat) * a.s * a.ldx;
   float* __restrict__ W = static_cast<float*>(d.w);
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  const bool vec = (d.cols & 3) == 0;
+  const bool vec = ((d.cols | int(d.ld)) & 3) == 0;
   const int cc = tx * 4, c = c0 + cc;
   const int nv = min(4, d.cols - c);
   float w[4][4];
@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(256) apply_kernel(ApplyArgs a) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) w[pass][i] = 0.f;
       if (r < d.rows && nv > 0) {
-        const size_t off = size_t(r) * d.cols + c;
+        const size_t off = size_t(r) * size_t(d.ld) + c;
         if (vec) {
           const float4 wv = __ldcs(reinterpret_cast<const float4*>(W + off));
           w[pass][0] = wv.x; w[pass][1] = wv.y; w[pass][2] = wv.z; w[pass][3] = wv.w;
@@ -256,7 +256,7 @@ __global__ void __launch_bounds__(256) apply_kernel(ApplyArgs a) {
   for (int pass = 0; pass < 4; ++pass) {
     const int r = r0 + ty + pass * 16;
     if (r < d.rows && nv > 0) {
-      const size_t off = size_t(r) * d.cols + c;
+      const size_t off = size_t(r) * size_t(d.ld) + c;
       if (UPD) {
         float4 o;
         o.x = w[pass][0] * decay - step * XConv<XT>::to(xv[pass][0]);

@@ -22,6 +22,7 @@ struct alignas(16) MatDesc {
   const void* g;    // step: gradients                   | orthogonalize: input matrix
   void* m;          // step: fp32 momenta (in/out)       | orthogonalize: unused
   void* o;          // step: optional copy of the NS output O in the NS element type (may be null)
+  int64_t ld;           // elements between consecutive rows of w, g, m and o (== cols for dense matrices)
   int32_t rows, cols;
   int32_t transposed;   // rows > cols: X holds the transpose
   float scale;          // 0.2*sqrt(max(rows, cols))

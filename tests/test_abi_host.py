@@ -32,6 +32,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_sizes_match_the_header():
     assert C.sizeof(mb.Shape) == 8
+    assert C.sizeof(mb.View) == 16
     assert C.sizeof(mb.Segment) == 32
     assert C.sizeof(mb.LayoutDesc) == 48
     assert C.sizeof(mb.Options) == 32

@@ -343,3 +343,44 @@ def test_step_out_and_flat_host_path_match_the_plain_step():
         assert np.array_equal(back[i], Oa[i].view(torch.int16).cpu().numpy().view(np.uint16))
     L.close()
     ctx.close()
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_per_step_coefficient_sets_on_the_bf16_engines(engine):
+    """A different (a_k, b_k, c_k) at every step -- the form the paper's default 'asymmetric five-step' variant
+    takes (its values are not printed, so arbitrary per-step triples stand in)."""
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "bf16", engine, coeffs_per_step=1)
+    co = [4.0, -6.0, 2.5, 3.8, -5.5, 2.2, 3.4445, -4.7750, 2.0315, 2.9, -3.6, 1.6, 2.3, -2.0, 0.7]
+    shapes = [(256, 384), (384, 256), (130, 200)]
+    mats = [wl.grad_np("perstep16", 0, i, s) for i, s in enumerate(shapes)]
+    outs, vals = _ortho(mb, ctx, mats, steps=5, coeffs=co)
+    for o, v in zip(outs, vals):
+        assert rel(o, orc.newton_schulz(v, 5, co, 1e-7, "bf16")) <= TOL_BF16
+    ctx.close()
+
+
+def test_plain_momentum_rule_and_eps_option():
+    """nesterov = 0 (u = M') and a non-default epsilon are options of the context, not compile-time choices."""
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "fp32", "tensor", "fp32", nesterov=0, eps=5e-2)
+    shapes = [(96, 160), (160, 96)]
+    ctx.ensure_workspace(shapes)
+    Wn = [wl.param_np("plain", i, s) for i, s in enumerate(shapes)]
+    Mn = [wl.grad_np("plain", 7, i, s) for i, s in enumerate(shapes)]
+    Gn = [wl.grad_np("plain", 0, i, s) for i, s in enumerate(shapes)]
+    W, M, G = [dev_f32(x) for x in Wn], [dev_f32(x) for x in Mn], [dev_f32(x) for x in Gn]
+    ctx.muon_step_batched(W, G, M, shapes, 0.02, 0.9, 0.05, 5, QUINTIC)
+    torch.cuda.synchronize()
+    for i in range(len(shapes)):
+        Wr, Mr, _ = orc.muon_step(Wn[i].astype(np.float64), Gn[i].astype(np.float64), Mn[i].astype(np.float64), 0.02, 0.9, 0.05, 5,
+                                  QUINTIC, 5e-2, False, "fp64")
+        assert rel(host_f64(M[i]), Mr) <= 1e-6
+        assert rel(host_f64(W[i]) - Wn[i], Wr - Wn[i]) <= TOL_FP32
+        # eps = 5e-2 is comparable to ||u||_F here, so a wrong epsilon or a Nesterov look-ahead would be far outside 1e-4
+        Wbad = orc.muon_step(Wn[i].astype(np.float64), Gn[i].astype(np.float64), Mn[i].astype(np.float64), 0.02, 0.9, 0.05, 5,
+                             QUINTIC, 1e-7, False, "fp64")[0]
+        assert rel(Wbad - Wn[i], Wr - Wn[i]) > 1e-2
+    ctx.close()
