@@ -234,10 +234,23 @@ def run_ours(args, world, rank, local):
         g.zero_()
     torch.cuda.synchronize()
 
-    def one_step():
-        ctx.muon_materialize(flat_g, L, G)
-        ctx.muon_step_batched_out(W, G, M, O, shapes, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
-        ctx.muon_scatter(flat_o, L, O)
+    if args.path == "flat_state":
+        # sharded-state flow: parameters and momenta live in flat fp32 shard buffers too; no whole-matrix state
+        flat_w = torch.zeros(layout.flat_len, dtype=torch.float32, device=dev)
+        flat_m = torch.zeros(layout.flat_len, dtype=torch.float32, device=dev)
+        L4 = mb.Layout(ctx, layout, 4)
+        ctx.muon_scatter(flat_w, L4, W)
+        torch.cuda.synchronize()
+        W, M, G, O = [], [], [], []
+        torch.cuda.empty_cache()
+
+        def one_step():
+            ctx.muon_step_flat(L, flat_w, flat_g, flat_m, flat_o, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
+    else:
+        def one_step():
+            ctx.muon_materialize(flat_g, L, G)
+            ctx.muon_step_batched_out(W, G, M, O, shapes, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
+            ctx.muon_scatter(flat_o, L, O)
 
     for _ in range(args.warmup):
         one_step()
@@ -273,7 +286,7 @@ def run_ours(args, world, rank, local):
 
     # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and args.path == "materialize":
         host_in = host_out = None
         try:
             host_in = torch.empty(layout.flat_len, dtype=torch.bfloat16).pin_memory()
@@ -333,7 +346,9 @@ def run_ours(args, world, rank, local):
         "config": {"workload": f"llama8b: {len(shapes)} matrices ({args.layers} layers x {{Wq, Wo 4096x4096; Wk, Wv 1024x4096; "
                                "gate, up 14336x4096; down 4096x14336}), bf16 row-scaled grads in 8 flat shards, fp32 params and momenta",
                    "elements": n_elem, "ns_steps": wl.NS_STEPS, "coeffs": list(wl.QUINTIC), "lr": LR, "mu": MU, "wd": WD,
-                   "l2": "inputs_exceed_l2", "parallelism": "replicas" if world > 1 else "single"},
+                   "l2": "inputs_exceed_l2", "parallelism": "replicas" if world > 1 else "single",
+                   "path": "materialize -> step -> scatter" if args.path == "materialize" else
+                           "sharded-state flow (muon_step_flat: gather and scatter fused into the elementwise kernels)"},
         "roofline": roofline,
         "ns_tflops": {"algorithmic_symmetric": achieved, "dense_equivalent_effective": dense / ns_s_per_step / 1e12},
         "phases": {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] // args.steps} for k, v in phases.items()},
@@ -354,6 +369,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--layers", type=int, default=32, help="layers of the Llama-3-8B set (32 = the benchmark workload)")
+    ap.add_argument("--path", choices=["materialize", "flat_state"], default="materialize",
+                    help="materialize: the benchmark step (gather, step, scatter); flat_state: the fused sharded-state flow")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -192,6 +192,23 @@ int muon_step_batched_views(muon_ctx_t* ctx, void* const* params, const void* co
                             void* const* updates, const muon_view_t* views, int32_t count, float lr, float mu,
                             float wd, int32_t ns_steps, const float* coeffs, void* stream);
 
+/* muon_step_flat: the sharded-state flow of Section 6.2 on one device -- parameters, momenta and
+ * gradients STAY in flat shard buffers that share one layout ("momentum stays sharded throughout, so
+ * optimizer-state memory never reflows"; "each rank extracts its own slice and applies the update").
+ * The momentum rule reads and writes the flat momentum shards in place and stages the cast result
+ * straight into the Newton-Schulz workspace (the gather is fused away); the update is applied straight
+ * onto the flat fp32 parameter shards and, when flat_updates is given, O is written straight into it
+ * (the scatter is fused away).  No whole-matrix copy of any state exists.
+ *   flat_params, flat_momenta : device, fp32, num_shards*shard_len elements, in/out
+ *   flat_grads                : device, opt.grad_dtype, same element layout
+ *   flat_updates              : device or NULL, NS element type, same element layout; padding untouched
+ * The layout's elem_size is irrelevant here (offsets are in elements).  Requires a layout whose segments
+ * hold whole rows (per-parameter row splits do); otherwise MUON_ERR_UNSUPPORTED and nothing is launched.
+ * Results are bit-identical to muon_materialize + muon_step_batched_out + muon_scatter. */
+int muon_step_flat(muon_ctx_t* ctx, const muon_layout_t* layout, void* flat_params, const void* flat_grads,
+                   void* flat_momenta, void* flat_updates, float lr, float mu, float wd, int32_t ns_steps,
+                   const float* coeffs, void* stream);
+
 /* muon_step_flat_host: the whole path on HOST flat buffers, for end-to-end use and timing.
  * host_flat_grads / host_flat_updates are host buffers of num_shards*shard_len elements in the
  * layout's format (pinned memory makes the copies asynchronous).  Per batch of matrices (the chunks of

@@ -74,6 +74,7 @@ _sig = {
                                         C.c_int32, C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
     "muon_step_batched_views": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(View),
                                           C.c_int32, C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
+    "muon_step_flat": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
     "muon_step_flat_host": (C.c_int, [_vp, _vp, _vp, _vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp),
                                       C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
     "muon_orthogonalize_batched": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(Shape), C.c_int32,
@@ -301,6 +302,13 @@ class Context:
         _check(lib.muon_step_batched_views(self.handle, _ptrs(params), _ptrs(grads), _ptrs(momenta),
                                            None if updates is None else _ptrs(updates), va, len(views), lr, mu, wd, ns_steps,
                                            co, _stream(stream)), "muon_step_batched_views")
+
+    def muon_step_flat(self, layout: Layout, flat_params, flat_grads, flat_momenta, flat_updates, lr, mu, wd, ns_steps, coeffs,
+                       stream=None) -> None:
+        co = (C.c_float * len(coeffs))(*[float(c) for c in coeffs])
+        _check(lib.muon_step_flat(self.handle, layout.handle, flat_params.data_ptr(), flat_grads.data_ptr(),
+                                  flat_momenta.data_ptr(), None if flat_updates is None else flat_updates.data_ptr(),
+                                  lr, mu, wd, ns_steps, co, _stream(stream)), "muon_step_flat")
 
     def muon_step_flat_host(self, host_flat_grads, host_flat_updates, layout: Layout, params, grads, momenta,
                             updates, lr, mu, wd, ns_steps, coeffs, stream=None) -> None:

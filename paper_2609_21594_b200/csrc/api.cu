@@ -1,4 +1,5 @@
 // extern "C" entry points of libmuon_b200: argument validation, plan lookup, kernel sequencing.
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -117,7 +118,8 @@ struct ChunkRun {
   const float* coeffs;
 };
 
-int run_chunk(muon_ctx* ctx, const Chunk& ch, const MatDesc* d_descs, const ChunkRun& r, cudaStream_t st) {
+int run_chunk(muon_ctx* ctx, const Chunk& ch, const MatDesc* d_descs, const ChunkRun& r, cudaStream_t st,
+              const RowSeg* d_segs = nullptr) {
   const WsCarve w = carve_chunk(ctx->opt, ch);
   char* base = static_cast<char*>(ctx->ws);
   void* x0 = base + w.x0;
@@ -130,6 +132,7 @@ int run_chunk(muon_ctx* ctx, const Chunk& ch, const MatDesc* d_descs, const Chun
   {
     Span sp(ctx, MUON_PHASE_MOMENTUM, st);
     StageArgs sa;
+    sa.segs = d_segs;
     sa.descs = d_descs + ch.desc_begin;
     sa.x = x0;
     sa.partials = partials;
@@ -189,6 +192,7 @@ int run_chunk(muon_ctx* ctx, const Chunk& ch, const MatDesc* d_descs, const Chun
   {
     Span sp(ctx, MUON_PHASE_UPDATE, st);
     ApplyArgs aa;
+    aa.segs = d_segs;
     aa.descs = d_descs + ch.desc_begin;
     aa.x = cur;
     aa.count = ch.count;
@@ -229,7 +233,7 @@ cudaEvent_t next_sync_event(muon_ctx* ctx) {
 
 int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const* m, void* const* o,
                 const muon_shape_t* shapes, int32_t count, const ChunkRun& r, cudaStream_t st,
-                const HostPipe* pipe = nullptr, const int64_t* lds = nullptr) {
+                const HostPipe* pipe = nullptr, const int64_t* lds = nullptr, const muon_layout* flat = nullptr) {
   int status;
   Plan* plan = get_plan(ctx, shapes, count, &status);
   if (!plan) return status;
@@ -250,7 +254,9 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
       d.rows = shapes[i].rows;
       d.cols = shapes[i].cols;
       d.ld = lds ? lds[i] : int64_t(d.cols);
-      if (d.ld < d.cols) return MUON_ERR_INVALID_ARG;
+      if (d.ld < d.cols || d.ld > 0x7fffffffLL) return MUON_ERR_INVALID_ARG;
+      d.seg_begin = flat ? flat->rowseg_begin[size_t(i)] : 0;
+      d.seg_count = flat ? flat->rowseg_count[size_t(i)] : 0;
       d.transposed = d.rows > d.cols ? 1 : 0;
       d.scale = float(0.2 * std::sqrt(double(std::max(d.rows, d.cols))));
     }
@@ -260,7 +266,7 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
   if (status != MUON_OK) return status;
   if (!pipe) {
     for (const Chunk& ch : plan->chunks) {
-      status = run_chunk(ctx, ch, static_cast<const MatDesc*>(d_descs), r, st);
+      status = run_chunk(ctx, ch, static_cast<const MatDesc*>(d_descs), r, st, flat ? flat->d_rowsegs : nullptr);
       if (status != MUON_OK) return status;
     }
     return MUON_OK;
@@ -435,10 +441,38 @@ int muon_layout_create(muon_ctx_t* ctx, const muon_layout_desc_t* desc, muon_lay
   L->segs_of.resize(size_t(desc->num_matrices));
   for (int64_t k = 0; k < desc->num_segments; ++k)
     if (desc->segments[k].elem_count > 0) L->segs_of[size_t(desc->segments[k].matrix)].push_back(desc->segments[k]);
+  // Row-aligned layouts (every segment holds whole rows) can also be addressed in place by the step kernels.
+  L->row_aligned = true;
+  for (int64_t k = 0; k < desc->num_segments && L->row_aligned; ++k) {
+    const muon_segment_t& sg = desc->segments[k];
+    const int64_t cols = desc->shapes[sg.matrix].cols;
+    if (sg.elem_count > 0 && (sg.elem_begin % cols || sg.elem_count % cols)) L->row_aligned = false;
+  }
+  if (L->row_aligned) {
+    std::vector<RowSeg> rs;
+    L->rowseg_begin.assign(size_t(desc->num_matrices), 0);
+    L->rowseg_count.assign(size_t(desc->num_matrices), 0);
+    for (int32_t i = 0; i < desc->num_matrices; ++i) {
+      std::vector<muon_segment_t> v = L->segs_of[size_t(i)];
+      std::sort(v.begin(), v.end(), [](const muon_segment_t& a, const muon_segment_t& b) { return a.elem_begin < b.elem_begin; });
+      L->rowseg_begin[size_t(i)] = int32_t(rs.size());
+      L->rowseg_count[size_t(i)] = int32_t(v.size());
+      const int64_t cols = desc->shapes[i].cols;
+      for (const muon_segment_t& sg : v)
+        rs.push_back(RowSeg{int32_t(sg.elem_begin / cols), int32_t(sg.elem_count / cols), sg.flat_offset});
+    }
+    if (!rs.empty() && (cudaMalloc(&L->d_rowsegs, rs.size() * sizeof(RowSeg)) != cudaSuccess ||
+                        cudaMemcpy(L->d_rowsegs, rs.data(), rs.size() * sizeof(RowSeg), cudaMemcpyHostToDevice) != cudaSuccess)) {
+      if (L->d_rowsegs) cudaFree(L->d_rowsegs);
+      delete L;
+      return MUON_ERR_CUDA;
+    }
+  }
   if (!items.empty()) {
     if (cudaMalloc(&L->d_items, items.size() * sizeof(CopyItem)) != cudaSuccess ||
         cudaMemcpy(L->d_items, items.data(), items.size() * sizeof(CopyItem), cudaMemcpyHostToDevice) != cudaSuccess) {
       if (L->d_items) cudaFree(L->d_items);
+      if (L->d_rowsegs) cudaFree(L->d_rowsegs);
       delete L;
       return MUON_ERR_CUDA;
     }
@@ -449,10 +483,9 @@ int muon_layout_create(muon_ctx_t* ctx, const muon_layout_desc_t* desc, muon_lay
 
 void muon_layout_destroy(muon_layout_t* L) {
   if (!L) return;
-  if (L->d_items) {
-    cudaDeviceSynchronize();
-    cudaFree(L->d_items);
-  }
+  if (L->d_items || L->d_rowsegs) cudaDeviceSynchronize();
+  if (L->d_items) cudaFree(L->d_items);
+  if (L->d_rowsegs) cudaFree(L->d_rowsegs);
   delete L;
 }
 
@@ -536,6 +569,25 @@ int muon_step_batched(muon_ctx_t* ctx, void* const* params, const void* const* g
                       const muon_shape_t* shapes, int32_t count, float lr, float mu, float wd, int32_t ns_steps,
                       const float* coeffs, void* stream) {
   return muon_step_batched_out(ctx, params, grads, momenta, nullptr, shapes, count, lr, mu, wd, ns_steps, coeffs, stream);
+}
+
+int muon_step_flat(muon_ctx_t* ctx, const muon_layout_t* layout, void* flat_params, const void* flat_grads,
+                   void* flat_momenta, void* flat_updates, float lr, float mu, float wd, int32_t ns_steps,
+                   const float* coeffs, void* stream) {
+  if (!ctx || !layout) return MUON_ERR_INVALID_ARG;
+  const int32_t count = layout->desc.num_matrices;
+  int rc = check_common(ctx, layout->shapes.data(), count, ns_steps, coeffs);
+  if (rc != MUON_OK) return rc;
+  if (count == 0) return MUON_OK;
+  if (!flat_params || !flat_grads || !flat_momenta || layout->device != ctx->device) return MUON_ERR_INVALID_ARG;
+  if (!std::isfinite(lr) || !std::isfinite(mu) || !std::isfinite(wd)) return MUON_ERR_INVALID_ARG;
+  if (!layout->row_aligned) return MUON_ERR_UNSUPPORTED;   // a segment cuts through a row: use materialize / scatter
+  // Every matrix addresses the flat buffers through its row segments; the per-matrix pointers are the bases.
+  std::vector<void*> w(size_t(count), flat_params), m(size_t(count), flat_momenta), o(size_t(count), flat_updates);
+  std::vector<const void*> g(size_t(count), flat_grads);
+  ChunkRun r{1, 1, lr, mu, wd, ns_steps, coeffs};
+  return run_batched(ctx, w.data(), g.data(), m.data(), flat_updates ? o.data() : nullptr, layout->shapes.data(), count, r,
+                     static_cast<cudaStream_t>(stream), nullptr, nullptr, layout);
 }
 
 int muon_step_flat_host(muon_ctx_t* ctx, const void* host_flat_grads, void* host_flat_updates,
@@ -757,6 +809,7 @@ extern "C" int muon_orthogonalize_static(const void* in, void* out, int32_t rows
   d.ld = cols;
   d.transposed = rows > cols ? 1 : 0;
   d.scale = 0.f;
+  d.seg_begin = d.seg_count = 0;
   MatDesc* d_desc = reinterpret_cast<MatDesc*>(sb + 256);
   // Pageable source: the runtime stages the 48 bytes before returning, so `d` may go out of scope.
   if (cudaMemcpyAsync(d_desc, &d, sizeof(d), cudaMemcpyHostToDevice, st) != cudaSuccess) return MUON_ERR_CUDA;

@@ -29,6 +29,40 @@ template <typename GT> __device__ __forceinline__ float load_g(const GT* p);
 template <> __device__ __forceinline__ float load_g<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 template <> __device__ __forceinline__ float load_g<float>(const float* p) { return *p; }
 
+// Where the rows of a matrix live inside the buffers w/g/m/o point at.  Dense or strided matrices are one
+// run of rows with pitch ld; in flat-shard mode a matrix is a few runs of whole rows (sorted by row, covering
+// every row) with pitch cols.  A thread's four rows almost always fall into one run, so the cursor keeps the
+// current run and only searches when a row leaves it.
+template <bool FLAT>
+struct RowCursor {
+  int row_begin, row_end;
+  size_t base, pitch;
+  __device__ __forceinline__ void init(const MatDesc& d, const RowSeg* __restrict__ segs, int r) {
+    if (!FLAT) {
+      row_begin = 0; row_end = d.rows; base = 0; pitch = size_t(d.ld);
+    } else {
+      pitch = size_t(d.cols);
+      seek(d, segs, r);
+    }
+  }
+  __device__ __forceinline__ void seek(const MatDesc& d, const RowSeg* __restrict__ segs, int r) {
+    row_begin = 0; row_end = 0; base = 0;
+    for (int i = 0; i < d.seg_count; ++i) {
+      const RowSeg sg = segs[d.seg_begin + i];
+      if (r < sg.row_begin + sg.row_count) {
+        row_begin = sg.row_begin; row_end = sg.row_begin + sg.row_count; base = size_t(sg.flat_offset);
+        return;
+      }
+    }
+  }
+  // element offset of (r, 0); r must be a valid row of the matrix
+  __device__ __forceinline__ size_t at(const MatDesc& d, const RowSeg* __restrict__ segs, int r) {
+    if (!FLAT) return size_t(unsigned(r)) * unsigned(d.ld);
+    if (r >= row_end) seek(d, segs, r);
+    return base + size_t(r - row_begin) * pitch;
+  }
+};
+
 __device__ __forceinline__ float block_sum_256(float v, float* red) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -45,7 +79,7 @@ __device__ __forceinline__ float block_sum_256(float v, float* red) {
 
 // GT: gradient/input element type; XT: NS element type; MOM: momentum rule on/off.
 // Thread (ty = tid/16, tx = tid%16) handles 4 consecutive columns tx*4.. of rows ty, ty+16, ty+32, ty+48.
-template <typename GT, typename XT, bool MOM>
+template <typename GT, typename XT, bool MOM, bool FLAT>
 __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
   __shared__ XT tile[T][PADT];
   __shared__ float red[8];
@@ -60,13 +94,15 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   const bool vec = ((d.cols | int(d.ld)) & 3) == 0;
   float sum = 0.f;
+  RowCursor<FLAT> cur;
+  cur.init(d, a.segs, min(r0 + ty, d.rows - 1));
 #pragma unroll
   for (int pass = 0; pass < 4; ++pass) {
     const int rr = ty + pass * 16, cc = tx * 4;
     const int r = r0 + rr, c = c0 + cc;
     float u[4] = {0.f, 0.f, 0.f, 0.f};
     if (r < d.rows && c < d.cols) {
-      const size_t off = size_t(r) * size_t(d.ld) + c;
+      const size_t off = cur.at(d, a.segs, r) + c;
       float g[4], m[4] = {0.f, 0.f, 0.f, 0.f};
       const int nv = min(4, d.cols - c);
       if (vec) {
@@ -171,8 +207,8 @@ __global__ void __launch_bounds__(256) norm_kernel(const float* __restrict__ par
 // XT: NS element type; UPD: 1 = weight update, 0 = plain store of O into d.w (element type XT).
 // The weights of all four passes are requested first, then the O tile (through shared memory when it has
 // to be transposed back), then the arithmetic and the stores.
-template <typename XT, bool UPD>
-__global__ void __launch_bounds__(256) apply_kernel(ApplyArgs a) {
+template <typename XT, bool UPD, bool FLAT>
+__global__ void __launch_bounds__(256, FLAT ? 5 : 6) apply_kernel(ApplyArgs a) {
   __shared__ XT tile[T][PADT];
   const int mat = blockIdx.x / a.tiles_per_mat;
   const int t = blockIdx.x - mat * a.tiles_per_mat;
@@ -187,6 +223,16 @@ __global__ void __launch_bounds__(256) apply_kernel(ApplyArgs a) {
   const int nv = min(4, d.cols - c);
   float w[4][4];
   alignas(16) XT xv[4][4];
+  size_t offs[FLAT ? 4 : 1];
+  if (FLAT) {
+    RowCursor<true> cur;
+    cur.init(d, a.segs, min(r0 + ty, d.rows - 1));
+#pragma unroll
+    for (int pass = 0; pass < 4; ++pass) {
+      const int r = r0 + ty + pass * 16;
+      offs[FLAT ? pass : 0] = r < d.rows ? cur.at(d, a.segs, r) + c : 0;
+    }
+  }
   // ---- loads: W (update mode), then O
   if (UPD) {
 #pragma unroll
@@ -195,7 +241,7 @@ __global__ void __launch_bounds__(256) apply_kernel(ApplyArgs a) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) w[pass][i] = 0.f;
       if (r < d.rows && nv > 0) {
-        const size_t off = size_t(r) * size_t(d.ld) + c;
+        const size_t off = FLAT ? offs[FLAT ? pass : 0] : size_t(unsigned(r)) * unsigned(d.ld) + unsigned(c);
         if (vec) {
           const float4 wv = __ldcs(reinterpret_cast<const float4*>(W + off));
           w[pass][0] = wv.x; w[pass][1] = wv.y; w[pass][2] = wv.z; w[pass][3] = wv.w;
@@ -256,7 +302,7 @@ __global__ void __launch_bounds__(256) apply_kernel(ApplyArgs a) {
   for (int pass = 0; pass < 4; ++pass) {
     const int r = r0 + ty + pass * 16;
     if (r < d.rows && nv > 0) {
-      const size_t off = size_t(r) * size_t(d.ld) + c;
+      const size_t off = FLAT ? offs[FLAT ? pass : 0] : size_t(unsigned(r)) * unsigned(d.ld) + unsigned(c);
       if (UPD) {
         float4 o;
         o.x = w[pass][0] * decay - step * XConv<XT>::to(xv[pass][0]);
@@ -293,40 +339,50 @@ __global__ void __launch_bounds__(256) apply_kernel(ApplyArgs a) {
 
 }  // namespace
 
+template <bool FLAT>
+static void launch_stage_t(const StageArgs& a, unsigned g, cudaStream_t st) {
+  const bool xbf = a.ns_precision == MUON_NS_BF16;
+  if (a.momentum) {
+    const bool gbf = a.grad_dtype == MUON_DTYPE_BF16;
+    if (gbf && xbf) stage_kernel<__nv_bfloat16, __nv_bfloat16, true, FLAT><<<g, 256, 0, st>>>(a);
+    else if (gbf && !xbf) stage_kernel<__nv_bfloat16, float, true, FLAT><<<g, 256, 0, st>>>(a);
+    else if (!gbf && xbf) stage_kernel<float, __nv_bfloat16, true, FLAT><<<g, 256, 0, st>>>(a);
+    else stage_kernel<float, float, true, FLAT><<<g, 256, 0, st>>>(a);
+  } else {
+    if (xbf) stage_kernel<__nv_bfloat16, __nv_bfloat16, false, FLAT><<<g, 256, 0, st>>>(a);
+    else stage_kernel<float, float, false, FLAT><<<g, 256, 0, st>>>(a);
+  }
+}
+
 int launch_stage(const StageArgs& a, cudaStream_t st) {
   const int64_t blocks = int64_t(a.count) * a.tiles_per_mat;
   if (blocks == 0) return 0;
   if (blocks > 0x7fffffffLL) return MUON_ERR_UNSUPPORTED;
-  const unsigned g = unsigned(blocks);
-  const bool xbf = a.ns_precision == MUON_NS_BF16;
-  if (a.momentum) {
-    const bool gbf = a.grad_dtype == MUON_DTYPE_BF16;
-    if (gbf && xbf) stage_kernel<__nv_bfloat16, __nv_bfloat16, true><<<g, 256, 0, st>>>(a);
-    else if (gbf && !xbf) stage_kernel<__nv_bfloat16, float, true><<<g, 256, 0, st>>>(a);
-    else if (!gbf && xbf) stage_kernel<float, __nv_bfloat16, true><<<g, 256, 0, st>>>(a);
-    else stage_kernel<float, float, true><<<g, 256, 0, st>>>(a);
-  } else {
-    if (xbf) stage_kernel<__nv_bfloat16, __nv_bfloat16, false><<<g, 256, 0, st>>>(a);
-    else stage_kernel<float, float, false><<<g, 256, 0, st>>>(a);
-  }
+  if (a.segs) launch_stage_t<true>(a, unsigned(blocks), st);
+  else launch_stage_t<false>(a, unsigned(blocks), st);
   if (cudaGetLastError() != cudaSuccess) return MUON_ERR_CUDA;
   norm_kernel<<<unsigned(a.count), 256, 0, st>>>(a.partials, a.rnorm, a.tiles_per_mat, a.eps, a.normalize);
   return cudaGetLastError() == cudaSuccess ? 2 : MUON_ERR_CUDA;
+}
+
+template <bool FLAT>
+static void launch_apply_t(const ApplyArgs& a, unsigned g, cudaStream_t st) {
+  const bool xbf = a.ns_precision == MUON_NS_BF16;
+  if (a.update) {
+    if (xbf) apply_kernel<__nv_bfloat16, true, FLAT><<<g, 256, 0, st>>>(a);
+    else apply_kernel<float, true, FLAT><<<g, 256, 0, st>>>(a);
+  } else {
+    if (xbf) apply_kernel<__nv_bfloat16, false, FLAT><<<g, 256, 0, st>>>(a);
+    else apply_kernel<float, false, FLAT><<<g, 256, 0, st>>>(a);
+  }
 }
 
 int launch_apply(const ApplyArgs& a, cudaStream_t st) {
   const int64_t blocks = int64_t(a.count) * a.tiles_per_mat;
   if (blocks == 0) return 0;
   if (blocks > 0x7fffffffLL) return MUON_ERR_UNSUPPORTED;
-  const unsigned g = unsigned(blocks);
-  const bool xbf = a.ns_precision == MUON_NS_BF16;
-  if (a.update) {
-    if (xbf) apply_kernel<__nv_bfloat16, true><<<g, 256, 0, st>>>(a);
-    else apply_kernel<float, true><<<g, 256, 0, st>>>(a);
-  } else {
-    if (xbf) apply_kernel<__nv_bfloat16, false><<<g, 256, 0, st>>>(a);
-    else apply_kernel<float, false><<<g, 256, 0, st>>>(a);
-  }
+  if (a.segs) launch_apply_t<true>(a, unsigned(blocks), st);
+  else launch_apply_t<false>(a, unsigned(blocks), st);
   return cudaGetLastError() == cudaSuccess ? 1 : MUON_ERR_CUDA;
 }
 

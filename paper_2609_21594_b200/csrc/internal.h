@@ -26,6 +26,14 @@ struct alignas(16) MatDesc {
   int32_t rows, cols;
   int32_t transposed;   // rows > cols: X holds the transpose
   float scale;          // 0.2*sqrt(max(rows, cols))
+  int32_t seg_begin;    // flat-shard mode: first RowSeg of this matrix; w, g, m, o are then the flat buffers' bases
+  int32_t seg_count;    // 0 = dense/strided addressing through ld
+};
+
+// Rows [row_begin, row_begin + row_count) of a matrix live contiguously at flat_offset (elements) of a flat shard buffer.
+struct alignas(16) RowSeg {
+  int32_t row_begin, row_count;
+  int64_t flat_offset;
 };
 
 // One batched Newton-Schulz invocation: `count` matrices of one core shape (s <= l).
@@ -85,6 +93,9 @@ struct muon_layout {
   int64_t num_items = 0;
   int device = 0;
   std::vector<std::vector<muon_segment_t>> segs_of;   // host copy of the segment table, grouped by matrix
+  bool row_aligned = false;                           // every segment holds whole rows: the flat buffers can be addressed in place
+  muon::RowSeg* d_rowsegs = nullptr;                  // device, all matrices' row segments, sorted by row inside a matrix
+  std::vector<int32_t> rowseg_begin, rowseg_count;    // per matrix: its range in d_rowsegs
 };
 
 struct muon_ctx {
@@ -115,6 +126,7 @@ int launch_copy(const CopyItem* items, int64_t num_items, void* flat, void* cons
                 bool scatter, cudaStream_t st);
 
 struct StageArgs {
+  const RowSeg* segs;     // device row-segment table (flat-shard mode), else null
   const MatDesc* descs;   // device, first record of the chunk
   void* x;                // device, chunk X buffer (bf16 or fp32)
   float* partials;        // device, count*tiles_per_mat
@@ -128,6 +140,7 @@ struct StageArgs {
 int launch_stage(const StageArgs& a, cudaStream_t st);
 
 struct ApplyArgs {
+  const RowSeg* segs;     // device row-segment table (flat-shard mode), else null
   const MatDesc* descs;
   const void* x;          // final NS iterate
   int32_t count, tiles_per_mat, s, l, ldx;
