@@ -214,7 +214,11 @@ def run_ours(args, world, rank, local):
         raise SystemExit("bench.py needs a CUDA device: the Muon path has no CPU fallback")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    shapes = wl.shapes_llama8b(args.layers)
+    if args.config == "llama8b":
+        shapes = wl.shapes_llama8b(args.layers)
+    else:                                   # the other configurations: extra data points, never the headline
+        shapes = wl.CONFIGS[args.config]()
+    cfg, row_scaled = args.config, args.config == "llama8b"
     n_elem = sum(m * n for m, n in shapes)
     layout = wl.layout_per_param(shapes, NUM_SHARDS)
     ctx = mb.Context()
@@ -223,9 +227,9 @@ def run_ours(args, world, rank, local):
     stream = torch.cuda.current_stream()
 
     # ---- state and inputs (seeded, synthetic; drawn on the device)
-    W = [wl.device_draw("llama8b", 0, i, "param", s, dev, std=0.02, dtype=torch.float32) for i, s in enumerate(shapes)]
+    W = [wl.device_draw(cfg, 0, i, "param", s, dev, std=0.02, dtype=torch.float32) for i, s in enumerate(shapes)]
     M = [torch.zeros(s, dtype=torch.float32, device=dev) for s in shapes]
-    G = [wl.device_draw("llama8b", 0, i, "grad", s, dev, std=1e-3, dtype=torch.bfloat16, row_scaled=True) for i, s in enumerate(shapes)]
+    G = [wl.device_draw(cfg, 0, i, "grad", s, dev, std=1e-3, dtype=torch.bfloat16, row_scaled=row_scaled) for i, s in enumerate(shapes)]
     O = [torch.empty(s, dtype=torch.bfloat16, device=dev) for s in shapes]
     flat_g = torch.zeros(layout.flat_len, dtype=torch.bfloat16, device=dev)
     flat_o = torch.zeros(layout.flat_len, dtype=torch.bfloat16, device=dev)
@@ -343,8 +347,9 @@ def run_ours(args, world, rank, local):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": f"llama8b: {len(shapes)} matrices ({args.layers} layers x {{Wq, Wo 4096x4096; Wk, Wv 1024x4096; "
-                               "gate, up 14336x4096; down 4096x14336}), bf16 row-scaled grads in 8 flat shards, fp32 params and momenta",
+        "config": {"workload": (f"llama8b: {len(shapes)} matrices ({args.layers} layers x {{Wq, Wo 4096x4096; Wk, Wv 1024x4096; "
+                                "gate, up 14336x4096; down 4096x14336}), bf16 row-scaled grads in 8 flat shards, fp32 params and momenta")
+                               if cfg == "llama8b" else f"{cfg}: {len(shapes)} matrices, bf16 grads in 8 flat shards, fp32 params and momenta",
                    "elements": n_elem, "ns_steps": wl.NS_STEPS, "coeffs": list(wl.QUINTIC), "lr": LR, "mu": MU, "wd": WD,
                    "l2": "inputs_exceed_l2", "parallelism": "replicas" if world > 1 else "single",
                    "path": "materialize -> step -> scatter" if args.path == "materialize" else
@@ -357,7 +362,7 @@ def run_ours(args, world, rank, local):
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and not args.no_cpu_baseline and cfg == "llama8b":
         line["cpu_baseline"] = cpu_baseline(shapes)
     print(json.dumps(line), flush=True)
 
@@ -369,6 +374,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--layers", type=int, default=32, help="layers of the Llama-3-8B set (32 = the benchmark workload)")
+    ap.add_argument("--config", choices=sorted(wl.CONFIGS), default="llama8b",
+                    help="llama8b is the benchmark workload; the others are extra data points")
     ap.add_argument("--path", choices=["materialize", "flat_state"], default="materialize",
                     help="materialize: the benchmark step (gather, step, scatter); flat_state: the fused sharded-state flow")
     ap.add_argument("--e2e-steps", type=int, default=3)
