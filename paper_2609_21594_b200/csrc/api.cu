@@ -199,6 +199,7 @@ int run_chunk(muon_ctx* ctx, const Chunk& ch, const MatDesc* d_descs, const Chun
     aa.tiles_per_mat = ch.tiles_per_mat;
     aa.s = ch.s; aa.l = ch.l; aa.ldx = ch.ldx;
     aa.lr = r.lr; aa.wd = r.wd;
+    aa.decay = 1.0f - r.lr * r.wd;
     aa.ns_precision = ctx->opt.ns_precision;
     aa.update = r.momentum;
     n = launch_apply(aa, st);

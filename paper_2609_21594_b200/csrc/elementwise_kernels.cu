@@ -296,7 +296,7 @@ __global__ void __launch_bounds__(256, FLAT ? 5 : 6) apply_kernel(ApplyArgs a) {
     }
   }
   // ---- arithmetic and stores
-  const float decay = 1.0f - a.lr * a.wd;
+  const float decay = a.decay;
   const float step = a.lr * d.scale;
 #pragma unroll
   for (int pass = 0; pass < 4; ++pass) {
@@ -304,11 +304,13 @@ __global__ void __launch_bounds__(256, FLAT ? 5 : 6) apply_kernel(ApplyArgs a) {
     if (r < d.rows && nv > 0) {
       const size_t off = FLAT ? offs[FLAT ? pass : 0] : size_t(unsigned(r)) * unsigned(d.ld) + unsigned(c);
       if (UPD) {
+        // two explicit roundings (product, then fused multiply-add): the result does not depend on how the
+        // compiler contracts the expression
         float4 o;
-        o.x = w[pass][0] * decay - step * XConv<XT>::to(xv[pass][0]);
-        o.y = w[pass][1] * decay - step * XConv<XT>::to(xv[pass][1]);
-        o.z = w[pass][2] * decay - step * XConv<XT>::to(xv[pass][2]);
-        o.w = w[pass][3] * decay - step * XConv<XT>::to(xv[pass][3]);
+        o.x = __fmaf_rn(-step, XConv<XT>::to(xv[pass][0]), __fmul_rn(w[pass][0], decay));
+        o.y = __fmaf_rn(-step, XConv<XT>::to(xv[pass][1]), __fmul_rn(w[pass][1], decay));
+        o.z = __fmaf_rn(-step, XConv<XT>::to(xv[pass][2]), __fmul_rn(w[pass][2], decay));
+        o.w = __fmaf_rn(-step, XConv<XT>::to(xv[pass][3]), __fmul_rn(w[pass][3], decay));
         if (vec) {
           __stcs(reinterpret_cast<float4*>(W + off), o);
         } else {

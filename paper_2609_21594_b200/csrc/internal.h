@@ -145,6 +145,7 @@ struct ApplyArgs {
   const void* x;          // final NS iterate
   int32_t count, tiles_per_mat, s, l, ldx;
   float lr, wd;
+  float decay;            // 1 - lr*wd, computed once on the host so that every update route uses the same value
   int32_t ns_precision;
   int32_t update;         // 1: W <- W(1-lr*wd) - lr*scale*O ; 0: write O into descs[i].w in the NS element type
 };

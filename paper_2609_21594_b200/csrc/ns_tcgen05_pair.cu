@@ -35,8 +35,6 @@ constexpr int STAGES = 6;
 constexpr int A_BYTES = BM * BK * 2;          // 16 KiB
 constexpr int B_BYTES = BNH * BK * 2;         // 16 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int EPI_COLS = 64;
-constexpr int EPI_BYTES = BM * EPI_COLS * 2;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * EPI_BYTES + 1024 + 256;
 constexpr int TMEM_COLS = 512;
 constexpr int NUM_THREADS = 192;
@@ -235,104 +233,23 @@ ns_product_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps (per CTA: its 128 rows)
-    const int quad = warp & 3;
-    const int etid = threadIdx.x - 64;
-    const bool leader = etid == 0;
-    const int lrow = quad * 32 + lane;
-    uint32_t tile_it = 0, g = 0, eph = 0;
+    const int quad = warp & 3;                     // TMEM lane quadrant this warp may read
+    EpilogueState est;
+    uint32_t tile_it = 0;
     bool ok = true;
-    auto group_sync = [&]() -> bool {
-      __syncwarp();
-      if (lane == 0) mbar_arrive(egroup_bar);
-      const bool done = mbar_wait(egroup_bar, eph, abort_flag);
-      eph ^= 1u;
-      return done;
-    };
     for (int t = pair_id; t < total_tiles && ok; t += num_pairs, ++tile_it) {
       const Tile tl = decode_tile(t, a);
-      const int m0 = tl.m0 + int(rank) * BM;
       const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-      float gamma = 1.f;
-      if (a.gamma_mode) {
-        const float r = a.rnorm[tl.mat];
-        gamma = a.gamma_mode == 1 ? r : r * r;
-      }
-      const int row = m0 + lrow;
-      const bool row_ok = row < a.m;
-      __nv_bfloat16* cmat = a.c + size_t(tl.mat) * a.stride_c;
       const bool mirror = a.symmetric && tl.n0 > tl.m0;          // pair tile strictly above the diagonal block
       const uint32_t taddr = tmem_base + acc * uint32_t(BN) + (uint32_t(quad * 32) << 16);
-      bool acc_ready = false;
-#pragma unroll 1
-      for (int cb = 0; cb < BN / EPI_COLS; ++cb, ++g) {
-        const int c0 = tl.n0 + cb * EPI_COLS;
-        if (c0 >= a.n) break;
-        const uint32_t b = g & 1u;
-        const uint32_t ebuf = epi_base + b * EPI_BYTES;
-        if (leader) {
-          tma_wait_read<1>();
-          if (a.d) {
-            mbar_expect_tx(dfull_bar(int(b)), EPI_BYTES);
-            tma_load_3d(ebuf, &map_d, dfull_bar(int(b)), c0, m0, tl.mat);
-          }
-        }
-        if (!acc_ready) {
-          if (!mbar_wait(tfull_bar(int(acc)), aph, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          acc_ready = true;
-        }
-        if (a.d) {
-          if (!mbar_wait(dfull_bar(int(b)), (g >> 1) & 1u, abort_flag)) { ok = false; break; }
-        } else {
-          if (!group_sync()) { ok = false; break; }
-        }
-        uint32_t v[64];
-        tc_ld32(taddr + uint32_t(cb * EPI_COLS), *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
-        tc_ld32(taddr + uint32_t(cb * EPI_COLS + 32), *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
-        tc_wait_ld();
-        const uint32_t srow = ebuf + uint32_t(lrow) * 128u;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          const uint32_t addr = srow + (uint32_t(q ^ (lrow & 7)) << 4);
-          uint32_t d0 = 0, d1 = 0, d2 = 0, d3 = 0;
-          if (a.d) asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3) : "r"(addr));
-          const uint32_t dd[4] = {d0, d1, d2, d3};
-          uint32_t oo[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            float x0 = a.alpha * __uint_as_float(v[q * 8 + 2 * e]), x1 = a.alpha * __uint_as_float(v[q * 8 + 2 * e + 1]);
-            if (a.d) {
-              const __nv_bfloat162 dp = *reinterpret_cast<const __nv_bfloat162*>(&dd[e]);
-              x0 += a.beta * __low2float(dp);
-              x1 += a.beta * __high2float(dp);
-            }
-            const __nv_bfloat162 o = __floats2bfloat162_rn(gamma * x0, gamma * x1);
-            oo[e] = *reinterpret_cast<const uint32_t*>(&o);
-          }
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(oo[0]), "r"(oo[1]), "r"(oo[2]), "r"(oo[3]) : "memory");
-          if (mirror && row_ok) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int c = c0 + q * 8 + 2 * e;
-              const __nv_bfloat162 o = *reinterpret_cast<const __nv_bfloat162*>(&oo[e]);
-              if (c < a.n) cmat[size_t(c) * a.ldc + row] = __low2bfloat16(o);
-              if (c + 1 < a.n) cmat[size_t(c + 1) * a.ldc + row] = __high2bfloat16(o);
-            }
-          }
-        }
-        fence_async_smem();
-        if (!group_sync()) { ok = false; break; }
-        if (leader) {
-          tma_store_3d(&map_c, ebuf, c0, m0, tl.mat);
-          tma_commit();
-        }
-      }
+      ok = epilogue_tile(a, &map_d, &map_c, tl.mat, tl.m0 + int(rank) * BM, tl.n0, mirror, taddr, epi_base, dfull_bar(0),
+                         egroup_bar, tfull_bar(int(acc)), aph, abort_flag, est, quad, lane);
       if (!ok) break;
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(int(acc)), 0));   // the leader CTA counts both epilogues
     }
-    if (leader) tma_wait_all();
+    if (quad == 2 && lane == 0) tma_wait_all();     // every store has landed before the CTA retires
     if (!ok && lane == 0) {
       *abort_flag = 1;
       atomicExch(a.status, 14);

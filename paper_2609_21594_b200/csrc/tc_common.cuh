@@ -133,6 +133,114 @@ __host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major, int umma_m, i
          (uint32_t(umma_m >> 4) << 24);
 }
 
+
+// ------------------------------------------------------------------ epilogue of one 128 x 256 accumulator tile
+constexpr int EPI_TILE_N = 256;
+constexpr int EPI_ROWS = 128;
+constexpr int EPI_COLS = 64;                         // columns per chunk (one 128-byte swizzle row of bf16)
+constexpr int EPI_BYTES = EPI_ROWS * EPI_COLS * 2;   // 16 KiB staging buffer, two of them
+
+// State the four epilogue warps carry from tile to tile.
+struct EpilogueState {
+  uint32_t g = 0;      // chunks processed so far (staging buffer = g & 1)
+  uint32_t eph = 0;    // phase of the group rendezvous
+};
+
+// Thread = one accumulator row (TMEM lane).  The tile leaves in four 64-column chunks through two
+// 128B-swizzled staging buffers: TMA brings the D chunk in, every thread turns its own row of D into its
+// row of C in place (one bf16 rounding of gamma*(beta*D + alpha*acc)), TMA stores the chunk; a strictly
+// upper tile of a symmetric product is also written transposed with plain stores (64 contiguous bytes per
+// warp instruction).  Returns false when a bounded wait expired.
+__device__ __forceinline__ bool epilogue_tile(const TcArgs& a, const CUtensorMap* map_d, const CUtensorMap* map_c, int mat,
+                                              int m0, int n0, bool mirror, uint32_t taddr, uint32_t epi_base,
+                                              uint32_t dfull_bar0, uint32_t egroup_bar, uint32_t tfull_bar, uint32_t aph,
+                                              volatile int* abort_flag, EpilogueState& st, int quad, int lane) {
+  const bool leader = quad == 2 && lane == 0;        // warp 2 is the first epilogue warp
+  const int lrow = quad * 32 + lane;
+  auto group_sync = [&]() -> bool {                  // rendezvous of the four warps on an mbarrier: bounded like every wait
+    __syncwarp();
+    if (lane == 0) mbar_arrive(egroup_bar);
+    const bool done = mbar_wait(egroup_bar, st.eph, abort_flag);
+    st.eph ^= 1u;
+    return done;
+  };
+  float gamma = 1.f;
+  if (a.gamma_mode) {
+    const float r = a.rnorm[mat];
+    gamma = a.gamma_mode == 1 ? r : r * r;
+  }
+  const int row = m0 + lrow;
+  const bool row_ok = row < a.m;
+  __nv_bfloat16* cmat = a.c + size_t(mat) * a.stride_c;
+  bool acc_ready = false;
+#pragma unroll 1
+  for (int cb = 0; cb < EPI_TILE_N / EPI_COLS; ++cb, ++st.g) {
+    const int c0 = n0 + cb * EPI_COLS;
+    if (c0 >= a.n) break;                             // uniform over the group
+    const uint32_t b = st.g & 1u;
+    const uint32_t ebuf = epi_base + b * EPI_BYTES;
+    const uint32_t dbar = dfull_bar0 + b * 8u;
+    if (leader) {
+      tma_wait_read<1>();                             // the store that last used this buffer has read it
+      if (a.d) {
+        mbar_expect_tx(dbar, EPI_BYTES);
+        tma_load_3d(ebuf, map_d, dbar, c0, m0, mat);
+      }
+    }
+    if (!acc_ready) {
+      if (!mbar_wait(tfull_bar, aph, abort_flag)) return false;
+      tc_fence_after();
+      acc_ready = true;
+    }
+    if (a.d) {
+      if (!mbar_wait(dbar, (st.g >> 1) & 1u, abort_flag)) return false;
+    } else {
+      if (!group_sync()) return false;                // the leader's wait_group above frees the buffer for everyone
+    }
+    uint32_t v[64];
+    tc_ld32(taddr + uint32_t(cb * EPI_COLS), *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+    tc_ld32(taddr + uint32_t(cb * EPI_COLS + 32), *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+    tc_wait_ld();
+    const uint32_t srow = ebuf + uint32_t(lrow) * 128u;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {                     // 16-byte piece q of the row sits at piece q ^ (row & 7)
+      const uint32_t addr = srow + (uint32_t(q ^ (lrow & 7)) << 4);
+      uint32_t d0 = 0, d1 = 0, d2 = 0, d3 = 0;
+      if (a.d) asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3) : "r"(addr));
+      const uint32_t dd[4] = {d0, d1, d2, d3};
+      uint32_t oo[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float x0 = a.alpha * __uint_as_float(v[q * 8 + 2 * e]), x1 = a.alpha * __uint_as_float(v[q * 8 + 2 * e + 1]);
+        if (a.d) {
+          const __nv_bfloat162 dp = *reinterpret_cast<const __nv_bfloat162*>(&dd[e]);
+          x0 += a.beta * __low2float(dp);
+          x1 += a.beta * __high2float(dp);
+        }
+        const __nv_bfloat162 o = __floats2bfloat162_rn(gamma * x0, gamma * x1);
+        oo[e] = *reinterpret_cast<const uint32_t*>(&o);
+      }
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(oo[0]), "r"(oo[1]), "r"(oo[2]), "r"(oo[3]) : "memory");
+      if (mirror && row_ok) {                         // C[c][row] = C[row][c]
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int c = c0 + q * 8 + 2 * e;
+          const __nv_bfloat162 o = *reinterpret_cast<const __nv_bfloat162*>(&oo[e]);
+          if (c < a.n) cmat[size_t(c) * a.ldc + row] = __low2bfloat16(o);
+          if (c + 1 < a.n) cmat[size_t(c + 1) * a.ldc + row] = __high2bfloat16(o);
+        }
+      }
+    }
+    fence_async_smem();                               // generic-proxy writes -> visible to the TMA store
+    if (!group_sync()) return false;                  // everyone is done with the buffer (reads of D, writes of C)
+    if (leader) {
+      tma_store_3d(map_c, ebuf, c0, m0, mat);         // rows/columns beyond the matrix are clipped
+      tma_commit();
+    }
+  }
+  return true;
+}
+
 // ------------------------------------------------------------------ host: tensor maps
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
