@@ -384,3 +384,20 @@ def test_plain_momentum_rule_and_eps_option():
                              QUINTIC, 1e-7, False, "fp64")[0]
         assert rel(Wbad - Wn[i], Wr - Wn[i]) > 1e-2
     ctx.close()
+
+
+@pytest.mark.parametrize("engine", ["tensor", "tensor_1cta"])
+def test_ns_ragged_multi_tile_shapes(engine):
+    """Shapes that are no multiple of any tile size and span several 256-wide tiles: the last CTA pair owns a
+    partly (1300 = 5*256 + 20) or a half-empty (1408 = 5*256 + 128) row block, columns end inside a TMA box."""
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "bf16", engine)
+    shapes = [(1300, 2100), (2100, 1300), (1408, 2048), (520, 520), (385, 1031)]
+    mats = [wl.grad_np("ragged_big", 0, i, s) for i, s in enumerate(shapes)]
+    outs, vals = _ortho(mb, ctx, mats)
+    for i, (o, v) in enumerate(zip(outs, vals)):
+        assert np.isfinite(o).all()
+        ref = orc.newton_schulz(v, 5, QUINTIC, 1e-7, "bf16")
+        assert rel(o, ref) <= TOL_BF16, (i, shapes[i], rel(o, ref))
+    ctx.close()
