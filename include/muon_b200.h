@@ -291,6 +291,15 @@ int muon_orthogonalize_static(const void* in, void* out, int32_t rows, int32_t c
  * after synchronising `stream`; 0 = no bounded wait ever expired on this context. */
 int muon_last_device_status(muon_ctx_t* ctx, void* stream, int32_t* status);
 
+/* Resets the status word to 0 (stream-ordered). */
+int muon_clear_device_status(muon_ctx_t* ctx, void* stream);
+
+/* Failure-detection self-test: launches one tiny kernel that waits, with a limit of about a millisecond,
+ * on a barrier nothing ever arrives at, using the same bounded-wait routine as the tensor-core pipelines.
+ * The wait must expire, the kernel records code 100 in the status word and returns normally; the context
+ * stays usable.  No real pipeline is involved and nothing can hang. */
+int muon_self_test_bounded_wait(muon_ctx_t* ctx, void* stream);
+
 /* Phase timing (off by default).  When on, the library brackets each phase with CUDA
  * events on the caller's stream; muon_profile_read synchronises those events and adds up,
  * per phase, device milliseconds and kernel launches since the last muon_profile_reset. */

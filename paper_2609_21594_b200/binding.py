@@ -85,6 +85,8 @@ _sig = {
     "muon_orthogonalize_static": (C.c_int, [_vp, _vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_float),
                                             C.c_float, C.c_uint32, _vp, _vp]),
     "muon_last_device_status": (C.c_int, [_vp, _vp, C.POINTER(C.c_int32)]),
+    "muon_clear_device_status": (C.c_int, [_vp, _vp]),
+    "muon_self_test_bounded_wait": (C.c_int, [_vp, _vp]),
     "muon_profile_enable": (C.c_int, [_vp, C.c_int32]),
     "muon_profile_reset": (C.c_int, [_vp]),
     "muon_profile_read": (C.c_int, [_vp, C.c_int32, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
@@ -334,6 +336,12 @@ class Context:
         v = C.c_int32(0)
         _check(lib.muon_last_device_status(self.handle, _stream(stream), C.byref(v)), "muon_last_device_status")
         return int(v.value)
+
+    def muon_clear_device_status(self, stream=None) -> None:
+        _check(lib.muon_clear_device_status(self.handle, _stream(stream)), "muon_clear_device_status")
+
+    def muon_self_test_bounded_wait(self, stream=None) -> None:
+        _check(lib.muon_self_test_bounded_wait(self.handle, _stream(stream)), "muon_self_test_bounded_wait")
 
     # -- profiling
     def muon_profile_enable(self, on: bool) -> None:

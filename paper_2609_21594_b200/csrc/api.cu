@@ -666,6 +666,21 @@ int muon_last_device_status(muon_ctx_t* ctx, void* stream, int32_t* status) {
   return MUON_OK;
 }
 
+int muon_clear_device_status(muon_ctx_t* ctx, void* stream) {
+  if (!ctx) return MUON_ERR_INVALID_ARG;
+  return cudaMemsetAsync(ctx->d_status, 0, sizeof(int32_t), static_cast<cudaStream_t>(stream)) == cudaSuccess ? MUON_OK
+                                                                                                               : MUON_ERR_CUDA;
+}
+
+int muon_self_test_bounded_wait(muon_ctx_t* ctx, void* stream) {
+  if (!ctx) return MUON_ERR_INVALID_ARG;
+  if (!DeviceGuardCheck::ok(ctx)) return MUON_ERR_CUDA;
+  const int n = launch_bounded_wait_probe(ctx, static_cast<cudaStream_t>(stream));
+  if (n < 0) return n;
+  ctx->launches += n;
+  return MUON_OK;
+}
+
 int muon_profile_enable(muon_ctx_t* ctx, int32_t on) {
   if (!ctx) return MUON_ERR_INVALID_ARG;
   ctx->profiling = on != 0;

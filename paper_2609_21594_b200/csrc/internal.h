@@ -169,5 +169,6 @@ int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st);   // tcge
 bool tc_supported(const GemmArgs& a);
 int launch_gemm_tc_pair(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st);   // two-CTA (cta_group::2) variant
 bool tc_pair_supported(const GemmArgs& a);
+int launch_bounded_wait_probe(muon_ctx* ctx, cudaStream_t st);            // a wait that must expire (self-test)
 
 }  // namespace muon

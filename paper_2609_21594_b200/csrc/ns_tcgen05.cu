@@ -223,7 +223,29 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
 constexpr int kMaxDevices = 64;
 int g_num_sms[kMaxDevices] = {};
 
+// A wait that nothing ever satisfies, with a short limit: exercises the bounded-wait machinery (deadline,
+// status word, clean return) without putting any real pipeline at risk.
+__global__ void bounded_wait_probe_kernel(int32_t* status, long long limit_cycles) {
+  __shared__ alignas(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const bool done = mbar_wait(smem_u32(&bar), 0, &abort_flag, true, limit_cycles);   // nobody arrives: must expire
+    if (!done) atomicExch(status, 100);
+  }
+}
+
 }  // namespace
+
+int launch_bounded_wait_probe(muon_ctx* ctx, cudaStream_t st) {
+  bounded_wait_probe_kernel<<<1, 32, 0, st>>>(ctx->d_status, 2000000LL);   // about a millisecond
+  return cudaGetLastError() == cudaSuccess ? 1 : MUON_ERR_CUDA;
+}
 
 bool tc_supported(const GemmArgs& a) {
   if (a.m < 1 || a.n < 1 || a.kdim < 1 || a.batch < 1) return false;
