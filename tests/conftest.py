@@ -10,6 +10,11 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
+    # The tests talk to the in-tree shared library; build it when it is missing or older than its sources
+    # (nvcc cross-compiles for sm_100a without a GPU).
+    from paper_2609_21594_b200 import build
+
+    build.build()
 
 
 def pytest_collection_modifyitems(config, items):
