@@ -263,28 +263,43 @@ def run_ours(args, world, rank, local):
         raise SystemExit("a bounded device-side wait expired during warm-up")
 
     # ---- device-resident timing
-    ctx.muon_profile_enable(True)
-    ctx.muon_profile_reset()
-    launches0 = ctx.muon_launch_count()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    barrier(world)
-    torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(args.steps):
-        one_step()
-    e1.record(stream)
-    torch.cuda.synchronize()
-    barrier(world)
-    clocks = sampler.stop() if rank == 0 else {}
-    ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
-    launches = ctx.muon_launch_count() - launches0
-    phases = ctx.muon_profile_read()
-    ctx.muon_profile_enable(False)
-    if ctx.muon_last_device_status() != 0:
-        raise SystemExit("a bounded device-side wait expired during the timed region")
+
+    def timed_region():
+        ctx.muon_profile_enable(True)
+        ctx.muon_profile_reset()
+        launches0 = ctx.muon_launch_count()
+        sampler = ClockSampler(local)
+        if rank == 0:
+            sampler.start()
+        barrier(world)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(args.steps):
+            one_step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        barrier(world)
+        clk = sampler.stop() if rank == 0 else {}
+        t = max_over_ranks(e0.elapsed_time(e1), world, dev)
+        n = ctx.muon_launch_count() - launches0
+        ph = ctx.muon_profile_read()
+        ctx.muon_profile_enable(False)
+        if ctx.muon_last_device_status() != 0:
+            raise SystemExit("a bounded device-side wait expired during the timed region")
+        return t, n, ph, clk
+
+    ms, launches, phases, clocks = timed_region()
+    # A region that saw a hardware or thermal slowdown, or clocks stuck low with no reason (a leftover lock), does
+    # not count: measure once more.  sw_power_cap alone is normal for a dense-GEMM workload on a 1 kW part.
+    bad = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
+    stuck = 0.0
+    if rank == 0 and clocks.get("sm_mhz") and clocks.get("sm_max_mhz"):
+        stuck = 1.0 if (not clocks.get("reasons") and clocks["sm_mhz"] < 0.6 * clocks["sm_max_mhz"]) else 0.0
+    redo = 1.0 if (rank == 0 and (bad & set(clocks.get("reasons", [])) or stuck)) else 0.0
+    if max_over_ranks(redo, world, dev) > 0:
+        ms, launches, phases, clocks = timed_region()
+        clocks["remeasured"] = True
     ms_per_step = ms / args.steps
     value = world * 1e3 / ms_per_step
 

@@ -28,11 +28,11 @@ constexpr int BM = 128;          // tile rows   (UMMA M)
 constexpr int BN = 256;          // tile cols   (UMMA N)
 constexpr int BK = 64;           // k per stage (one 128-byte swizzle atom of bf16)
 constexpr int UK = 16;           // k per tcgen05.mma for 16-bit inputs
-constexpr int STAGES = 4;
+constexpr int STAGES = 3;
 constexpr int A_BYTES = BM * BK * 2;          // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;          // 32 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * EPI_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BUFS * EPI_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int TMEM_COLS = 512;
 constexpr int NUM_THREADS = 192;
 
@@ -75,12 +75,12 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
   const uint32_t base = (raw + 1023u) & ~1023u;            // swizzled tiles need 1024-byte alignment
   uint8_t* gen_base = smem_raw + (base - raw);
   const uint32_t epi_base = base + STAGES * STAGE_BYTES;    // two epilogue staging buffers follow the ring
-  constexpr int BAR_OFF = STAGES * STAGE_BYTES + 2 * EPI_BYTES;
+  constexpr int BAR_OFF = STAGES * STAGE_BYTES + EPI_BUFS * EPI_BYTES;
   const uint32_t bars = base + BAR_OFF;                     // barrier block follows the buffers
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + BAR_OFF + 128);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + BAR_OFF + 136);
   auto dfull_bar = [&](int i) { return bars + uint32_t(2 * STAGES + 4 + i) * 8u; };
-  const uint32_t egroup_bar = bars + uint32_t(2 * STAGES + 6) * 8u;   // 128-thread rendezvous of the epilogue group
+  const uint32_t egroup_bar = bars + uint32_t(2 * STAGES + 4 + EPI_BUFS) * 8u;   // 128-thread rendezvous of the epilogue group
   auto full_bar = [&](int s) { return bars + uint32_t(s) * 8u; };
   auto empty_bar = [&](int s) { return bars + uint32_t(STAGES + s) * 8u; };
   auto tfull_bar = [&](int i) { return bars + uint32_t(2 * STAGES + i) * 8u; };
@@ -98,8 +98,8 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
     for (int i = 0; i < 2; ++i) {
       mbar_init(tfull_bar(i), 1);
       mbar_init(tempty_bar(i), 4);
-      mbar_init(dfull_bar(i), 1);
     }
+    for (int i = 0; i < EPI_BUFS; ++i) mbar_init(dfull_bar(i), 1);
     mbar_init(egroup_bar, 4);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -196,14 +196,24 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
       const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
       const bool mirror = a.symmetric && tl.n0 >= tl.m0 + BM;   // tile lies strictly above the diagonal
       const uint32_t taddr = tmem_base + acc * uint32_t(BN) + (uint32_t(quad * 32) << 16);
-      ok = epilogue_tile(a, &map_d, &map_c, tl.mat, tl.m0, tl.n0, mirror, taddr, epi_base, dfull_bar(0), egroup_bar,
-                         tfull_bar(int(acc)), aph, abort_flag, est, quad, lane);
+      const EpiTile cur{tl.mat, tl.m0, tl.n0, true};
+      EpiTile nxt{0, 0, 0, false};
+      if (t + int(gridDim.x) < total_tiles) {
+        const Tile tn = decode_tile(t + int(gridDim.x), a);
+        nxt = EpiTile{tn.mat, tn.m0, tn.n0, true};
+      }
+      ok = epilogue_tile(a, &map_d, &map_c, cur, nxt, mirror, taddr, epi_base, dfull_bar(0), egroup_bar, tfull_bar(int(acc)),
+                         aph, abort_flag, est, quad, lane);
       if (!ok) break;
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(int(acc)));
     }
-    if (quad == 2 && lane == 0) tma_wait_all();     // every store has landed before the CTA retires
+    if (quad == 2 && lane == 0) {
+      tma_wait_all();                               // every store has landed before the CTA retires
+      if (!ok)                                      // a prefetched D chunk may still be landing: give it (bounded) time
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    }
     if (!ok && lane == 0) {
       *abort_flag = 1;
       atomicExch(a.status, 4);

@@ -6,7 +6,7 @@
 //
 // A pair owns a 256 x 256 output tile.  CTA r of the pair (r = 0, 1) owns rows [128 r, 128 r + 128):
 // it loads those 128 rows of P and HALF of the Q tile (128 of the 256 columns of the output) per
-// 64-wide k-block -- 32 KiB per stage instead of 48 KiB, so six stages fit and the bytes that cross
+// 64-wide k-block -- 32 KiB per stage instead of 48 KiB, so five stages and a three-buffer epilogue ring fit and the bytes that cross
 // L2 -> shared memory per flop drop by a third.  The leader (r = 0) issues every MMA; the hardware
 // reads each CTA's own P rows and both CTAs' Q halves.  Each CTA keeps its 128 x 256 fp32 accumulator
 // in its own TMEM (double-buffered) and runs its own epilogue.
@@ -31,11 +31,11 @@ constexpr int BN = 256;          // columns of the pair's tile
 constexpr int BNH = 128;         // columns of Q each CTA stages
 constexpr int BK = 64;
 constexpr int UK = 16;
-constexpr int STAGES = 6;
+constexpr int STAGES = 5;
 constexpr int A_BYTES = BM * BK * 2;          // 16 KiB
 constexpr int B_BYTES = BNH * BK * 2;         // 16 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * EPI_BYTES + 1024 + 256;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BUFS * EPI_BYTES + 1024 + 256;
 constexpr int TMEM_COLS = 512;
 constexpr int NUM_THREADS = 192;
 
@@ -114,7 +114,7 @@ ns_product_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (base - raw);
   const uint32_t epi_base = base + STAGES * STAGE_BYTES;
-  constexpr int BAR_OFF = STAGES * STAGE_BYTES + 2 * EPI_BYTES;
+  constexpr int BAR_OFF = STAGES * STAGE_BYTES + EPI_BUFS * EPI_BYTES;
   const uint32_t bars = base + BAR_OFF;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + BAR_OFF + 192);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + BAR_OFF + 200);
@@ -123,7 +123,7 @@ ns_product_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
   auto tfull_bar = [&](int i) { return bars + uint32_t(2 * STAGES + i) * 8u; };
   auto tempty_bar = [&](int i) { return bars + uint32_t(2 * STAGES + 2 + i) * 8u; };
   auto dfull_bar = [&](int i) { return bars + uint32_t(2 * STAGES + 4 + i) * 8u; };
-  const uint32_t egroup_bar = bars + uint32_t(2 * STAGES + 6) * 8u;
+  const uint32_t egroup_bar = bars + uint32_t(2 * STAGES + 4 + EPI_BUFS) * 8u;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();
@@ -140,8 +140,8 @@ ns_product_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
     for (int i = 0; i < 2; ++i) {
       mbar_init(tfull_bar(i), 1);
       mbar_init(tempty_bar(i), 8);
-      mbar_init(dfull_bar(i), 1);
     }
+    for (int i = 0; i < EPI_BUFS; ++i) mbar_init(dfull_bar(i), 1);
     mbar_init(egroup_bar, 4);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -242,14 +242,24 @@ ns_product_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
       const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
       const bool mirror = a.symmetric && tl.n0 > tl.m0;          // pair tile strictly above the diagonal block
       const uint32_t taddr = tmem_base + acc * uint32_t(BN) + (uint32_t(quad * 32) << 16);
-      ok = epilogue_tile(a, &map_d, &map_c, tl.mat, tl.m0 + int(rank) * BM, tl.n0, mirror, taddr, epi_base, dfull_bar(0),
-                         egroup_bar, tfull_bar(int(acc)), aph, abort_flag, est, quad, lane);
+      const EpiTile cur{tl.mat, tl.m0 + int(rank) * BM, tl.n0, true};
+      EpiTile nxt{0, 0, 0, false};
+      if (t + num_pairs < total_tiles) {
+        const Tile tn = decode_tile(t + num_pairs, a);
+        nxt = EpiTile{tn.mat, tn.m0 + int(rank) * BM, tn.n0, true};
+      }
+      ok = epilogue_tile(a, &map_d, &map_c, cur, nxt, mirror, taddr, epi_base, dfull_bar(0), egroup_bar, tfull_bar(int(acc)),
+                         aph, abort_flag, est, quad, lane);
       if (!ok) break;
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(int(acc)), 0));   // the leader CTA counts both epilogues
     }
-    if (quad == 2 && lane == 0) tma_wait_all();     // every store has landed before the CTA retires
+    if (quad == 2 && lane == 0) {
+      tma_wait_all();                               // every store has landed before the CTA retires
+      if (!ok)                                      // a prefetched D chunk may still be landing: give it (bounded) time
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    }
     if (!ok && lane == 0) {
       *abort_flag = 1;
       atomicExch(a.status, 14);

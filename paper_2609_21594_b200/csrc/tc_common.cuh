@@ -138,23 +138,32 @@ __host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major, int umma_m, i
 constexpr int EPI_TILE_N = 256;
 constexpr int EPI_ROWS = 128;
 constexpr int EPI_COLS = 64;                         // columns per chunk (one 128-byte swizzle row of bf16)
-constexpr int EPI_BYTES = EPI_ROWS * EPI_COLS * 2;   // 16 KiB staging buffer, two of them
+constexpr int EPI_BYTES = EPI_ROWS * EPI_COLS * 2;   // 16 KiB staging buffer
+constexpr int EPI_BUFS = 3;                          // ring of staging buffers: chunk g uses buffer g % 3
+
+// Where a tile of C lives: matrix, first row of this CTA's 128 rows, first column.
+struct EpiTile {
+  int mat, m0, n0;
+  bool valid;
+};
 
 // State the four epilogue warps carry from tile to tile.
 struct EpilogueState {
-  uint32_t g = 0;      // chunks processed so far (staging buffer = g & 1)
-  uint32_t eph = 0;    // phase of the group rendezvous
+  uint32_t g = 0;            // chunks processed so far
+  uint32_t eph = 0;          // phase of the group rendezvous
+  bool d_in_flight = false;  // the D load of chunk g has already been issued (prefetched during chunk g-1)
 };
 
-// Thread = one accumulator row (TMEM lane).  The tile leaves in four 64-column chunks through two
-// 128B-swizzled staging buffers: TMA brings the D chunk in, every thread turns its own row of D into its
-// row of C in place (one bf16 rounding of gamma*(beta*D + alpha*acc)), TMA stores the chunk; a strictly
-// upper tile of a symmetric product is also written transposed with plain stores (64 contiguous bytes per
-// warp instruction).  Returns false when a bounded wait expired.
-__device__ __forceinline__ bool epilogue_tile(const TcArgs& a, const CUtensorMap* map_d, const CUtensorMap* map_c, int mat,
-                                              int m0, int n0, bool mirror, uint32_t taddr, uint32_t epi_base,
-                                              uint32_t dfull_bar0, uint32_t egroup_bar, uint32_t tfull_bar, uint32_t aph,
-                                              volatile int* abort_flag, EpilogueState& st, int quad, int lane) {
+// Thread = one accumulator row (TMEM lane).  The tile leaves in four 64-column chunks through a ring of three
+// 128B-swizzled staging buffers: TMA brings the D chunk in (requested one chunk ahead, across tile boundaries,
+// so its latency hides behind the previous chunk), every thread turns its own row of D into its row of C in
+// place (one bf16 rounding of gamma*(beta*D + alpha*acc)), TMA stores the chunk; a strictly upper tile of a
+// symmetric product is also written transposed with plain stores (64 contiguous bytes per warp instruction).
+// `next` is the tile this CTA processes afterwards (for the prefetch).  Returns false when a bounded wait expired.
+__device__ __forceinline__ bool epilogue_tile(const TcArgs& a, const CUtensorMap* map_d, const CUtensorMap* map_c,
+                                              const EpiTile& cur, const EpiTile& next, bool mirror, uint32_t taddr,
+                                              uint32_t epi_base, uint32_t dfull_bar0, uint32_t egroup_bar, uint32_t tfull_bar,
+                                              uint32_t aph, volatile int* abort_flag, EpilogueState& st, int quad, int lane) {
   const bool leader = quad == 2 && lane == 0;        // warp 2 is the first epilogue warp
   const int lrow = quad * 32 + lane;
   auto group_sync = [&]() -> bool {                  // rendezvous of the four warps on an mbarrier: bounded like every wait
@@ -164,6 +173,7 @@ __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, const CUtensorMap
     st.eph ^= 1u;
     return done;
   };
+  const int mat = cur.mat, m0 = cur.m0, n0 = cur.n0;
   float gamma = 1.f;
   if (a.gamma_mode) {
     const float r = a.rnorm[mat];
@@ -177,14 +187,28 @@ __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, const CUtensorMap
   for (int cb = 0; cb < EPI_TILE_N / EPI_COLS; ++cb, ++st.g) {
     const int c0 = n0 + cb * EPI_COLS;
     if (c0 >= a.n) break;                             // uniform over the group
-    const uint32_t b = st.g & 1u;
+    const uint32_t b = st.g % EPI_BUFS;
     const uint32_t ebuf = epi_base + b * EPI_BYTES;
     const uint32_t dbar = dfull_bar0 + b * 8u;
+    // the chunk after this one: the next chunk of this tile, or the first chunk of the next tile
+    const bool more_here = cb + 1 < EPI_TILE_N / EPI_COLS && c0 + EPI_COLS < a.n;
+    const bool have_next = more_here || next.valid;
     if (leader) {
-      tma_wait_read<1>();                             // the store that last used this buffer has read it
       if (a.d) {
-        mbar_expect_tx(dbar, EPI_BYTES);
-        tma_load_3d(ebuf, map_d, dbar, c0, m0, mat);
+        if (!st.d_in_flight) {                        // only the very first chunk of a CTA is not prefetched
+          tma_wait_read<2>();                         // buffer b was last read by the store of chunk g-3
+          mbar_expect_tx(dbar, EPI_BYTES);
+          tma_load_3d(ebuf, map_d, dbar, c0, m0, mat);
+        }
+        if (have_next) {
+          const uint32_t nb = (st.g + 1) % EPI_BUFS;
+          tma_wait_read<1>();                         // buffer nb was last read by the store of chunk g-2
+          mbar_expect_tx(dfull_bar0 + nb * 8u, EPI_BYTES);
+          if (more_here) tma_load_3d(epi_base + nb * EPI_BYTES, map_d, dfull_bar0 + nb * 8u, c0 + EPI_COLS, m0, mat);
+          else tma_load_3d(epi_base + nb * EPI_BYTES, map_d, dfull_bar0 + nb * 8u, next.n0, next.m0, next.mat);
+        }
+      } else {
+        tma_wait_read<2>();                           // buffer b was last read by the store of chunk g-3
       }
     }
     if (!acc_ready) {
@@ -193,10 +217,11 @@ __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, const CUtensorMap
       acc_ready = true;
     }
     if (a.d) {
-      if (!mbar_wait(dbar, (st.g >> 1) & 1u, abort_flag)) return false;
+      if (!mbar_wait(dbar, (st.g / EPI_BUFS) & 1u, abort_flag)) return false;
     } else {
       if (!group_sync()) return false;                // the leader's wait_group above frees the buffer for everyone
     }
+    st.d_in_flight = a.d && have_next;
     uint32_t v[64];
     tc_ld32(taddr + uint32_t(cb * EPI_COLS), *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
     tc_ld32(taddr + uint32_t(cb * EPI_COLS + 32), *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
