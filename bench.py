@@ -39,9 +39,9 @@ NUM_SHARDS = 8
 
 # DRAM bytes (read + write) of one launch of the Newton-Schulz product kernel: the mean over the three
 # products (G1, G2, G3) captured with ncu on the 4096x14336 group with 3 matrices per launch
-# (0.856 + 0.176 + 1.010 GB in the committed ncu summary of that kernel), scaled by 9/3 to the 9 matrices a
+# (0.856 + 0.173 + 0.984 GB in the committed ncu summary of that kernel), scaled by 9/3 to the 9 matrices a
 # benchmark launch of that group holds (matrices are independent, so traffic grows in proportion).
-NS_KERNEL_DRAM_BYTES_PER_LAUNCH = (0.856e9 + 0.176e9 + 1.010e9) / 3 * (9 / 3)
+NS_KERNEL_DRAM_BYTES_PER_LAUNCH = (0.856e9 + 0.173e9 + 0.984e9) / 3 * (9 / 3)
 
 
 # ----------------------------------------------------------------------------- helpers
