@@ -346,7 +346,7 @@ def run_ours(args, world, rank, local):
     # them, so the algorithmic work of the variant that runs is steps*(3 s^2 l + s^3) per matrix.
     achieved = sym / ns_s_per_step / 1e12
     per_launch_ms = ns_ms / max(1, ns_launches)
-    roofline = {"bound": "tensor", "kernel": "ns_product_tc_kernel", "achieved": achieved, "peak": peaks["bf16_sustained"],
+    roofline = {"bound": "tensor", "kernel": "ns_product_pair_kernel", "achieved": achieved, "peak": peaks["bf16_sustained"],
                 "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"], "traffic": NS_KERNEL_DRAM_BYTES_PER_LAUNCH,
                 "peak_source": f"bf16_tflops_sustained of {peaks['source']} (kernel timed inside a long step)",
                 "flops_per_launch": sym / (ns_launches / args.steps), "ms_per_launch": per_launch_ms,

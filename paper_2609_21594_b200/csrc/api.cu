@@ -278,8 +278,26 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
   if (!ev || cudaEventRecord(ev, st) != cudaSuccess) return MUON_ERR_CUDA;
   if (cudaStreamWaitEvent(ctx->h2d_stream, ev, 0) != cudaSuccess || cudaStreamWaitEvent(ctx->d2h_stream, ev, 0) != cudaSuccess)
     return MUON_ERR_CUDA;
+  // Order of the batches: only the first batch's inbound copy and the last batch's outbound copy are exposed,
+  // so the smallest batch goes first and the second smallest last; the others keep the plan's order.
+  std::vector<size_t> order(plan->chunks.size());
+  for (size_t c = 0; c < order.size(); ++c) order[c] = c;
+  auto elems = [&](size_t c) { return int64_t(plan->chunks[c].count) * plan->chunks[c].s * plan->chunks[c].l; };
+  if (order.size() > 2) {
+    size_t small = 0;
+    for (size_t c = 1; c < order.size(); ++c)
+      if (elems(c) < elems(small)) small = c;
+    order.erase(order.begin() + long(small));
+    size_t second = 0;
+    for (size_t k = 1; k < order.size(); ++k)
+      if (elems(order[k]) < elems(order[second])) second = k;
+    const size_t last = order[second];
+    order.erase(order.begin() + long(second));
+    order.insert(order.begin(), small);
+    order.push_back(last);
+  }
   std::vector<cudaEvent_t> arrived(plan->chunks.size());
-  for (size_t c = 0; c < plan->chunks.size(); ++c) {            // all inbound copies are queued up front, in chunk order
+  for (size_t c : order) {                                       // all inbound copies are queued up front, in batch order
     for (int32_t i : plan->chunks[c].mats)
       for (const muon_segment_t& sg : pipe->layout->segs_of[size_t(i)])
         if (cudaMemcpyAsync(static_cast<char*>(const_cast<void*>(g[i])) + size_t(sg.elem_begin) * es,
@@ -289,7 +307,7 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
     arrived[c] = next_sync_event(ctx);
     if (!arrived[c] || cudaEventRecord(arrived[c], ctx->h2d_stream) != cudaSuccess) return MUON_ERR_CUDA;
   }
-  for (size_t c = 0; c < plan->chunks.size(); ++c) {
+  for (size_t c : order) {
     const Chunk& ch = plan->chunks[c];
     if (cudaStreamWaitEvent(st, arrived[c], 0) != cudaSuccess) return MUON_ERR_CUDA;
     status = run_chunk(ctx, ch, static_cast<const MatDesc*>(d_descs), r, st);
