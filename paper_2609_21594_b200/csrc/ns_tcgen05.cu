@@ -1,22 +1,22 @@
-// Tensor-core Newton-Schulz engine for sm_100a: batched products of Eq. 1 with bf16 operands and
-// fp32 accumulation in tensor memory.
+// Tensor-core Newton-Schulz engine for sm_100a, single-CTA kernel: batched products of Eq. 1 with bf16
+// operands and fp32 accumulation in tensor memory.  It serves matrices of at most 128 rows and is the
+// cross-check of the paired-CTA kernel, which runs everything else.
 //
 //   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k]^T)     nn = 0   (A = X X^T,  B = bA + cA A^T)
 //   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k])       nn = 1   (X' = aX + B X)
 //
 // One persistent CTA per SM, 192 threads, warp-specialised:
 //   warp 0      TMA producer: cp.async.bulk.tensor loads of 128B-swizzled operand tiles into a
-//               4-stage shared-memory ring (one mbarrier pair per stage)
+//               3-stage shared-memory ring of 48 KiB stages (one mbarrier pair per stage)
 //   warp 1      MMA issuer: one thread issues tcgen05.mma (M128 x N256 x K16, kind::f16) on shared-memory
 //               descriptors; accumulators live in TMEM, double-buffered (2 x 256 columns)
-//   warps 2..5  epilogue: tcgen05.ld of the accumulator, fused gamma*(beta*D + alpha*acc), one bf16
-//               rounding, 16-byte global stores; overlaps the next tile's main loop
+//   warps 2..5  epilogue (shared with the paired kernel): tcgen05.ld of the accumulator, D chunk by TMA,
+//               fused gamma*(beta*D + alpha*acc) with one bf16 rounding, TMA store; overlaps the next
+//               tile's main loop
 // P tiles are K-major.  Q tiles are K-major for nn = 0 and MN-major for nn = 1 (X is read as stored,
 // row-major s x l, so no transposed copy of X is ever made).
 // Every wait on an mbarrier is bounded: on expiry the CTA records a code in the context's status
 // word, stops issuing work, waits (bounded) for its own TMA copies, frees its TMEM and returns.
-#include <cstring>
-
 #include "tc_common.cuh"
 
 namespace muon {

@@ -17,8 +17,6 @@
 //   empty[s]   in each CTA; the leader's tcgen05.commit arrives on both (commit multicast).
 //   tfull[a]   in each CTA; commit multicast after a tile's last k-block.
 //   tempty[a]  leader only, 8 arrivals: the four epilogue warps of each CTA (remote arrive).
-#include <cstring>
-
 #include "tc_common.cuh"
 
 namespace muon {
