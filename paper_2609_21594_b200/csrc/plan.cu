@@ -39,15 +39,21 @@ int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t co
   for (const auto& key : order) {
     const std::vector<int32_t>& idx = groups[key];
     const int64_t per = int64_t(key.first) * key.second;
-    const int64_t per_chunk = std::max<int64_t>(1, cap / per);
-    for (size_t b = 0; b < idx.size(); b += size_t(per_chunk)) {
+    // as few chunks as the cap allows, of (nearly) equal size: a short last chunk would run its fifteen
+    // products on a mostly idle device
+    const int64_t max_per_chunk = std::max<int64_t>(1, cap / per);
+    const int64_t num_chunks = (int64_t(idx.size()) + max_per_chunk - 1) / max_per_chunk;
+    const size_t base = idx.size() / size_t(num_chunks), rem = idx.size() % size_t(num_chunks);
+    size_t b = 0;
+    for (int64_t ci = 0; ci < num_chunks; ++ci) {
       Chunk ch;
       ch.s = key.first;
       ch.l = key.second;
       ch.ldx = int32_t(up(size_t(ch.l), 8));
       ch.lda = int32_t(up(size_t(ch.s), 8));
-      const size_t e = std::min(idx.size(), b + size_t(per_chunk));
-      ch.mats.assign(idx.begin() + b, idx.begin() + e);
+      const size_t e = b + base + (size_t(ci) < rem ? 1 : 0);
+      ch.mats.assign(idx.begin() + long(b), idx.begin() + long(e));
+      b = e;
       ch.count = int32_t(ch.mats.size());
       const int32_t ts = (ch.s + kElemTile - 1) / kElemTile, tl = (ch.l + kElemTile - 1) / kElemTile;
       ch.tiles_per_mat = ts * tl;
