@@ -401,3 +401,25 @@ def test_ns_ragged_multi_tile_shapes(engine):
         ref = orc.newton_schulz(v, 5, QUINTIC, 1e-7, "bf16")
         assert rel(o, ref) <= TOL_BF16, (i, shapes[i], rel(o, ref))
     ctx.close()
+
+
+def test_many_small_heterogeneous_matrices():
+    """1500 small matrices of a dozen interleaved shapes (several shape groups, tall and wide mixed in one group,
+    batches far larger than the SM count): every 50th one is checked against the oracle, all must be finite and
+    batched == alone for a few."""
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "bf16", "tensor")
+    base = [(16, 16), (32, 48), (48, 32), (64, 64), (8, 120), (120, 8), (96, 160), (160, 96), (130, 40), (24, 24), (1, 64), (100, 100)]
+    shapes = [base[i % len(base)] for i in range(1500)]
+    mats = [wl.grad_np("swarm", 0, i, s) for i, s in enumerate(shapes)]
+    outs, vals = _ortho(mb, ctx, mats)
+    for o in outs:
+        assert np.isfinite(o).all()
+    for i in range(0, len(shapes), 50):
+        ref = orc.newton_schulz(vals[i], 5, QUINTIC, 1e-7, "bf16")
+        assert rel(outs[i], ref) <= TOL_BF16, (i, shapes[i], rel(outs[i], ref))
+    for i in (3, 700, 1499):
+        alone, _ = _ortho(mb, ctx, [mats[i]])
+        assert np.array_equal(alone[0], outs[i])
+    ctx.close()
