@@ -357,7 +357,8 @@ def run_ours(args, world, rank, local):
         pms, _ = phases[name]
         if pms > 0:
             gbs = n_elem * bytes_per_elem / (pms / 1e3 / args.steps) / 1e9
-            hbm[name] = {"ms_per_step": pms / args.steps, "gbs": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]}
+            hbm[name] = {"ms_per_step": pms / args.steps, "gbs": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
+                         "frac_of_nominal_8000": gbs / 8000.0}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
