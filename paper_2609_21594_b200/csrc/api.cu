@@ -119,7 +119,8 @@ struct ChunkRun {
 };
 
 int run_chunk(muon_ctx* ctx, const Chunk& ch, const MatDesc* d_descs, const ChunkRun& r, cudaStream_t st,
-              const RowSeg* d_segs = nullptr) {
+              const RowSeg* d_segs = nullptr, bool pitch8 = true) {
+  const int32_t wide = (pitch8 && ch.s % 8 == 0 && ch.l % 8 == 0) ? 1 : 0;
   const WsCarve w = carve_chunk(ctx->opt, ch);
   char* base = static_cast<char*>(ctx->ws);
   void* x0 = base + w.x0;
@@ -146,6 +147,7 @@ int run_chunk(muon_ctx* ctx, const Chunk& ch, const MatDesc* d_descs, const Chun
     sa.ns_precision = ctx->opt.ns_precision;
     sa.momentum = r.momentum;
     sa.normalize = r.normalize;
+    sa.wide = wide;
     n = launch_stage(sa, st);
     if (n < 0) return n;
     ctx->launches += n;
@@ -202,6 +204,7 @@ int run_chunk(muon_ctx* ctx, const Chunk& ch, const MatDesc* d_descs, const Chun
     aa.decay = 1.0f - r.lr * r.wd;
     aa.ns_precision = ctx->opt.ns_precision;
     aa.update = r.momentum;
+    aa.wide = wide;
     n = launch_apply(aa, st);
     if (n < 0) return n;
     ctx->launches += n;
@@ -241,6 +244,7 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
   if (plan->live == 0) return MUON_OK;
   if (!ctx->ws || ctx->ws_bytes < plan->ws_bytes) return MUON_ERR_WORKSPACE_TOO_SMALL;
   std::vector<MatDesc> descs(size_t(plan->live));
+  bool pitch8 = true;                                  // every row pitch a multiple of 8 elements
   for (const Chunk& ch : plan->chunks) {
     for (int32_t j = 0; j < ch.count; ++j) {
       const int32_t i = ch.mats[size_t(j)];
@@ -256,6 +260,7 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
       d.cols = shapes[i].cols;
       d.ld = lds ? lds[i] : int64_t(d.cols);
       if (d.ld < d.cols || d.ld > 0x7fffffffLL) return MUON_ERR_INVALID_ARG;
+      if (d.ld % 8) pitch8 = false;
       d.seg_begin = flat ? flat->rowseg_begin[size_t(i)] : 0;
       d.seg_count = flat ? flat->rowseg_count[size_t(i)] : 0;
       d.transposed = d.rows > d.cols ? 1 : 0;
@@ -267,7 +272,7 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
   if (status != MUON_OK) return status;
   if (!pipe) {
     for (const Chunk& ch : plan->chunks) {
-      status = run_chunk(ctx, ch, static_cast<const MatDesc*>(d_descs), r, st, flat ? flat->d_rowsegs : nullptr);
+      status = run_chunk(ctx, ch, static_cast<const MatDesc*>(d_descs), r, st, flat ? flat->d_rowsegs : nullptr, pitch8);
       if (status != MUON_OK) return status;
     }
     return MUON_OK;
@@ -310,7 +315,7 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
   for (size_t c : order) {
     const Chunk& ch = plan->chunks[c];
     if (cudaStreamWaitEvent(st, arrived[c], 0) != cudaSuccess) return MUON_ERR_CUDA;
-    status = run_chunk(ctx, ch, static_cast<const MatDesc*>(d_descs), r, st);
+    status = run_chunk(ctx, ch, static_cast<const MatDesc*>(d_descs), r, st, nullptr, pitch8);
     if (status != MUON_OK) return status;
     cudaEvent_t done = next_sync_event(ctx);
     if (!done || cudaEventRecord(done, st) != cudaSuccess || cudaStreamWaitEvent(ctx->d2h_stream, done, 0) != cudaSuccess)

@@ -6,6 +6,8 @@
 //   apply : W <- W (1 - lr*wd) - lr * 0.2 sqrt(max(m,n)) * O, O read back through the transpose
 // All three are HBM-bound.  Reductions use a fixed shuffle/shared-memory tree and per-tile
 // partial sums, never floating-point atomics, so results are bit-identical run to run.
+#include <algorithm>
+
 #include "internal.h"
 
 namespace muon {
@@ -339,6 +341,194 @@ __global__ void __launch_bounds__(256, FLAT ? 5 : 6) apply_kernel(ApplyArgs a) {
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------------------------
+// "Wide" variants for matrices whose rows, cols and row pitches are all multiples of 8: 64 x 128 tiles, every
+// thread moves 8 consecutive elements per access (16-byte bf16 / 2 x 16-byte fp32 vectors), so the instruction
+// count per byte is about a third of the generic kernels' -- which is what keeps these HBM-bound kernels at
+// bandwidth when the SM clock sits low under the power cap of a Newton-Schulz-heavy step.
+// Transposition goes through a 128 x 64 bf16 shared tile T[c][r] (128 bytes per c-row, no padding) whose
+// 16-byte chunks are XOR-swizzled with bits 3..5 of c: the element-wise side (one c-row per thread column)
+// then spreads over 8 bank groups, the vector side reads/writes whole 16-byte chunks without conflicts.
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int WR = 64, WC = 128;
+
+__device__ __forceinline__ uint32_t wide_tile_addr(int c_local, int r_local) {   // byte offset of T[c][r]
+  return uint32_t(c_local) * 128u + (uint32_t((r_local >> 3) ^ ((c_local >> 3) & 7)) << 4) + uint32_t(r_local & 7) * 2u;
+}
+
+__host__ __device__ inline int wide_tiles(int rows, int cols) { return ((rows + WR - 1) / WR) * ((cols + WC - 1) / WC); }
+
+template <typename GT, bool MOM, bool FLAT>
+__global__ void __launch_bounds__(256) stage_wide_kernel(StageArgs a, int tiles_wide) {
+  __shared__ __align__(16) unsigned char tsm[WC * 128];
+  __shared__ float red[8];
+  const int mat = blockIdx.x / tiles_wide;
+  const int t = blockIdx.x - mat * tiles_wide;
+  const MatDesc d = a.descs[mat];
+  const int tiles_c = (d.cols + WC - 1) / WC;
+  float sum = 0.f;
+  if (t < wide_tiles(d.rows, d.cols)) {                      // block-uniform: the grid is sized for the larger orientation
+    const int r0 = (t / tiles_c) * WR, c0 = (t % tiles_c) * WC;
+    const GT* __restrict__ G = static_cast<const GT*>(d.g);
+    float* __restrict__ M = static_cast<float*>(d.m);
+    __nv_bfloat16* __restrict__ X = static_cast<__nv_bfloat16*>(a.x) + size_t(mat) * a.s * a.ldx;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int c = c0 + 8 * tx;
+    RowCursor<FLAT> cur;
+    cur.init(d, a.segs, min(r0 + ty, d.rows - 1));
+    if (c < d.cols) {
+#pragma unroll
+      for (int pass = 0; pass < 4; ++pass) {
+        const int rl = ty + pass * 16, r = r0 + rl;
+        if (r < d.rows) {
+          const size_t off = cur.at(d, a.segs, r) + size_t(c);
+          float g[8], m[8];
+          if (sizeof(GT) == 2) {
+            const uint4 raw = __ldcs(reinterpret_cast<const uint4*>(G + off));
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              g[2 * i] = __uint_as_float(w[i] << 16);
+              g[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+            }
+          } else {
+            const float4 g0 = __ldcs(reinterpret_cast<const float4*>(G + off));
+            const float4 g1 = __ldcs(reinterpret_cast<const float4*>(G + off) + 1);
+            g[0] = g0.x; g[1] = g0.y; g[2] = g0.z; g[3] = g0.w; g[4] = g1.x; g[5] = g1.y; g[6] = g1.z; g[7] = g1.w;
+          }
+          if (MOM) {
+            const float4 m0 = __ldcs(reinterpret_cast<const float4*>(M + off));
+            const float4 m1 = __ldcs(reinterpret_cast<const float4*>(M + off) + 1);
+            m[0] = m0.x; m[1] = m0.y; m[2] = m0.z; m[3] = m0.w; m[4] = m1.x; m[5] = m1.y; m[6] = m1.z; m[7] = m1.w;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              m[i] = a.mu * m[i] + g[i];
+              g[i] = a.nesterov ? g[i] + a.mu * m[i] : m[i];      // g now holds u
+            }
+            __stcs(reinterpret_cast<float4*>(M + off), make_float4(m[0], m[1], m[2], m[3]));
+            __stcs(reinterpret_cast<float4*>(M + off) + 1, make_float4(m[4], m[5], m[6], m[7]));
+          }
+          uint32_t pk[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 b = __floats2bfloat162_rn(g[2 * i], g[2 * i + 1]);
+            pk[i] = *reinterpret_cast<const uint32_t*>(&b);
+            const float q0 = __uint_as_float(pk[i] << 16), q1 = __uint_as_float(pk[i] & 0xffff0000u);
+            sum += q0 * q0;
+            sum += q1 * q1;
+          }
+          if (!d.transposed) {
+            *reinterpret_cast<uint4*>(X + size_t(r) * a.ldx + c) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const uint16_t h = uint16_t(i & 1 ? pk[i >> 1] >> 16 : pk[i >> 1] & 0xffffu);
+              *reinterpret_cast<uint16_t*>(tsm + wide_tile_addr(8 * tx + i, rl)) = h;
+            }
+          }
+        }
+      }
+    }
+    if (d.transposed) {
+      __syncthreads();
+#pragma unroll
+      for (int pass = 0; pass < 4; ++pass) {                 // X[c][r0 + 8*og .. +7]: one 16-byte chunk per thread
+        const int oc = (threadIdx.x >> 3) + 32 * pass, og = threadIdx.x & 7;
+        const int cc = c0 + oc, r = r0 + 8 * og;
+        if (cc < d.cols && r < d.rows)
+          *reinterpret_cast<uint4*>(X + size_t(cc) * a.ldx + r) = *reinterpret_cast<const uint4*>(tsm + wide_tile_addr(oc, 8 * og));
+      }
+    }
+  }
+  const float tot = block_sum_256(sum, red);
+  if (threadIdx.x == 0) a.partials[blockIdx.x] = tot;
+}
+
+template <bool UPD, bool FLAT>
+__global__ void __launch_bounds__(256) apply_wide_kernel(ApplyArgs a, int tiles_wide) {
+  __shared__ __align__(16) unsigned char tsm[WC * 128];
+  const int mat = blockIdx.x / tiles_wide;
+  const int t = blockIdx.x - mat * tiles_wide;
+  const MatDesc d = a.descs[mat];
+  if (t >= wide_tiles(d.rows, d.cols)) return;               // block-uniform
+  const int tiles_c = (d.cols + WC - 1) / WC;
+  const int r0 = (t / tiles_c) * WR, c0 = (t % tiles_c) * WC;
+  const __nv_bfloat16* __restrict__ X = static_cast<const __nv_bfloat16*>(a.x) + size_t(mat) * a.s * a.ldx;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int c = c0 + 8 * tx;
+  const bool col_ok = c < d.cols;
+  size_t offs[4];
+  {
+    RowCursor<FLAT> cur;
+    cur.init(d, a.segs, min(r0 + ty, d.rows - 1));
+#pragma unroll
+    for (int pass = 0; pass < 4; ++pass) {
+      const int r = r0 + ty + pass * 16;
+      offs[pass] = r < d.rows ? cur.at(d, a.segs, r) + size_t(c) : 0;
+    }
+  }
+  if (d.transposed) {
+#pragma unroll
+    for (int pass = 0; pass < 4; ++pass) {                   // X[c][r0 + 8*og .. +7] -> T[c][.]
+      const int oc = (threadIdx.x >> 3) + 32 * pass, og = threadIdx.x & 7;
+      const int cc = c0 + oc, r = r0 + 8 * og;
+      if (cc < d.cols && r < d.rows)
+        *reinterpret_cast<uint4*>(tsm + wide_tile_addr(oc, 8 * og)) = __ldcs(reinterpret_cast<const uint4*>(X + size_t(cc) * a.ldx + r));
+    }
+    __syncthreads();
+  }
+  const float decay = a.decay;
+  const float step = a.lr * d.scale;
+#pragma unroll
+  for (int pass = 0; pass < 4; ++pass) {
+    const int rl = ty + pass * 16, r = r0 + rl;
+    if (!col_ok || r >= d.rows) continue;
+    uint32_t pk[4];
+    if (!d.transposed) {
+      const uint4 v = __ldcs(reinterpret_cast<const uint4*>(X + size_t(r) * a.ldx + c));
+      pk[0] = v.x; pk[1] = v.y; pk[2] = v.z; pk[3] = v.w;
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t lo = *reinterpret_cast<const uint16_t*>(tsm + wide_tile_addr(8 * tx + 2 * i, rl));
+        const uint32_t hi = *reinterpret_cast<const uint16_t*>(tsm + wide_tile_addr(8 * tx + 2 * i + 1, rl));
+        pk[i] = lo | (hi << 16);
+      }
+    }
+    const size_t off = offs[pass];
+    if (UPD) {
+      float4 w[1][2];
+      {
+        const float* __restrict__ Wr = static_cast<const float*>(d.w);
+        w[0][0] = __ldcs(reinterpret_cast<const float4*>(Wr + off));
+        w[0][1] = __ldcs(reinterpret_cast<const float4*>(Wr + off) + 1);
+      }
+      float o[8];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        o[2 * i] = __uint_as_float(pk[i] << 16);
+        o[2 * i + 1] = __uint_as_float(pk[i] & 0xffff0000u);
+      }
+      float* W = static_cast<float*>(d.w);
+      float4 n0, n1;
+      n0.x = __fmaf_rn(-step, o[0], __fmul_rn(w[0][0].x, decay));
+      n0.y = __fmaf_rn(-step, o[1], __fmul_rn(w[0][0].y, decay));
+      n0.z = __fmaf_rn(-step, o[2], __fmul_rn(w[0][0].z, decay));
+      n0.w = __fmaf_rn(-step, o[3], __fmul_rn(w[0][0].w, decay));
+      n1.x = __fmaf_rn(-step, o[4], __fmul_rn(w[0][1].x, decay));
+      n1.y = __fmaf_rn(-step, o[5], __fmul_rn(w[0][1].y, decay));
+      n1.z = __fmaf_rn(-step, o[6], __fmul_rn(w[0][1].z, decay));
+      n1.w = __fmaf_rn(-step, o[7], __fmul_rn(w[0][1].w, decay));
+      __stcs(reinterpret_cast<float4*>(W + off), n0);
+      __stcs(reinterpret_cast<float4*>(W + off) + 1, n1);
+      if (d.o) __stcs(reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(d.o) + off), make_uint4(pk[0], pk[1], pk[2], pk[3]));
+    } else {
+      *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(d.w) + off) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    }
+  }
+}
+
 }  // namespace
 
 template <bool FLAT>
@@ -356,14 +546,34 @@ static void launch_stage_t(const StageArgs& a, unsigned g, cudaStream_t st) {
   }
 }
 
+template <bool FLAT>
+static void launch_stage_wide_t(const StageArgs& a, unsigned g, int tw, cudaStream_t st) {
+  if (a.momentum) {
+    if (a.grad_dtype == MUON_DTYPE_BF16) stage_wide_kernel<__nv_bfloat16, true, FLAT><<<g, 256, 0, st>>>(a, tw);
+    else stage_wide_kernel<float, true, FLAT><<<g, 256, 0, st>>>(a, tw);
+  } else {
+    stage_wide_kernel<__nv_bfloat16, false, FLAT><<<g, 256, 0, st>>>(a, tw);
+  }
+}
+
+// Tiles per matrix of the wide kernels: a chunk mixes both orientations of its core shape, the grid takes the larger count.
+static int wide_tiles_of_chunk(int s, int l) { return std::max(wide_tiles(s, l), wide_tiles(l, s)); }
+
 int launch_stage(const StageArgs& a, cudaStream_t st) {
-  const int64_t blocks = int64_t(a.count) * a.tiles_per_mat;
+  const bool wide = a.wide && a.ns_precision == MUON_NS_BF16;
+  const int tiles = wide ? wide_tiles_of_chunk(a.s, a.l) : a.tiles_per_mat;
+  const int64_t blocks = int64_t(a.count) * tiles;
   if (blocks == 0) return 0;
   if (blocks > 0x7fffffffLL) return MUON_ERR_UNSUPPORTED;
-  if (a.segs) launch_stage_t<true>(a, unsigned(blocks), st);
-  else launch_stage_t<false>(a, unsigned(blocks), st);
+  if (wide) {
+    if (a.segs) launch_stage_wide_t<true>(a, unsigned(blocks), tiles, st);
+    else launch_stage_wide_t<false>(a, unsigned(blocks), tiles, st);
+  } else {
+    if (a.segs) launch_stage_t<true>(a, unsigned(blocks), st);
+    else launch_stage_t<false>(a, unsigned(blocks), st);
+  }
   if (cudaGetLastError() != cudaSuccess) return MUON_ERR_CUDA;
-  norm_kernel<<<unsigned(a.count), 256, 0, st>>>(a.partials, a.rnorm, a.tiles_per_mat, a.eps, a.normalize);
+  norm_kernel<<<unsigned(a.count), 256, 0, st>>>(a.partials, a.rnorm, tiles, a.eps, a.normalize);
   return cudaGetLastError() == cudaSuccess ? 2 : MUON_ERR_CUDA;
 }
 
@@ -380,11 +590,24 @@ static void launch_apply_t(const ApplyArgs& a, unsigned g, cudaStream_t st) {
 }
 
 int launch_apply(const ApplyArgs& a, cudaStream_t st) {
-  const int64_t blocks = int64_t(a.count) * a.tiles_per_mat;
+  const bool wide = a.wide && a.ns_precision == MUON_NS_BF16;
+  const int tiles = wide ? wide_tiles_of_chunk(a.s, a.l) : a.tiles_per_mat;
+  const int64_t blocks = int64_t(a.count) * tiles;
   if (blocks == 0) return 0;
   if (blocks > 0x7fffffffLL) return MUON_ERR_UNSUPPORTED;
-  if (a.segs) launch_apply_t<true>(a, unsigned(blocks), st);
-  else launch_apply_t<false>(a, unsigned(blocks), st);
+  const unsigned g = unsigned(blocks);
+  if (wide) {
+    if (a.update) {
+      if (a.segs) apply_wide_kernel<true, true><<<g, 256, 0, st>>>(a, tiles);
+      else apply_wide_kernel<true, false><<<g, 256, 0, st>>>(a, tiles);
+    } else {
+      if (a.segs) apply_wide_kernel<false, true><<<g, 256, 0, st>>>(a, tiles);
+      else apply_wide_kernel<false, false><<<g, 256, 0, st>>>(a, tiles);
+    }
+  } else {
+    if (a.segs) launch_apply_t<true>(a, g, st);
+    else launch_apply_t<false>(a, g, st);
+  }
   return cudaGetLastError() == cudaSuccess ? 1 : MUON_ERR_CUDA;
 }
 

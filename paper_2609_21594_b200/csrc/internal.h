@@ -136,6 +136,7 @@ struct StageArgs {
   int32_t nesterov, grad_dtype, ns_precision;
   int32_t momentum;       // 1: full momentum rule; 0: plain staging of the input (orthogonalize)
   int32_t normalize;      // 0: rnorm = 1
+  int32_t wide;           // 1: rows, cols and every row pitch are multiples of 8: the 8-elements-per-thread kernels apply
 };
 int launch_stage(const StageArgs& a, cudaStream_t st);
 
@@ -148,6 +149,7 @@ struct ApplyArgs {
   float decay;            // 1 - lr*wd, computed once on the host so that every update route uses the same value
   int32_t ns_precision;
   int32_t update;         // 1: W <- W(1-lr*wd) - lr*scale*O ; 0: write O into descs[i].w in the NS element type
+  int32_t wide;           // as in StageArgs
 };
 int launch_apply(const ApplyArgs& a, cudaStream_t st);
 
