@@ -360,7 +360,7 @@ __device__ __forceinline__ uint32_t wide_tile_addr(int c_local, int r_local) {  
 __host__ __device__ inline int wide_tiles(int rows, int cols) { return ((rows + WR - 1) / WR) * ((cols + WC - 1) / WC); }
 
 template <typename GT, bool MOM, bool FLAT>
-__global__ void __launch_bounds__(256) stage_wide_kernel(StageArgs a, int tiles_wide) {
+__global__ void __launch_bounds__(256, 6) stage_wide_kernel(StageArgs a, int tiles_wide) {
   __shared__ __align__(16) unsigned char tsm[WC * 128];
   __shared__ float red[8];
   const int mat = blockIdx.x / tiles_wide;
