@@ -423,3 +423,25 @@ def test_many_small_heterogeneous_matrices():
         alone, _ = _ortho(mb, ctx, [mats[i]])
         assert np.array_equal(alone[0], outs[i])
     ctx.close()
+
+
+def test_torch_optimizer_front_end_matches_the_oracle():
+    """The torch.optim wrapper only marshals: two optimizer steps on three parameters equal the oracle's."""
+    from paper_2609_21594_b200.optim import Muon
+
+    shapes = [(256, 384), (384, 256), (128, 128)]
+    params = [torch.nn.Parameter(dev_f32(wl.param_np("optim", i, s))) for i, s in enumerate(shapes)]
+    opt = Muon(params, lr=0.02, momentum=0.95, weight_decay=0.01, ns_precision="fp32")
+    W = [host_f64(p) for p in params]
+    M = [np.zeros(s) for s in shapes]
+    for t in range(2):
+        for i, p in enumerate(params):
+            p.grad = dev_f32(wl.grad_np("optim", t, i, shapes[i]))
+        opt.step()
+        torch.cuda.synchronize()
+        for i, p in enumerate(params):
+            g = wl.grad_np("optim", t, i, shapes[i]).astype(np.float64)
+            Wn, Mn, _ = orc.muon_step(W[i], g, M[i], 0.02, 0.95, 0.01, 5, QUINTIC, 1e-7, True, "fp64")
+            assert rel(host_f64(p) - W[i], Wn - W[i]) <= TOL_FP32
+            assert rel(host_f64(opt.state[p]["momentum_buffer"]), Mn) <= 1e-6
+            W[i], M[i] = host_f64(p), host_f64(opt.state[p]["momentum_buffer"])
