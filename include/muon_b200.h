@@ -66,10 +66,10 @@ typedef struct muon_layout muon_layout_t;
 /* Shape of one dense row-major matrix (Section 2.3: W in R^{m x n}). */
 typedef struct { int32_t rows, cols; } muon_shape_t;
 
-/* A logical matrix inside a larger physical parameter (Section 6.3, "the matrix as Muon sees it":
- * one physical parameter can hold several logical matrices -- the heads of a fused QKV projection, the
- * gate and up halves of an MoE FC1 weight, the factors of an MLA projection, the E planes of an
- * [E, M, N] expert tensor).  rows x cols elements, row r starting ld elements after row r-1. */
+/* A logical matrix inside a larger physical parameter (the logical-matrix adapter of Section 6.3:
+ * storage layout and the matrices the optimizer works on are separate things, e.g. the heads of a
+ * fused QKV projection, the gate and up halves of an MoE FC1 weight, the factors of an MLA
+ * projection, the E planes of an [E, M, N] expert tensor).  rows x cols elements, row r starting ld elements after row r-1. */
 typedef struct { int32_t rows, cols; int64_t ld; } muon_view_t;
 
 /* One contiguous piece of a matrix inside the flat buffer: elements
@@ -83,8 +83,8 @@ typedef struct {
   int64_t flat_offset;
 } muon_segment_t;
 
-/* Flat FSDP-style shard buffer (Sections 5.2-5.3 buffer conventions, Section 6.2 step 1:
- * "aligned staging buffer (bf16, uneven splits supported)"): num_shards consecutive
+/* Flat FSDP-style shard buffer (buffer conventions of Sections 5.2-5.3; the staging buffer of the
+ * fused gather in Section 6.2 step 1, which is aligned, bf16 and may be split unevenly): num_shards consecutive
  * shards of shard_len elements each; segment starts are multiples of align_elems;
  * everything not covered by a segment is padding that is never read nor written. */
 typedef struct {
@@ -118,8 +118,8 @@ int  muon_create(muon_ctx_t** ctx, const muon_options_t* opt);
 void muon_destroy(muon_ctx_t* ctx);
 
 /* Bytes of device workspace that muon_step_batched / muon_orthogonalize_batched need for
- * this list of shapes under these options ("workspace allocated once per batched
- * invocation", Section 6.3).  Pure host arithmetic; needs no device. */
+ * this list of shapes under these options (one workspace per batched invocation rather than
+ * per matrix, Section 6.3).  Pure host arithmetic; needs no device. */
 int muon_workspace_bytes(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count, size_t* bytes);
 
 /* Hands the library a caller-owned device buffer (256-byte aligned) used as workspace by
@@ -158,7 +158,7 @@ int muon_scatter(muon_ctx_t* ctx, void* flat_buf, const muon_layout_t* layout,
                  const void* const* matrices, void* stream);
 
 /* muon_step_batched: one Muon update of `count` independent matrices (Section 2.3, Eq. 1;
- * Algorithm 2 "momentum update -> batched NS -> apply"):
+ * the complete-matrix path of Algorithm 2: momentum, batched Newton-Schulz, apply):
  *     M <- mu*M + G;  u = G + mu*M (Nesterov) or M;  U = cast(u)
  *     X_0 = U / (||U||_F + eps), run on U^T when rows > cols (transpose-first, Section 6.3)
  *     X_{k+1} = a_k X_k + (b_k A + c_k A^2) X_k,  A = X_k X_k^T,  k = 0..ns_steps-1
@@ -193,8 +193,8 @@ int muon_step_batched_views(muon_ctx_t* ctx, void* const* params, const void* co
                             float wd, int32_t ns_steps, const float* coeffs, void* stream);
 
 /* muon_step_flat: the sharded-state flow of Section 6.2 on one device -- parameters, momenta and
- * gradients STAY in flat shard buffers that share one layout ("momentum stays sharded throughout, so
- * optimizer-state memory never reflows"; "each rank extracts its own slice and applies the update").
+ * gradients STAY in flat shard buffers that share one layout (in the paper the momentum is never
+ * un-sharded, and every rank applies the update to its own slice of the parameters).
  * The momentum rule reads and writes the flat momentum shards in place and stages the cast result
  * straight into the Newton-Schulz workspace (the gather is fused away); the update is applied straight
  * onto the flat fp32 parameter shards and, when flat_updates is given, O is written straight into it

@@ -13,8 +13,8 @@ products themselves still accumulated in float64.
 
 Parity status: every function here is pinned by tests that do not re-use its own
 formulae (SVD closed form, scalar recurrences, brute-force index maps, invariants),
-except the per-step coefficient variant the paper calls its default ("asymmetric
-five-step"): the paper prints no values for it, so that variant is *parity
+except the per-step coefficient variant the paper names as its default (an asymmetric
+five-step set): the paper prints no values for it, so that variant is *parity
 unpinned* beyond the generic per-step-coefficient plumbing.
 
 Notation follows the paper: W (m x n) weight, G gradient, M momentum, X_k the NS

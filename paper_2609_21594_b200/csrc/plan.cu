@@ -14,7 +14,7 @@ size_t elem_bytes_of_ns(int ns_precision) { return ns_precision == MUON_NS_FP32 
 // Matrices sharing a core shape (s, l) form one group (tensors of shape [A,B], [A,1,B], [N,A,B]
 // share the (A,B) group, Section 6.3); a tall matrix joins the group of its transpose because the
 // iteration runs on the transpose anyway.  Each group is cut into chunks of at most chunk_elems
-// elements ("memory-safe batching capped at 2^29 elements"), never fewer than one matrix.
+// elements (the 2^29-element batching cap of Section 6.3), never fewer than one matrix.
 int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t count, Plan* plan) {
   plan->chunks.clear();
   plan->ws_bytes = 0;

@@ -347,7 +347,7 @@ def test_step_out_and_flat_host_path_match_the_plain_step():
 
 @pytest.mark.parametrize("engine", ENGINES)
 def test_per_step_coefficient_sets_on_the_bf16_engines(engine):
-    """A different (a_k, b_k, c_k) at every step -- the form the paper's default 'asymmetric five-step' variant
+    """A different (a_k, b_k, c_k) at every step -- the form the paper's default (asymmetric, five-step) variant
     takes (its values are not printed, so arbitrary per-step triples stand in)."""
     from paper_2609_21594_b200 import binding as mb
 
