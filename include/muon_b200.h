@@ -50,7 +50,7 @@ extern "C" {
 #define MUON_DTYPE_BF16 0
 #define MUON_DTYPE_FP32 1
 
-#define MUON_NS_BF16 0   /* bf16 operands, fp32 accumulation on the tensor cores (Section 6.3: "bf16 arithmetic") */
+#define MUON_NS_BF16 0   /* bf16 operands, fp32 accumulation on the tensor cores (Section 6.6: "bf16 arithmetic") */
 #define MUON_NS_FP32 1   /* every product and intermediate in fp32 (no counterpart in the paper; accuracy anchor)  */
 
 #define MUON_ENGINE_TENSOR      0   /* tensor cores; CTA pairs (cta_group::2) wherever a matrix has more than 128 rows */
@@ -66,10 +66,10 @@ typedef struct muon_layout muon_layout_t;
 /* Shape of one dense row-major matrix (Section 2.3: W in R^{m x n}). */
 typedef struct { int32_t rows, cols; } muon_shape_t;
 
-/* A logical matrix inside a larger physical parameter (the logical-matrix adapter of Section 6.3:
+/* A logical matrix inside a larger physical parameter (the model adapter of Section 6.6:
  * storage layout and the matrices the optimizer works on are separate things, e.g. the heads of a
  * fused QKV projection, the gate and up halves of an MoE FC1 weight, the factors of an MLA
- * projection, the E planes of an [E, M, N] expert tensor).  rows x cols elements, row r starting ld elements after row r-1. */
+ * projection, the E planes of an [E, M, N] expert tensor, which Section 6.3 says are E separate matrices).  rows x cols elements, row r starting ld elements after row r-1. */
 typedef struct { int32_t rows, cols; int64_t ld; } muon_view_t;
 
 /* One contiguous piece of a matrix inside the flat buffer: elements
@@ -83,8 +83,8 @@ typedef struct {
   int64_t flat_offset;
 } muon_segment_t;
 
-/* Flat FSDP-style shard buffer (buffer conventions of Sections 5.2-5.3; the staging buffer of the
- * fused gather in Section 6.2 step 1, which is aligned, bf16 and may be split unevenly): num_shards consecutive
+/* Flat FSDP-style shard buffer (the aligned, padded fused buffer of Section 5.2; the staging buffer of the
+ * fused gather, Section 6.4 step 1, which is aligned, bf16 and may be split unevenly): num_shards consecutive
  * shards of shard_len elements each; segment starts are multiples of align_elems;
  * everything not covered by a segment is padding that is never read nor written. */
 typedef struct {
@@ -101,12 +101,12 @@ typedef struct {
 typedef struct {
   int32_t grad_dtype;      /* MUON_DTYPE_BF16 | MUON_DTYPE_FP32: element type of `grads`                     */
   int32_t ns_precision;    /* MUON_NS_BF16 | MUON_NS_FP32                                                    */
-  int32_t nesterov;        /* 1: u = G + mu*M' (Section 7 set-up), 0: u = M'                                 */
+  int32_t nesterov;        /* 1: u = G + mu*M' (Section 7.4 set-up), 0: u = M'                                 */
   int32_t coeffs_per_step; /* 0: coeffs[3] used at every step; 1: coeffs[3*ns_steps], (a_k,b_k,c_k) per step */
   float   eps;             /* epsilon of Eq. 1, added to the Frobenius norm; default 1e-7                    */
   int32_t engine;          /* MUON_ENGINE_TENSOR (default) | MUON_ENGINE_TENSOR_1CTA | MUON_ENGINE_CUDA_CORE (bf16  */
                            /* products on CUDA cores; slow cross-check); fp32 NS always runs on CUDA cores          */
-  int64_t chunk_elems;     /* batching cap in elements per batched NS invocation; default 1<<29 (Section 6.3) */
+  int64_t chunk_elems;     /* batching cap in elements per batched NS invocation; default 1<<29 (Section 6.6) */
 } muon_options_t;
 
 /* Fills *opt with the defaults: bf16 grads, bf16 NS, Nesterov, constant coefficients, eps 1e-7, cap 2^29. */
@@ -119,7 +119,7 @@ void muon_destroy(muon_ctx_t* ctx);
 
 /* Bytes of device workspace that muon_step_batched / muon_orthogonalize_batched need for
  * this list of shapes under these options (one workspace per batched invocation rather than
- * per matrix, Section 6.3).  Pure host arithmetic; needs no device. */
+ * per matrix, Section 6.6).  Pure host arithmetic; needs no device. */
 int muon_workspace_bytes(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count, size_t* bytes);
 
 /* Hands the library a caller-owned device buffer (256-byte aligned) used as workspace by
@@ -127,7 +127,7 @@ int muon_workspace_bytes(const muon_options_t* opt, const muon_shape_t* shapes, 
 int muon_set_workspace(muon_ctx_t* ctx, void* dev_ptr, size_t bytes);
 
 /* Host-only description of how a shape list is batched: matrices are grouped by core
- * shape (min(m,n), max(m,n)) -- the paper's shape-fused batching, Section 6.3 -- and each
+ * shape (min(m,n), max(m,n)) -- the paper's shape-fused batching, Section 6.6 -- and each
  * group is cut into chunks of at most chunk_elems elements (at least one matrix).
  * chunk_of[i] receives the chunk index of matrix i (may be NULL); *num_chunks the count. */
 int muon_plan_describe(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count,
@@ -144,7 +144,7 @@ int  muon_layout_create(muon_ctx_t* ctx, const muon_layout_desc_t* desc, muon_la
 void muon_layout_destroy(muon_layout_t* layout);
 
 /* muon_materialize: unpack the flat shard buffer into whole matrices -- the copy-out half
- * of a fused gather (Section 6.2 step 1; the pack/unpack passes of Section 5.2).
+ * of a fused gather (Section 6.4 step 1; the copy-in / copy-out passes of Section 5.1).
  *   flat_buf : device, num_shards*shard_len elements of elem_size bytes, 16-byte aligned
  *   matrices : host array [num_matrices] of device pointers, each rows*cols elements
  * Bit-exact byte movement; padding is never read. */
@@ -152,7 +152,7 @@ int muon_materialize(muon_ctx_t* ctx, const void* flat_buf, const muon_layout_t*
                      void* const* matrices, void* stream);
 
 /* muon_scatter: the inverse -- pack whole matrices into the flat shard buffer (the pack
- * before the relay broadcast, Section 6.2 step 3).  Padding elements of flat_buf are
+ * before the relay broadcast, Section 6.4 step 3).  Padding elements of flat_buf are
  * never written. */
 int muon_scatter(muon_ctx_t* ctx, void* flat_buf, const muon_layout_t* layout,
                  const void* const* matrices, void* stream);
@@ -160,7 +160,7 @@ int muon_scatter(muon_ctx_t* ctx, void* flat_buf, const muon_layout_t* layout,
 /* muon_step_batched: one Muon update of `count` independent matrices (Section 2.3, Eq. 1;
  * the complete-matrix path of Algorithm 2: momentum, batched Newton-Schulz, apply):
  *     M <- mu*M + G;  u = G + mu*M (Nesterov) or M;  U = cast(u)
- *     X_0 = U / (||U||_F + eps), run on U^T when rows > cols (transpose-first, Section 6.3)
+ *     X_0 = U / (||U||_F + eps), run on U^T when rows > cols (transpose-first, Section 6.6)
  *     X_{k+1} = a_k X_k + (b_k A + c_k A^2) X_k,  A = X_k X_k^T,  k = 0..ns_steps-1
  *     W <- W (1 - lr*wd) - lr * 0.2 sqrt(max(rows, cols)) * X_ns
  *   params, momenta : host arrays [count] of device pointers to fp32 matrices (in/out)
@@ -175,7 +175,7 @@ int muon_step_batched(muon_ctx_t* ctx, void* const* params, const void* const* g
 
 /* muon_step_batched_out: muon_step_batched that additionally writes each matrix's orthogonalised
  * update O = X_ns (shape rows x cols, element type of the NS precision) to updates[i] -- the payload
- * owners pack for the relay broadcast (Section 6.2 step 3).  updates may be NULL (then identical to
+ * owners pack for the relay broadcast (Section 6.4 step 3).  updates may be NULL (then identical to
  * muon_step_batched); otherwise a host array [count] of 16-byte-aligned device pointers. */
 int muon_step_batched_out(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
                           void* const* updates, const muon_shape_t* shapes, int32_t count, float lr, float mu,
@@ -183,7 +183,7 @@ int muon_step_batched_out(muon_ctx_t* ctx, void* const* params, const void* cons
 
 /* muon_step_batched_views: muon_step_batched_out on strided views, so that logical matrices are
  * updated in place inside their physical parameters without split/concatenate copies and without a
- * restore pass (the zero-copy view and the restore mapping of the model adapter, Section 6.3).
+ * restore pass (the zero-copy view and the restore mapping of the model adapter, Section 6.6).
  * params[i], grads[i], momenta[i] and, when given, updates[i] point at element (0,0) of view i inside
  * tensors that share the physical layout; all use views[i].ld as row stride (ld >= cols).  Pointers must
  * be 16-byte aligned; the vectorised path also needs ld to be a multiple of 4 elements (other strides
@@ -192,7 +192,7 @@ int muon_step_batched_views(muon_ctx_t* ctx, void* const* params, const void* co
                             void* const* updates, const muon_view_t* views, int32_t count, float lr, float mu,
                             float wd, int32_t ns_steps, const float* coeffs, void* stream);
 
-/* muon_step_flat: the sharded-state flow of Section 6.2 on one device -- parameters, momenta and
+/* muon_step_flat: the sharded-state flow of Section 6.4 (steps 1 and 4) on one device -- parameters, momenta and
  * gradients STAY in flat shard buffers that share one layout (in the paper the momentum is never
  * un-sharded, and every rank applies the update to its own slice of the parameters).
  * The momentum rule reads and writes the flat momentum shards in place and stages the cast result
@@ -213,7 +213,7 @@ int muon_step_flat(muon_ctx_t* ctx, const muon_layout_t* layout, void* flat_para
  * host_flat_grads / host_flat_updates are host buffers of num_shards*shard_len elements in the
  * layout's format (pinned memory makes the copies asynchronous).  Per batch of matrices (the chunks of
  * muon_plan_describe) the gradient segments are copied by DMA straight into grads[] -- the copy engine
- * performs the gather of Section 6.2 step 1 -- the batch is updated as in muon_step_batched_out, and
+ * performs the gather of Section 6.4 step 1 -- the batch is updated as in muon_step_batched_out, and
  * its update segments are copied from updates[] straight into host_flat_updates (the pack of step 3).
  * Inbound copies of later batches and outbound copies of earlier ones overlap the Newton-Schulz work
  * on two internal copy streams; padding of host_flat_updates is never written.

@@ -57,7 +57,7 @@ def _round(x: np.ndarray, mode: str) -> np.ndarray:
     raise ValueError(f"unknown mode {mode!r}")
 
 
-# --------------------------------------------------------------------------- flat-shard layout (Sections 5.2-5.3, 6.2)
+# --------------------------------------------------------------------------- flat-shard layout (Sections 5.1-5.2, 6.4)
 # A layout is: shapes [(m, n)], and segments [(matrix, elem_begin, elem_count, flat_offset)].
 # Segment k says: elements [elem_begin, elem_begin + elem_count) of the row-major
 # linearisation of matrix `matrix` live at flat[flat_offset : flat_offset + elem_count].
@@ -102,7 +102,7 @@ def layout_is_valid(flat_len: int, shapes: Sequence[Tuple[int, int]], segments, 
     return all((c == 1).all() for c in cover) and (used <= 1).all()
 
 
-# --------------------------------------------------------------------------- momentum (Section 2.3; Section 7 set-up: momentum 0.95, Nesterov)
+# --------------------------------------------------------------------------- momentum (Section 2.3; Section 7.4 set-up: momentum 0.95, Nesterov)
 
 
 def momentum_nesterov(G: np.ndarray, M: np.ndarray, mu: float, nesterov: bool = True) -> Tuple[np.ndarray, np.ndarray]:
@@ -114,7 +114,7 @@ def momentum_nesterov(G: np.ndarray, M: np.ndarray, mu: float, nesterov: bool = 
     return M_new, u
 
 
-# --------------------------------------------------------------------------- Newton-Schulz (Eq. 1, Section 6.3)
+# --------------------------------------------------------------------------- Newton-Schulz (Eq. 1, Section 6.6)
 
 
 def _coeff(coeffs: Sequence[float], k: int) -> Tuple[float, float, float]:
@@ -128,7 +128,7 @@ def newton_schulz(U: np.ndarray, steps: int, coeffs: Sequence[float], eps: float
                   trace: list | None = None) -> np.ndarray:
     """Orthogonalise U by `steps` iterations of Eq. 1, X_0 = U / (||U||_F + eps).
 
-    Transpose-first rule (Section 6.3): when rows > cols the iteration runs on U^T so the
+    Transpose-first rule (Section 6.6): when rows > cols the iteration runs on U^T so the
     Gram factor A = X X^T is the small square; the result is transposed back.
 
     Rounding schedule in "bf16" mode ("cast then fold"): U is taken as given (already
@@ -178,7 +178,7 @@ def update_scale(rows: int, cols: int) -> float:
 
 
 def apply_update(W: np.ndarray, O: np.ndarray, lr: float, wd: float) -> np.ndarray:
-    """W' = W (1 - lr*wd) - lr * 0.2 sqrt(max(m,n)) * O: decoupled decay acts on the old W (Sections 6.1-6.2)."""
+    """W' = W (1 - lr*wd) - lr * 0.2 sqrt(max(m,n)) * O: decoupled decay acts on the old W (Section 6.3, Section 6.4 step 4)."""
     W = np.asarray(W, dtype=np.float64)
     rows, cols = W.shape
     return W * (1.0 - lr * wd) - lr * update_scale(rows, cols) * np.asarray(O, dtype=np.float64)
@@ -190,7 +190,7 @@ def muon_step(W: np.ndarray, G: np.ndarray, M: np.ndarray, lr: float, mu: float,
 
     The optimizer state is fp32: M' and W' are rounded to float32 when stored, and in
     "bf16" mode the staged u is cast fp32 -> bf16 before orthogonalisation (the cast the
-    fused gather performs on momentum shards, Section 6.2).
+    fused gather performs on momentum shards, Section 6.4 step 1).
     """
     M_new, u = momentum_nesterov(G, M, mu, nesterov)
     M_store = M_new.astype(np.float32).astype(np.float64)
@@ -201,17 +201,3 @@ def muon_step(W: np.ndarray, G: np.ndarray, M: np.ndarray, lr: float, mu: float,
     O = newton_schulz(U, steps, coeffs, eps, mode)
     W_new = apply_update(W, O, lr, wd).astype(np.float32).astype(np.float64)
     return W_new, M_store, O
-
-
-def muon_steps_batched(Ws, Gs_per_step, Ms, lr, mu, wd, steps, coeffs, eps=1e-7, nesterov=True, mode="fp64"):
-    """Consecutive optimizer steps over a list of matrices.  Gs_per_step[t][i] is the gradient of
-    matrix i at step t.  Matrices are independent; state is carried step to step as fp32."""
-    Ws = [np.asarray(w, dtype=np.float64) for w in Ws]
-    Ms = [np.asarray(m, dtype=np.float64) for m in Ms]
-    Os = []
-    for Gs in Gs_per_step:
-        Os = []
-        for i in range(len(Ws)):
-            Ws[i], Ms[i], O = muon_step(Ws[i], Gs[i], Ms[i], lr, mu, wd, steps, coeffs, eps, nesterov, mode)
-            Os.append(O)
-    return Ws, Ms, Os

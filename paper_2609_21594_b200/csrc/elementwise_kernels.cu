@@ -1,7 +1,7 @@
 // Fused elementwise kernels around the Newton-Schulz engine.
 //   stage : M <- mu*M + G, u = G + mu*M (Nesterov), U = cast(u) written into the NS workspace in
 //           wide orientation (transposed through shared memory when rows > cols: the
-//           transpose-first rule of Section 6.3), plus per-tile sums of U^2
+//           transpose-first rule of Section 6.6), plus per-tile sums of U^2
 //   norm  : r = 1 / (sqrt(sum U^2) + eps) per matrix, fixed-order reduction (Eq. 1, second line)
 //   apply : W <- W (1 - lr*wd) - lr * 0.2 sqrt(max(m,n)) * O, O read back through the transpose
 // All three are HBM-bound.  Reductions use a fixed shuffle/shared-memory tree and per-tile

@@ -1,6 +1,6 @@
 // Flat-shard gather/scatter: pure byte movement between the padded 1-D shard buffer and whole
 // row-major matrices (the unpack after a fused gather and the pack before the relay broadcast,
-// Section 6.2 steps 1 and 3).  HBM-bound; 16-byte vector loads/stores whenever both sides of a
+// Section 6.4 steps 1 and 3).  HBM-bound; 16-byte vector loads/stores whenever both sides of a
 // work item can be brought to a common 16-byte phase, element-wise otherwise.
 #include "internal.h"
 

@@ -1,4 +1,4 @@
-// Host-side planning: shape-fused batching (Section 6.3), workspace carving, layout validation.
+// Host-side planning: shape-fused batching (Section 6.6), workspace carving, layout validation.
 #include <algorithm>
 #include <map>
 #include <numeric>
@@ -12,9 +12,9 @@ static inline size_t up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 size_t elem_bytes_of_ns(int ns_precision) { return ns_precision == MUON_NS_FP32 ? 4 : 2; }
 
 // Matrices sharing a core shape (s, l) form one group (tensors of shape [A,B], [A,1,B], [N,A,B]
-// share the (A,B) group, Section 6.3); a tall matrix joins the group of its transpose because the
+// share the (A,B) group, Section 6.6); a tall matrix joins the group of its transpose because the
 // iteration runs on the transpose anyway.  Each group is cut into chunks of at most chunk_elems
-// elements (the 2^29-element batching cap of Section 6.3), never fewer than one matrix.
+// elements (the 2^29-element batching cap of Section 6.6), never fewer than one matrix.
 int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t count, Plan* plan) {
   plan->chunks.clear();
   plan->ws_bytes = 0;

@@ -18,8 +18,8 @@ import numpy as np
 
 Shape = Tuple[int, int]
 
-QUINTIC = (3.4445, -4.7750, 2.0315)   # legacy constant-coefficient quintic (Section 6.3 names it, prints no values)
-NS_STEPS = 5                          # "five NS iterations" (Section 7, Muon comparison set-up)
+QUINTIC = (3.4445, -4.7750, 2.0315)   # legacy constant-coefficient quintic (Section 6.6 names it, prints no values)
+NS_STEPS = 5                          # "five NS iterations" (Section 7.4, Muon comparison set-up)
 ALIGN_ELEMS = 128                     # pad alignment of every segment start, in elements
 
 
@@ -101,7 +101,7 @@ def _up(x: int, a: int) -> int:
 
 
 def layout_per_param(shapes: Sequence[Shape], num_shards: int, align: int = ALIGN_ELEMS) -> Layout:
-    """Per-parameter ceil-chunk row split (the uneven-split rule of Sections 4.5 / 5.5).
+    """Per-parameter ceil-chunk row split (the uneven ceil-chunk sharding of Sections 4.4 and 5.5).
 
     Shard r holds rows [r*ceil(m/S), min(m, (r+1)*ceil(m/S))) of every matrix; inside a
     shard the pieces are packed in matrix order, each start aligned up to `align`

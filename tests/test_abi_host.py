@@ -98,6 +98,12 @@ def test_layout_validate_rejects_malformed_layouts_like_the_bruteforce_checker()
     strad = wl.Layout(lay.shapes, 2, lay.shard_len, 8, (wl.Segment(0, 0, 256, 0),))
     if strad.shard_len < 256:
         assert mb.muon_layout_validate(mb.make_layout_desc(strad, 2)) == mb.ERR_BAD_LAYOUT
+    # the same hand-built table the oracle's own pin uses: 1 x 12 matrix, two shards of 8, one piece at offset 4
+    one_piece = wl.Layout(((1, 12),), 2, 8, 4, (wl.Segment(0, 0, 12, 4),))
+    cut = wl.Layout(((1, 12),), 2, 8, 4, (wl.Segment(0, 0, 4, 4), wl.Segment(0, 4, 8, 8)))
+    assert mb.muon_layout_validate(mb.make_layout_desc(one_piece, 2)) == mb.ERR_BAD_LAYOUT
+    assert mb.muon_layout_validate(mb.make_layout_desc(cut, 2)) == mb.OK
+    assert mb.muon_layout_validate(mb.make_layout_desc(wl.Layout(((1, 12),), 1, 16, 4, (wl.Segment(0, 0, 12, 4),)), 2)) == mb.OK
     d = mb.make_layout_desc(base, 3)
     assert mb.muon_layout_validate(d) == mb.ERR_INVALID_ARG      # element size must be 2 or 4
     d = mb.make_layout_desc(base, 2)

@@ -62,7 +62,7 @@ def test_ns_bf16_tiny_config_vs_oracle(engine):
         ref = orc.newton_schulz(v, 5, QUINTIC, 1e-7, "bf16")
         assert rel(o, ref) <= TOL_BF16, (i, shapes[i], rel(o, ref))
         hi = orc.newton_schulz(v, 5, QUINTIC, 1e-7, "fp64")
-        assert rel(o, hi) <= 1.5 * rel(ref, hi) + 2e-3
+        assert rel(o, hi) <= 1.5 * rel(ref, hi)       # the device is as far from the exact result as the bf16 oracle is
     ctx.close()
 
 
@@ -181,6 +181,24 @@ def test_batched_equals_alone_and_rerun_bit_exact(engine):
     ctx2.close()
 
 
+def test_batched_equals_alone_at_full_size_shapes():
+    """Bit-exact "batched == alone" where a persistent CTA pair walks many tiles of several matrices:
+    two 4096 x 4096 and two 1408 x 2048 matrices (and the tall orientation of the latter)."""
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "bf16", "tensor")
+    shapes = [(4096, 4096), (1408, 2048), (4096, 4096), (2048, 1408), (1408, 2048)]
+    mats = [wl.grad_np("batchbig", 0, i, s, row_scaled=(s[0] == 4096)) for i, s in enumerate(shapes)]
+    together, vals = _ortho(mb, ctx, mats)
+    for i in (0, 1, 3):
+        alone, _ = _ortho(mb, ctx, [mats[i]])
+        assert np.array_equal(alone[0], together[i]), i
+    # and one of them against the oracle, so that "identical" is also "right"
+    ref = orc.newton_schulz(vals[1], 5, QUINTIC, 1e-7, "bf16")
+    assert rel(together[1], ref) <= TOL_BF16
+    ctx.close()
+
+
 # ----------------------------------------------------------------------------- the full step
 def _run_steps(mb, ctx, config, shapes, n_steps, grad_bf16, row_scaled=False, lr=0.02, mu=0.95, wd=0.01):
     Ws = [wl.param_np(config, i, s) for i, s in enumerate(shapes)]
@@ -263,6 +281,43 @@ def test_update_limits_and_snapshot_resume():
     run((2, 3), Wc, Mc)
     for a, c in zip(Wa + Ma, Wc + Mc):
         assert torch.equal(a, c)
+    ctx.close()
+
+
+@pytest.mark.parametrize("engine", ["tensor", "cuda_core"])
+def test_zero_gradient_through_the_full_step(engine):
+    """G = 0 with M = 0: r = 1/eps = 1e7 is folded into the first epilogues and must multiply exact zeros.
+    The step then reduces to W' = W (1 - lr wd), M' = mu M = 0, with no NaN or Inf anywhere; with a non-zero
+    momentum and G = 0 the update follows the oracle like any other input."""
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "bf16", engine, "bf16")
+    shapes = [(256, 256), (384, 128), (64, 200)]
+    ctx.ensure_workspace(shapes)
+    lr, mu, wd = 0.02, 0.95, 0.01
+    W_np = [wl.param_np("zerog", i, s) for i, s in enumerate(shapes)]
+    Ws = [dev_f32(w) for w in W_np]
+    Ms = [torch.zeros(s, dtype=torch.float32, device="cuda") for s in shapes]
+    Gs = [torch.zeros(s, dtype=torch.bfloat16, device="cuda") for s in shapes]
+    Os = [torch.full(s, float("nan"), dtype=torch.bfloat16, device="cuda") for s in shapes]
+    ctx.muon_step_batched_out(Ws, Gs, Ms, Os, shapes, lr, mu, wd, 5, QUINTIC)
+    torch.cuda.synchronize()
+    assert ctx.muon_last_device_status() == 0
+    decay = np.float32(1.0) - np.float32(lr) * np.float32(wd)
+    for w, w0, m, o in zip(Ws, W_np, Ms, Os):
+        assert torch.count_nonzero(m).item() == 0 and torch.count_nonzero(o.float()).item() == 0
+        assert np.array_equal(w.cpu().numpy(), w0 * decay)       # one fp32 product per element, nothing else
+    # zero gradient on top of a live momentum: u = mu * M' is not zero, the oracle decides
+    M_np = [wl.grad_np("zerog", 1, i, s) for i, s in enumerate(shapes)]
+    Ms = [dev_f32(m) for m in M_np]
+    Ws = [dev_f32(w) for w in W_np]
+    ctx.muon_step_batched(Ws, Gs, Ms, shapes, lr, mu, wd, 5, QUINTIC)
+    torch.cuda.synchronize()
+    for i, s in enumerate(shapes):
+        Wn, Mn, _ = orc.muon_step(W_np[i].astype(np.float64), np.zeros(s), M_np[i].astype(np.float64), lr, mu, wd, 5,
+                                  QUINTIC, 1e-7, True, "bf16")
+        assert rel(host_f64(Ms[i]), Mn) <= 1e-6
+        assert rel(host_f64(Ws[i]) - W_np[i], Wn - W_np[i]) <= TOL_BF16, i
     ctx.close()
 
 

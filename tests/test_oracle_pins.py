@@ -131,6 +131,25 @@ def test_layout_validity_rejects_broken_tables():
     assert not orc.layout_is_valid(lay.flat_len, shapes, bad, 8, 2, lay.shard_len)               # misaligned
 
 
+def test_layout_validity_shard_straddle_rule_by_hand():
+    """A segment must lie inside one shard.  Hand-built table: one 1 x 12 matrix in a flat buffer of two shards
+    of 8 elements.  Stored as one piece at offset 4 it covers flat[4:16] and crosses the boundary at 8: invalid.
+    Cut at the boundary (4 elements in shard 0, 8 in shard 1) the same bytes are a valid layout, and the gather
+    of the split table returns exactly the elements the straddling table would have named."""
+    shapes = [(1, 12)]
+    whole = [(0, 0, 12, 4)]
+    split = [(0, 0, 4, 4), (0, 4, 8, 8)]
+    assert not orc.layout_is_valid(16, shapes, whole, 4, 2, 8)
+    assert orc.layout_is_valid(16, shapes, split, 4, 2, 8)
+    # with a single shard of 16 nothing is crossed, so the one-piece table is fine: the rule is about shards only
+    assert orc.layout_is_valid(16, shapes, whole, 4, 1, 16)
+    # a piece that ends exactly at the boundary does not straddle; one element more does
+    assert orc.layout_is_valid(16, [(1, 8)], [(0, 0, 8, 0)], 4, 2, 8)
+    assert not orc.layout_is_valid(16, [(1, 9)], [(0, 0, 9, 0)], 4, 2, 8)
+    flat = np.arange(100, 116)
+    assert np.array_equal(orc.materialize(flat, shapes, split)[0].ravel(), flat[4:16])
+
+
 # ----------------------------------------------------------------------------- momentum / update
 def test_momentum_hand_case_and_limits():
     G = np.array([[1.0, -2.0], [0.5, 4.0]])

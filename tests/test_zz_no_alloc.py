@@ -3,7 +3,9 @@ memory (allocator callbacks, processes whose device memory another runtime has f
 sections that must not hit an allocation's implicit synchronisation).  It takes no context and keeps
 all its scratch in a fixed array inside the library, so the test checks it against the ordinary
 entry point, muon_orthogonalize_batched, on two calls in a row: the second call runs on whatever the
-first one left in the shared scratch and must still be right.
+first one left in the shared scratch and must still be right.  Because both entry points run the same
+kernels, agreeing with each other is not enough: every result is also held against the CPU oracle, and
+the device's free memory is read before and after the calls to see that nothing was allocated.
 
 This file sorts last on purpose: if it fails under `pytest -x`, every other test has already run.
 """
@@ -11,8 +13,9 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import muon_oracle as orc
 from paper_2609_21594_b200 import workloads as wl
-from gpu_util import QUINTIC, bf16_input, dev_f32, host_f64
+from gpu_util import QUINTIC, bf16_input, dev_f32, host_f64, rel
 
 pytestmark = pytest.mark.gpu
 
@@ -37,7 +40,7 @@ def test_static_scratch_matches_regular_entry_point_twice_in_a_row(precision):
     # first a tall multi-tile matrix, then a smaller ragged one that leaves most of the old scratch in place
     for call, shape in enumerate([(1024, 256), (200, 264)]):
         g = wl.grad_np("noalloc", call, 0, shape)
-        x = bf16_input(g)[0] if precision == "bf16" else dev_f32(g)
+        x, vals = bf16_input(g) if precision == "bf16" else (dev_f32(g), g.astype(np.float64))
         expect = _reference(mb, prec, x, shape)
         out = torch.full_like(x, float("nan"))
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
@@ -51,6 +54,30 @@ def test_static_scratch_matches_regular_entry_point_twice_in_a_row(precision):
         tol = 1e-2 if precision == "bf16" else 1e-4
         assert np.linalg.norm(got - ref) <= tol * np.linalg.norm(ref)
         assert np.array_equal(got, ref)
+        # ... and right, not merely equal: the oracle in the matching arithmetic, at the benchmark spec's tolerances
+        want = orc.newton_schulz(vals, 5, QUINTIC, 1e-7, "bf16" if precision == "bf16" else "fp64")
+        assert rel(got, want) <= tol, (shape, rel(got, want))
+
+
+def test_static_scratch_allocates_no_device_memory():
+    """After the first call on the device (which resolves the array's address), further calls must leave the
+    amount of free device memory exactly as they found it: nothing is allocated, nothing is freed."""
+    from paper_2609_21594_b200 import binding as mb
+
+    shape = (384, 640)
+    x, _ = bf16_input(wl.grad_np("noalloc", 7, 0, shape))
+    outs = [torch.empty_like(x) for _ in range(3)]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    mb.muon_orthogonalize_static(x, outs[0], shape[0], shape[1], mb.NS_BF16, 5, QUINTIC, 1e-7, 0, status)   # set-up call
+    torch.cuda.synchronize()
+    free_before, total = torch.cuda.mem_get_info()
+    for out in outs[1:]:
+        mb.muon_orthogonalize_static(x, out, shape[0], shape[1], mb.NS_BF16, 5, QUINTIC, 1e-7, 0, status)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, (free_before, free_after)
+    assert int(status.item()) == 0
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[1], outs[2])
 
 
 def test_static_scratch_rejects_what_does_not_fit_and_bad_arguments():
