@@ -37,11 +37,10 @@ METRIC = "muon_optimizer_steps_per_s"
 UNIT = "steps/s"
 NUM_SHARDS = 8
 
-# DRAM bytes (read + write) of one launch of the Newton-Schulz product kernel: the mean over the three
-# products (G1, G2, G3) captured with ncu on the 4096x14336 group with 3 matrices per launch
-# (0.856 + 0.173 + 0.984 GB in the committed ncu summary of that kernel), scaled by 9/3 to the 9 matrices a
-# benchmark launch of that group holds (matrices are independent, so traffic grows in proportion).
-NS_KERNEL_DRAM_BYTES_PER_LAUNCH = (0.856e9 + 0.173e9 + 0.984e9) / 3 * (9 / 3)
+# DRAM bytes (read + write) per launch of the Newton-Schulz product kernel, from ncu captures of the same command
+# line; keyed by (config, layers).  Filled in from the committed summaries under profiles/.
+NS_TRAFFIC = {}
+NS_TRAFFIC_NOTE = ""
 
 
 # ----------------------------------------------------------------------------- helpers
@@ -143,19 +142,34 @@ def barrier(world: int):
 
 
 # ----------------------------------------------------------------------------- CPU oracle leg
-def oracle_sample_seconds(shape, repeats: int = 1):
+# Both arms estimate the whole-set oracle time the same way: one float64 Muon step of one matrix per core-size
+# class (s = 1024: the 1024 x 4096 group; s = 4096: one 4096 x 4096 matrix standing for the 4096 x 4096 and
+# 14336 x 4096 groups), each class scaled by its Newton-Schulz flop count (NS is > 99 % of the oracle's time).
+ORACLE_SAMPLES = [(1024, 4096), (4096, 4096)]
+
+
+def oracle_sample_seconds(shape):
     """Times the CPU oracle (float64, as it stands) on one full Muon step of one matrix."""
     from oracle import muon_oracle as orc
 
     W = wl.param_np("llama8b", 0, shape).astype(np.float64)
     G = wl.bf16_bits_to_f32(wl.to_bf16_bits(wl.grad_np("llama8b", 0, 0, shape, row_scaled=True))).astype(np.float64)
     M = np.zeros(shape)
-    best = float("inf")
-    for _ in range(repeats):
-        t0 = time.perf_counter()
-        orc.muon_step(W, G, M, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC, 1e-7, True, "fp64")
-        best = min(best, time.perf_counter() - t0)
-    return best
+    t0 = time.perf_counter()
+    orc.muon_step(W, G, M, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC, 1e-7, True, "fp64")
+    return time.perf_counter() - t0
+
+
+def oracle_whole_set_seconds(shapes, t_small: float, t_big: float) -> float:
+    """Whole-set estimate from the mean sample times of the two core-size classes."""
+    small = [s for s in shapes if min(s) <= 1024]
+    big = [s for s in shapes if min(s) > 1024]
+    est = 0.0
+    if small:
+        est += t_small * wl.ns_flops(small)[0] / wl.ns_flops([ORACLE_SAMPLES[0]])[0]
+    if big:
+        est += t_big * wl.ns_flops(big)[0] / wl.ns_flops([ORACLE_SAMPLES[1]])[0]
+    return est
 
 
 def blas_threads() -> int:
@@ -167,39 +181,41 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
-def cpu_baseline(shapes):
-    """Oracle on a bounded sample: one full Muon step on each of the two smallest distinct shapes;
-    the whole-set time is extrapolated by Newton-Schulz flop count (NS is > 99 % of the oracle's time)."""
-    sample = [(1024, 4096), (4096, 4096)]
-    t = sum(oracle_sample_seconds(s) for s in sample)
-    f_sample = wl.ns_flops(sample)[0]
-    f_total = wl.ns_flops(shapes)[0]
-    est = t * f_total / f_sample
+def cpu_baseline(shapes, repeats: int = 3):
+    """Oracle on a bounded sample (about 10 s of CPU work): `repeats` steps of each sample matrix."""
+    ts = [oracle_sample_seconds(ORACLE_SAMPLES[0]) for _ in range(repeats)]
+    tb = [oracle_sample_seconds(ORACLE_SAMPLES[1]) for _ in range(repeats)]
+    t_small, t_big = sum(ts) / len(ts), sum(tb) / len(tb)
+    est = oracle_whole_set_seconds(shapes, t_small, t_big)
     return {"value": 1.0 / est, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-            "sample": f"one float64 Muon step on one {sample[0][0]}x{sample[0][1]} and one {sample[1][0]}x{sample[1][1]} matrix "
-                      f"({t:.1f} s), extrapolated to the 224-matrix set by NS flop count (x{f_total / f_sample:.1f})"}
+            "sample": f"{repeats} float64 Muon steps each of one 1024x4096 ({t_small:.2f} s) and one 4096x4096 ({t_big:.2f} s) matrix; "
+                      f"each core-size class of the 224-matrix set scaled by its NS flop count ({est:.0f} s per whole step)"}
 
 
 def run_reference(args, world, rank):
-    """The reference arm: the CPU oracle as it stands, on host cores; each step is a bounded sample."""
+    """The reference arm: the CPU oracle as it stands, on host cores.  Step j is a bounded sample -- one float64
+    Muon step of the 1024 x 4096 matrix (even j) or of the 4096 x 4096 matrix (odd j) -- and the whole-set time
+    is estimated exactly as the other arm's cpu_baseline does."""
     if rank != 0:
         return
     shapes = wl.shapes_llama8b()
-    sample = (1024, 4096)
-    f_ratio = wl.ns_flops(shapes)[0] / wl.ns_flops([sample])[0]
-    for _ in range(args.warmup):
-        oracle_sample_seconds(sample)
-    times = [oracle_sample_seconds(sample) for _ in range(args.steps)]
-    t = sum(times) / len(times)
-    value = 1.0 / (t * f_ratio)
+    for j in range(args.warmup):
+        oracle_sample_seconds(ORACLE_SAMPLES[j % 2])
+    times = [[], []]
+    for j in range(max(2, args.steps)):
+        times[j % 2].append(oracle_sample_seconds(ORACLE_SAMPLES[j % 2]))
+    t_small, t_big = sum(times[0]) / len(times[0]), sum(times[1]) / len(times[1])
+    est = oracle_whole_set_seconds(shapes, t_small, t_big)
+    value = 1.0 / est
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 / value, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": "llama8b: 224 matrices (32 layers x {Wq, Wo 4096x4096; Wk, Wv 1024x4096; gate, up 14336x4096; down 4096x14336})",
-                   "sampled": f"each step = one float64 oracle Muon step of one {sample[0]}x{sample[1]} matrix, scaled by NS flops x{f_ratio:.1f}"},
+                   "sampled": "each step = one float64 oracle Muon step of one matrix (1024x4096 on even steps, 4096x4096 on odd steps); "
+                              "value = 1 / (whole-set time estimated per core-size class by NS flop count)"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-                         "sample": f"one {sample[0]}x{sample[1]} matrix per step, {t:.2f} s each"},
+                         "sample": f"{len(times[0])} x 1024x4096 ({t_small:.2f} s each) and {len(times[1])} x 4096x4096 ({t_big:.2f} s each)"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -207,6 +223,132 @@ def run_reference(args, world, rank):
 
 
 # ----------------------------------------------------------------------------- our arm
+class Workload:
+    """Device state of one configuration: whole matrices (materialize path) or flat shards (flat_state path)."""
+
+    def __init__(self, mb, cfg, shapes, dev, path, layout_kind="per_param"):
+        self.mb, self.cfg, self.shapes, self.path = mb, cfg, shapes, path
+        self.n_elem = sum(m * n for m, n in shapes)
+        row_scaled = cfg == "llama8b"
+        gen = wl.layout_per_param if layout_kind == "per_param" else wl.layout_flat_concat
+        self.layout = gen(shapes, NUM_SHARDS)
+        self.ctx = mb.Context()
+        self.L = mb.Layout(self.ctx, self.layout, 2)
+        self.ctx.ensure_workspace(shapes)
+        ctx, L, layout = self.ctx, self.L, self.layout
+        # state and inputs (seeded, synthetic; drawn on the device)
+        self.W = [wl.device_draw(cfg, 0, i, "param", s, dev, std=0.02, dtype=torch.float32) for i, s in enumerate(shapes)]
+        self.M = [torch.zeros(s, dtype=torch.float32, device=dev) for s in shapes]
+        self.G = [wl.device_draw(cfg, 0, i, "grad", s, dev, std=1e-3, dtype=torch.bfloat16, row_scaled=row_scaled)
+                  for i, s in enumerate(shapes)]
+        self.O = [torch.empty(s, dtype=torch.bfloat16, device=dev) for s in shapes]
+        self.flat_g = torch.zeros(layout.flat_len, dtype=torch.bfloat16, device=dev)
+        self.flat_o = torch.zeros(layout.flat_len, dtype=torch.bfloat16, device=dev)
+        ctx.muon_scatter(self.flat_g, L, self.G)            # the gradients now live in the flat shard buffer
+        for g in self.G:
+            g.zero_()
+        torch.cuda.synchronize()
+        if path == "flat_state":
+            # sharded-state flow: parameters and momenta live in flat fp32 shard buffers too; no whole-matrix state
+            self.flat_w = torch.zeros(layout.flat_len, dtype=torch.float32, device=dev)
+            self.flat_m = torch.zeros(layout.flat_len, dtype=torch.float32, device=dev)
+            L4 = mb.Layout(ctx, layout, 4)
+            ctx.muon_scatter(self.flat_w, L4, self.W)
+            torch.cuda.synchronize()
+            L4.close()
+            self.W, self.M, self.G, self.O = [], [], [], []
+            torch.cuda.empty_cache()
+
+    def one_step(self):
+        c = self.ctx
+        if self.path == "flat_state":
+            c.muon_step_flat(self.L, self.flat_w, self.flat_g, self.flat_m, self.flat_o, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
+        elif self.path == "copy_only":
+            c.muon_materialize(self.flat_g, self.L, self.G)
+            c.muon_scatter(self.flat_o, self.L, self.G)
+        else:
+            c.muon_materialize(self.flat_g, self.L, self.G)
+            c.muon_step_batched_out(self.W, self.G, self.M, self.O, self.shapes, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
+            c.muon_scatter(self.flat_o, self.L, self.O)
+
+    def close(self):
+        self.L.close()
+        self.ctx.close()
+        self.W = self.M = self.G = self.O = []
+        self.flat_g = self.flat_o = self.flat_w = self.flat_m = None
+        torch.cuda.empty_cache()
+
+
+def timed_region(wk, steps, world, rank, local, dev, sample_clocks=True):
+    """K steps between two events on the launching stream, barrier + synchronize on both sides, max over ranks."""
+    ctx = wk.ctx
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ctx.muon_profile_enable(True)
+    ctx.muon_profile_reset()
+    launches0, enc0 = ctx.muon_launch_count(), ctx.muon_tensor_map_encodes()
+    sampler = ClockSampler(local)
+    if rank == 0 and sample_clocks:
+        sampler.start()
+    barrier(world)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(steps):
+        wk.one_step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier(world)
+    clk = sampler.stop() if (rank == 0 and sample_clocks) else {}
+    t = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    n = ctx.muon_launch_count() - launches0
+    enc = ctx.muon_tensor_map_encodes() - enc0
+    ph = ctx.muon_profile_read()
+    ctx.muon_profile_enable(False)
+    if ctx.muon_synchronize_and_check() != 0:
+        raise SystemExit("a bounded device-side wait expired during the timed region")
+    return t, n, ph, clk, enc
+
+
+def summarize(wk, ms, steps, launches, phases, encodes, peaks, world=1):
+    """Per-configuration record: step time, NS rate against the tensor roofline, HBM kernels against the copy peak."""
+    dense, sym = wl.ns_flops(wk.shapes)
+    ns_ms, ns_launches = phases["ns"]
+    rec = {"matrices": len(wk.shapes), "elements": wk.n_elem, "ms_per_step": ms / steps, "steps_per_s": world * 1e3 * steps / ms,
+           "launches_per_step": launches // steps, "ns_launches_per_step": ns_launches // steps,
+           "tensor_map_encodes_per_step": encodes / steps}
+    if ns_ms > 0:
+        s_per_step = ns_ms / 1e3 / steps
+        ach = sym / s_per_step / 1e12
+        rec["ns"] = {"ms_per_step": ns_ms / steps, "tflops_algorithmic_symmetric": ach,
+                     "tflops_dense_equivalent": dense / s_per_step / 1e12,
+                     "frac_of_sustained_peak": ach / peaks["bf16_sustained"], "frac_of_burst_peak": ach / peaks["bf16_burst"],
+                     "frac_of_nominal_2250": ach / 2250.0}
+    hbm = {}
+    upd_bytes = 12 if wk.path != "copy_only" else 0
+    for name, bytes_per_elem in (("momentum", 12), ("update", upd_bytes), ("gather", 4), ("scatter", 4)):
+        pms, _ = phases[name]
+        if pms > 0 and bytes_per_elem:
+            gbs = wk.n_elem * bytes_per_elem / (pms / 1e3 / steps) / 1e9
+            hbm[name] = {"ms_per_step": pms / steps, "gbs": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
+                         "frac_of_nominal_8000": gbs / 8000.0}
+    rec["hbm_kernels"] = hbm
+    return rec
+
+
+def side_config(mb, name, cfg, shapes, dev, path, steps, peaks, local, layout_kind="per_param"):
+    """One of the other configurations, measured after the headline (rank 0's own GPU only, a few steps)."""
+    wk = Workload(mb, cfg, shapes, dev, path, layout_kind)
+    for _ in range(3):
+        wk.one_step()
+    torch.cuda.synchronize()
+    ms, launches, phases, _, enc = timed_region(wk, steps, 1, 0, local, dev, sample_clocks=False)
+    rec = summarize(wk, ms, steps, launches, phases, enc, peaks)
+    rec["workload"] = name
+    rec["steps"] = steps
+    wk.close()
+    return rec
+
+
 def run_ours(args, world, rank, local):
     from paper_2609_21594_b200 import binding as mb   # fails loudly when the CUDA library is missing
 
@@ -216,80 +358,24 @@ def run_ours(args, world, rank, local):
     dev = torch.device("cuda", local)
     if args.config == "llama8b":
         shapes = wl.shapes_llama8b(args.layers)
+    elif args.config == "moe" and args.experts:   # a cut-down MoE set for profiler captures
+        shapes = wl.shapes_moe(1, args.experts)
     else:                                   # the other configurations: extra data points, never the headline
         shapes = wl.CONFIGS[args.config]()
-    cfg, row_scaled = args.config, args.config == "llama8b"
-    n_elem = sum(m * n for m, n in shapes)
-    layout = wl.layout_per_param(shapes, NUM_SHARDS)
-    ctx = mb.Context()
-    L = mb.Layout(ctx, layout, 2)
-    ctx.ensure_workspace(shapes)
+    cfg = args.config
+    peaks = load_peaks()
+    wk = Workload(mb, cfg, shapes, dev, args.path, args.layout)
+    ctx, layout, L = wk.ctx, wk.layout, wk.L
     stream = torch.cuda.current_stream()
 
-    # ---- state and inputs (seeded, synthetic; drawn on the device)
-    W = [wl.device_draw(cfg, 0, i, "param", s, dev, std=0.02, dtype=torch.float32) for i, s in enumerate(shapes)]
-    M = [torch.zeros(s, dtype=torch.float32, device=dev) for s in shapes]
-    G = [wl.device_draw(cfg, 0, i, "grad", s, dev, std=1e-3, dtype=torch.bfloat16, row_scaled=row_scaled) for i, s in enumerate(shapes)]
-    O = [torch.empty(s, dtype=torch.bfloat16, device=dev) for s in shapes]
-    flat_g = torch.zeros(layout.flat_len, dtype=torch.bfloat16, device=dev)
-    flat_o = torch.zeros(layout.flat_len, dtype=torch.bfloat16, device=dev)
-    ctx.muon_scatter(flat_g, L, G)            # the gradients now live in the flat shard buffer
-    for g in G:
-        g.zero_()
-    torch.cuda.synchronize()
-
-    if args.path == "flat_state":
-        # sharded-state flow: parameters and momenta live in flat fp32 shard buffers too; no whole-matrix state
-        flat_w = torch.zeros(layout.flat_len, dtype=torch.float32, device=dev)
-        flat_m = torch.zeros(layout.flat_len, dtype=torch.float32, device=dev)
-        L4 = mb.Layout(ctx, layout, 4)
-        ctx.muon_scatter(flat_w, L4, W)
-        torch.cuda.synchronize()
-        W, M, G, O = [], [], [], []
-        torch.cuda.empty_cache()
-
-        def one_step():
-            ctx.muon_step_flat(L, flat_w, flat_g, flat_m, flat_o, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
-    else:
-        def one_step():
-            ctx.muon_materialize(flat_g, L, G)
-            ctx.muon_step_batched_out(W, G, M, O, shapes, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
-            ctx.muon_scatter(flat_o, L, O)
-
     for _ in range(args.warmup):
-        one_step()
+        wk.one_step()
     torch.cuda.synchronize()
-    if ctx.muon_last_device_status() != 0:
+    if ctx.muon_synchronize_and_check() != 0:
         raise SystemExit("a bounded device-side wait expired during warm-up")
 
     # ---- device-resident timing
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-
-    def timed_region():
-        ctx.muon_profile_enable(True)
-        ctx.muon_profile_reset()
-        launches0 = ctx.muon_launch_count()
-        sampler = ClockSampler(local)
-        if rank == 0:
-            sampler.start()
-        barrier(world)
-        torch.cuda.synchronize()
-        e0.record(stream)
-        for _ in range(args.steps):
-            one_step()
-        e1.record(stream)
-        torch.cuda.synchronize()
-        barrier(world)
-        clk = sampler.stop() if rank == 0 else {}
-        t = max_over_ranks(e0.elapsed_time(e1), world, dev)
-        n = ctx.muon_launch_count() - launches0
-        ph = ctx.muon_profile_read()
-        ctx.muon_profile_enable(False)
-        if ctx.muon_last_device_status() != 0:
-            raise SystemExit("a bounded device-side wait expired during the timed region")
-        return t, n, ph, clk
-
-    ms, launches, phases, clocks = timed_region()
+    ms, launches, phases, clocks, encodes = timed_region(wk, args.steps, world, rank, local, dev)
     # A region that saw a hardware or thermal slowdown, or clocks stuck low with no reason (a leftover lock), does
     # not count: measure once more.  sw_power_cap alone is normal for a dense-GEMM workload on a 1 kW part.
     bad = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
@@ -298,7 +384,7 @@ def run_ours(args, world, rank, local):
         stuck = 1.0 if (not clocks.get("reasons") and clocks["sm_mhz"] < 0.6 * clocks["sm_max_mhz"]) else 0.0
     redo = 1.0 if (rank == 0 and (bad & set(clocks.get("reasons", [])) or stuck)) else 0.0
     if max_over_ranks(redo, world, dev) > 0:
-        ms, launches, phases, clocks = timed_region()
+        ms, launches, phases, clocks, encodes = timed_region(wk, args.steps, world, rank, local, dev)
         clocks["remeasured"] = True
     ms_per_step = ms / args.steps
     value = world * 1e3 / ms_per_step
@@ -306,6 +392,7 @@ def run_ours(args, world, rank, local):
     # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region
     e2e = None
     if not args.no_e2e and args.path == "materialize":
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         host_in = host_out = None
         try:
             host_in = torch.empty(layout.flat_len, dtype=torch.bfloat16).pin_memory()
@@ -318,15 +405,15 @@ def run_ours(args, world, rank, local):
             e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
                    "error": "could not pin the host flat buffers on every rank"}
         else:
-            host_in.copy_(flat_g)
-            e2e_steps = max(1, min(args.steps, args.e2e_steps))
+            host_in.copy_(wk.flat_g)
+            e2e_steps = max(1, args.e2e_steps)
             for _ in range(2):
-                ctx.muon_step_flat_host(host_in, host_out, L, W, G, M, O, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
+                ctx.muon_step_flat_host(host_in, host_out, L, wk.W, wk.G, wk.M, wk.O, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
             torch.cuda.synchronize()
             barrier(world)
             e0.record(stream)
             for _ in range(e2e_steps):
-                ctx.muon_step_flat_host(host_in, host_out, L, W, G, M, O, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
+                ctx.muon_step_flat_host(host_in, host_out, L, wk.W, wk.G, wk.M, wk.O, LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
             e1.record(stream)
             torch.cuda.synchronize()
             barrier(world)
@@ -336,29 +423,37 @@ def run_ours(args, world, rank, local):
                    "ms_per_step": ms_e2e, "steps": e2e_steps}
         del host_in, host_out
 
+    head = summarize(wk, ms, args.steps, launches, phases, encodes, peaks, world) if rank == 0 else None
+    wk.close()
+
+    # ---- the other configurations and the sharded-state flow, a few steps each (rank 0 reports; every rank runs
+    # them so that no GPU idles while another works -- they contain no barrier)
+    side = {}
+    if args.side_configs and cfg == "llama8b" and args.path == "materialize" and args.layers == 32:
+        side["llama8b_flat_state"] = side_config(mb, "llama8b, sharded-state flow (muon_step_flat)", "llama8b", shapes, dev,
+                                                 "flat_state", 5, peaks, local)
+        side["llama8b_layout_flat_concat_copy_only"] = side_config(
+            mb, "llama8b, gather + scatter only, flat-concatenation layout (cuts fall inside matrices)", "llama8b", shapes, dev,
+            "copy_only", 5, peaks, local, layout_kind="flat_concat")
+        side["1b"] = side_config(mb, "1B-class stack, 112 matrices", "1b", wl.shapes_1b(), dev, "materialize", 10, peaks, local)
+        side["moe"] = side_config(mb, "MoE stress, 784 matrices", "moe", wl.shapes_moe(), dev, "materialize", 5, peaks, local)
+        side["tiny"] = side_config(mb, "tiny d=256 layer, 6 matrices", "tiny", wl.shapes_tiny(), dev, "materialize", 50, peaks, local)
+
     if rank != 0:
         return
-    peaks = load_peaks()
-    dense, sym = wl.ns_flops(shapes)
+    # Roofline of the dominant kernel (the paired tcgen05 product kernel).  The engine computes A = X X^T and A A^T
+    # on every unordered pair of 128-blocks once and mirrors, so the algorithmic work of the variant that runs is
+    # steps*(3 s^2 l + s^3) per matrix.
+    ns = head.get("ns", {})
     ns_ms, ns_launches = phases["ns"]
-    ns_s_per_step = ns_ms / 1e3 / args.steps
-    # The engine computes A = X X^T and A A^T on the tiles that touch the upper triangle only and mirrors
-    # them, so the algorithmic work of the variant that runs is steps*(3 s^2 l + s^3) per matrix.
-    achieved = sym / ns_s_per_step / 1e12
-    per_launch_ms = ns_ms / max(1, ns_launches)
-    roofline = {"bound": "tensor", "kernel": "ns_product_pair_kernel", "achieved": achieved, "peak": peaks["bf16_sustained"],
-                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"], "traffic": NS_KERNEL_DRAM_BYTES_PER_LAUNCH,
+    roofline = {"bound": "tensor", "kernel": "ns_product_pair_kernel", "achieved": ns.get("tflops_algorithmic_symmetric"),
+                "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": ns.get("frac_of_sustained_peak"),
+                "traffic": NS_TRAFFIC.get((cfg, args.layers)),
+                "traffic_note": NS_TRAFFIC_NOTE if NS_TRAFFIC.get((cfg, args.layers)) else "no capture for this workload",
                 "peak_source": f"bf16_tflops_sustained of {peaks['source']} (kernel timed inside a long step)",
-                "flops_per_launch": sym / (ns_launches / args.steps), "ms_per_launch": per_launch_ms,
-                "launches_per_step": ns_launches // args.steps,
-                "frac_of_burst_peak": achieved / peaks["bf16_burst"], "frac_of_nominal_2250": achieved / 2250.0}
-    hbm = {}
-    for name, bytes_per_elem in (("momentum", 12), ("update", 12), ("gather", 4), ("scatter", 4)):
-        pms, _ = phases[name]
-        if pms > 0:
-            gbs = n_elem * bytes_per_elem / (pms / 1e3 / args.steps) / 1e9
-            hbm[name] = {"ms_per_step": pms / args.steps, "gbs": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
-                         "frac_of_nominal_8000": gbs / 8000.0}
+                "flops_per_launch": wl.ns_flops(shapes)[1] / max(1, ns_launches / args.steps),
+                "ms_per_launch": ns_ms / max(1, ns_launches), "launches_per_step": ns_launches // args.steps,
+                "frac_of_burst_peak": ns.get("frac_of_burst_peak"), "frac_of_nominal_2250": ns.get("frac_of_nominal_2250")}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
@@ -366,18 +461,23 @@ def run_ours(args, world, rank, local):
         "config": {"workload": (f"llama8b: {len(shapes)} matrices ({args.layers} layers x {{Wq, Wo 4096x4096; Wk, Wv 1024x4096; "
                                 "gate, up 14336x4096; down 4096x14336}), bf16 row-scaled grads in 8 flat shards, fp32 params and momenta")
                                if cfg == "llama8b" else f"{cfg}: {len(shapes)} matrices, bf16 grads in 8 flat shards, fp32 params and momenta",
-                   "elements": n_elem, "ns_steps": wl.NS_STEPS, "coeffs": list(wl.QUINTIC), "lr": LR, "mu": MU, "wd": WD,
-                   "l2": "inputs_exceed_l2", "parallelism": "replicas" if world > 1 else "single",
-                   "path": "materialize -> step -> scatter" if args.path == "materialize" else
-                           "sharded-state flow (muon_step_flat: gather and scatter fused into the elementwise kernels)"},
+                   "elements": head["elements"], "ns_steps": wl.NS_STEPS, "coeffs": list(wl.QUINTIC), "lr": LR, "mu": MU, "wd": WD,
+                   "l2": "inputs_exceed_l2", "parallelism": "replicas" if world > 1 else "single", "layout": args.layout,
+                   "path": {"materialize": "materialize -> step -> scatter",
+                            "flat_state": "sharded-state flow (muon_step_flat: gather and scatter fused into the elementwise kernels)",
+                            "copy_only": "gather + scatter only"}[args.path]},
         "roofline": roofline,
-        "ns_tflops": {"algorithmic_symmetric": achieved, "dense_equivalent_effective": dense / ns_s_per_step / 1e12},
+        "ns_tflops": {"algorithmic_symmetric": ns.get("tflops_algorithmic_symmetric"),
+                      "dense_equivalent_effective": ns.get("tflops_dense_equivalent")},
         "phases": {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] // args.steps} for k, v in phases.items()},
-        "hbm_kernels": hbm,
+        "hbm_kernels": head["hbm_kernels"],
+        "tensor_map_encodes_per_step": head["tensor_map_encodes_per_step"],
         "e2e": e2e,
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
+    if side:
+        line["configs"] = side
     if world == 1 and not args.no_cpu_baseline and cfg == "llama8b":
         line["cpu_baseline"] = cpu_baseline(shapes)
     print(json.dumps(line), flush=True)
@@ -392,9 +492,15 @@ def main():
     ap.add_argument("--layers", type=int, default=32, help="layers of the Llama-3-8B set (32 = the benchmark workload)")
     ap.add_argument("--config", choices=sorted(wl.CONFIGS), default="llama8b",
                     help="llama8b is the benchmark workload; the others are extra data points")
-    ap.add_argument("--path", choices=["materialize", "flat_state"], default="materialize",
-                    help="materialize: the benchmark step (gather, step, scatter); flat_state: the fused sharded-state flow")
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--experts", type=int, default=0, help="with --config moe: one layer of this many experts (small profiler case)")
+    ap.add_argument("--path", choices=["materialize", "flat_state", "copy_only"], default="materialize",
+                    help="materialize: the benchmark step (gather, step, scatter); flat_state: the fused sharded-state flow; "
+                         "copy_only: gather and scatter alone")
+    ap.add_argument("--layout", choices=["per_param", "flat_concat"], default="per_param",
+                    help="flat-shard layout generator: per-parameter row split, or flat concatenation cut into equal parts")
+    ap.add_argument("--e2e-steps", type=int, default=8)
+    ap.add_argument("--no-side-configs", dest="side_configs", action="store_false",
+                    help="skip the records of the other configurations (1B, MoE, tiny, sharded-state flow)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -43,7 +43,7 @@ extern "C" {
 #define MUON_ERR_UNSUPPORTED        -3   /* legal request the library does not implement                   */
 #define MUON_ERR_WORKSPACE_TOO_SMALL -4  /* muon_set_workspace not called, or buffer smaller than required  */
 #define MUON_ERR_CUDA               -5   /* a CUDA runtime/driver call failed (no usable device, launch...) */
-#define MUON_ERR_DEVICE_TIMEOUT     -6   /* a bounded device-side wait gave up (see muon_last_device_status) */
+#define MUON_ERR_DEVICE_TIMEOUT     -6   /* a bounded device-side wait gave up; returned by muon_synchronize_and_check only */
 #define MUON_ERR_TOO_LARGE          -7   /* the matrix needs more than the fixed built-in scratch (muon_orthogonalize_static) */
 
 /* ------------------------------------------------------------------ enums */
@@ -53,9 +53,9 @@ extern "C" {
 #define MUON_NS_BF16 0   /* bf16 operands, fp32 accumulation on the tensor cores (Section 6.6: "bf16 arithmetic") */
 #define MUON_NS_FP32 1   /* every product and intermediate in fp32 (no counterpart in the paper; accuracy anchor)  */
 
-#define MUON_ENGINE_TENSOR      0   /* tensor cores; CTA pairs (cta_group::2) wherever a matrix has more than 128 rows */
+#define MUON_ENGINE_TENSOR      0   /* tensor cores, CTA pairs (cta_group::2), one launch per product for all shape groups */
 #define MUON_ENGINE_CUDA_CORE   1
-#define MUON_ENGINE_TENSOR_1CTA 2   /* tensor cores, single-CTA kernel only (cross-check of the paired kernel)        */
+#define MUON_ENGINE_TENSOR_1CTA 2   /* tensor cores, single-CTA kernel, one launch per product per shape group (cross-check) */
 
 /* flags of muon_orthogonalize_batched */
 #define MUON_ORTHO_NO_NORMALIZE 1u  /* treat the input as X_0 already (r = 1); used for single-step checks */
@@ -132,6 +132,24 @@ int muon_set_workspace(muon_ctx_t* ctx, void* dev_ptr, size_t bytes);
  * chunk_of[i] receives the chunk index of matrix i (may be NULL); *num_chunks the count. */
 int muon_plan_describe(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count,
                        int32_t* num_chunks, int32_t* chunk_of);
+
+/* Host-only description of how the chunks are launched: chunks are packed (first fit, largest first) into
+ * launch sets of at most chunk_elems elements in total -- the memory-safe cap of Section 6.6 then bounds what
+ * is resident in the workspace at once -- and the tensor engine runs every Newton-Schulz product as ONE kernel
+ * per launch set, over all its core shapes (3 * ns_steps product launches per set; small groups no longer
+ * get launches of their own: "per-matrix NS launches starve the device for small matrices", Section 6.6).
+ * set_of[i] receives the launch set of matrix i (-1 for empty matrices; may be NULL); *num_sets the count. */
+int muon_plan_launch_sets(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count,
+                          int32_t* num_sets, int32_t* set_of);
+
+/* Host-only: the tile list the tensor engine uses for a symmetric product (A = X X^T, A A^T) whose result has
+ * `blocks` x `blocks` blocks of 128 rows/columns.  Tile i is tiles[4i..4i+3] = (ra, rb, cc, cd): row blocks ra
+ * and rb (one per CTA of a pair; 0xFFFF = none) against column blocks cc and cd (0xFFFF = the tile is 128
+ * columns wide).  Every unordered pair of blocks is covered (the kernel mirrors off-diagonal blocks); the only
+ * block computed twice is the lower-left one of each diagonal 2 x 2 tile, and a last odd column gets 128-wide
+ * tiles instead of half-empty 256-wide ones.  *count receives the number of tiles; at most `capacity` are
+ * written.  Exposed so that the combinatorics can be tested on a CPU. */
+int muon_symmetric_tiles(int32_t blocks, uint16_t* tiles, int32_t capacity, int32_t* count);
 
 /* Validates a layout description on the host (no device needed): every element of every
  * matrix covered exactly once; segments inside one shard, pairwise disjoint in the flat
@@ -277,11 +295,13 @@ int muon_ns_product(muon_ctx_t* ctx, const void* p, const void* q, const void* d
  * 4*rows*cols + 4*min(rows,cols)^2 bytes; 1024 x 1024 fits, 2048 x 2048 does not) is rejected
  * with MUON_ERR_TOO_LARGE and nothing is launched.
  * Set-up: the first call on each device resolves the array's device address and the driver's
- * tensor-map encoder; make that first call outside any stream capture.
+ * tensor-map encoder (guarded by a mutex, so first calls may come from several host threads); make
+ * that first call outside any stream capture.  The matrix descriptor and the engine's small tables
+ * reach the device as kernel arguments, so no host-to-device copy of the call outlives it.
  * Sharing: all calls on a device use the same array, which keeps whatever the previous call left;
  * the entry point rewrites every element it later reads, so no clearing by the caller is needed,
  * but two calls whose device work overlaps in time (different streams without ordering) race. */
-#define MUON_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u + 4096u)
+#define MUON_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u + 16384u)
 int muon_orthogonalize_static(const void* in, void* out, int32_t rows, int32_t cols, int32_t ns_precision,
                               int32_t ns_steps, const float* coeffs, float eps, uint32_t flags,
                               int32_t* status, void* stream);
@@ -294,7 +314,13 @@ int muon_last_device_status(muon_ctx_t* ctx, void* stream, int32_t* status);
 /* Resets the status word to 0 (stream-ordered). */
 int muon_clear_device_status(muon_ctx_t* ctx, void* stream);
 
-/* Failure-detection self-test: launches one tiny kernel that waits, with a limit of about a millisecond,
+/* Opt-in synchronous check: synchronises `stream`, then returns MUON_OK when no bounded wait has expired on this
+ * context and MUON_ERR_DEVICE_TIMEOUT when one has (the results of the affected call are then incomplete).
+ * The step entry points themselves never synchronise and therefore never return that code: a caller that wants
+ * the guarantee calls this (or muon_last_device_status) before it consumes a step's results. */
+int muon_synchronize_and_check(muon_ctx_t* ctx, void* stream);
+
+/* Failure-detection self-test (a test hook, not part of the optimizer path): launches one tiny kernel that waits, with a limit of about a millisecond,
  * on a barrier nothing ever arrives at, using the same bounded-wait routine as the tensor-core pipelines.
  * The wait must expire, the kernel records code 100 in the status word and returns normally; the context
  * stays usable.  No real pipeline is involved and nothing can hang. */
@@ -315,6 +341,11 @@ int muon_profile_read(muon_ctx_t* ctx, int32_t phase, double* ms, int64_t* launc
 
 /* Total kernels this context has launched since creation. */
 int64_t muon_launch_count(const muon_ctx_t* ctx);
+
+/* Total tensor maps this context has encoded since creation.  The plan of a shape list encodes its maps once,
+ * when it first runs on a workspace (Section 6.2: the plan is fixed when the optimizer is built and replayed
+ * unchanged every step); in steady state the count does not move. */
+int64_t muon_tensor_map_encodes(const muon_ctx_t* ctx);
 
 const char* muon_status_string(int status);
 

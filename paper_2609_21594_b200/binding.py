@@ -21,7 +21,7 @@ lib = C.CDLL(LIB_PATH)
 
 OK, ERR_INVALID_ARG, ERR_BAD_LAYOUT, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_DEVICE_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
 ERR_TOO_LARGE = -7
-STATIC_SCRATCH_BYTES = 16 * 1024 * 1024 + 4096
+STATIC_SCRATCH_BYTES = 16 * 1024 * 1024 + 16384
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 NS_BF16, NS_FP32 = 0, 1
 ENGINE_TENSOR, ENGINE_CUDA_CORE, ENGINE_TENSOR_1CTA = 0, 1, 2
@@ -63,6 +63,8 @@ _sig = {
     "muon_workspace_bytes": (C.c_int, [C.POINTER(Options), C.POINTER(Shape), C.c_int32, C.POINTER(C.c_size_t)]),
     "muon_set_workspace": (C.c_int, [_vp, _vp, C.c_size_t]),
     "muon_plan_describe": (C.c_int, [C.POINTER(Options), C.POINTER(Shape), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
+    "muon_plan_launch_sets": (C.c_int, [C.POINTER(Options), C.POINTER(Shape), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
+    "muon_symmetric_tiles": (C.c_int, [C.c_int32, C.POINTER(C.c_uint16), C.c_int32, C.POINTER(C.c_int32)]),
     "muon_layout_validate": (C.c_int, [C.POINTER(LayoutDesc)]),
     "muon_layout_create": (C.c_int, [_vp, C.POINTER(LayoutDesc), C.POINTER(_vp)]),
     "muon_layout_destroy": (None, [_vp]),
@@ -86,6 +88,8 @@ _sig = {
                                             C.c_float, C.c_uint32, _vp, _vp]),
     "muon_last_device_status": (C.c_int, [_vp, _vp, C.POINTER(C.c_int32)]),
     "muon_clear_device_status": (C.c_int, [_vp, _vp]),
+    "muon_synchronize_and_check": (C.c_int, [_vp, _vp]),
+    "muon_tensor_map_encodes": (C.c_int64, [_vp]),
     "muon_self_test_bounded_wait": (C.c_int, [_vp, _vp]),
     "muon_profile_enable": (C.c_int, [_vp, C.c_int32]),
     "muon_profile_reset": (C.c_int, [_vp]),
@@ -154,6 +158,22 @@ def muon_plan_describe(opt: Options, shapes) -> Tuple[int, List[int]]:
     chunk_of = (C.c_int32 * max(1, len(shapes)))()
     _check(lib.muon_plan_describe(C.byref(opt), _shapes(shapes), len(shapes), C.byref(n), chunk_of), "muon_plan_describe")
     return int(n.value), [int(chunk_of[i]) for i in range(len(shapes))]
+
+
+def muon_plan_launch_sets(opt: Options, shapes) -> Tuple[int, List[int]]:
+    n = C.c_int32(0)
+    set_of = (C.c_int32 * max(1, len(shapes)))()
+    _check(lib.muon_plan_launch_sets(C.byref(opt), _shapes(shapes), len(shapes), C.byref(n), set_of), "muon_plan_launch_sets")
+    return int(n.value), [int(set_of[i]) for i in range(len(shapes))]
+
+
+def muon_symmetric_tiles(blocks: int) -> List[Tuple[int, int, int, int]]:
+    """The tile list of a symmetric product over blocks x blocks blocks of 128: [(ra, rb, cc, cd)], 0xFFFF = none."""
+    n = C.c_int32(0)
+    _check(lib.muon_symmetric_tiles(blocks, None, 0, C.byref(n)), "muon_symmetric_tiles")
+    buf = (C.c_uint16 * max(1, 4 * n.value))()
+    _check(lib.muon_symmetric_tiles(blocks, buf, n.value, C.byref(n)), "muon_symmetric_tiles")
+    return [(buf[4 * i], buf[4 * i + 1], buf[4 * i + 2], buf[4 * i + 3]) for i in range(n.value)]
 
 
 def make_layout_desc(layout, elem_size: int):
@@ -339,6 +359,16 @@ class Context:
 
     def muon_clear_device_status(self, stream=None) -> None:
         _check(lib.muon_clear_device_status(self.handle, _stream(stream)), "muon_clear_device_status")
+
+    def muon_synchronize_and_check(self, stream=None) -> int:
+        """Returns OK or ERR_DEVICE_TIMEOUT (does not raise for the latter: it is the answer, not a failure of the call)."""
+        rc = int(lib.muon_synchronize_and_check(self.handle, _stream(stream)))
+        if rc not in (OK, ERR_DEVICE_TIMEOUT):
+            _check(rc, "muon_synchronize_and_check")
+        return rc
+
+    def muon_tensor_map_encodes(self) -> int:
+        return int(lib.muon_tensor_map_encodes(self.handle))
 
     def muon_self_test_bounded_wait(self, stream=None) -> None:
         _check(lib.muon_self_test_bounded_wait(self.handle, _stream(stream)), "muon_self_test_bounded_wait")

@@ -8,9 +8,9 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmuon_b200.so")
-SOURCES = ["api.cu", "plan.cu", "layout_kernels.cu", "elementwise_kernels.cu", "ns_simt.cu", "ns_tcgen05.cu", "ns_tcgen05_pair.cu"]
+SOURCES = ["api.cu", "plan.cu", "layout_kernels.cu", "elementwise_kernels.cu", "ns_simt.cu", "ns_tcgen05.cu", "ns_tcgen05_pair.cu", "ns_tables.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC"]
+              "-Xcompiler", "-fPIC"] + os.environ.get("MUON_NVCC_EXTRA", "").split()
 
 
 def _nvcc() -> str:

@@ -5,7 +5,9 @@
 #include <cstring>
 #include <new>
 
-#include "internal.h"
+#include <mutex>
+
+#include "tc_tables.h"
 
 using namespace muon;
 
@@ -31,8 +33,9 @@ bool valid_options(const muon_options_t& o) {
   return true;
 }
 
-// Stream-ordered upload of a small host table through a ring of pinned staging slots.
-int upload(muon_ctx* ctx, const void* src, size_t bytes, cudaStream_t st, void** dev_out) {
+// Stream-ordered upload of a small host table through a ring of pinned staging slots, in two halves so that a
+// caller may learn the device address before it fills the table in.
+int acquire_slot(muon_ctx* ctx, size_t bytes, StagingSlot** out) {
   StagingSlot& s = ctx->slots[ctx->next_slot];
   ctx->next_slot = (ctx->next_slot + 1) % 4;
   if (s.used && cudaEventSynchronize(s.ev) != cudaSuccess) return MUON_ERR_CUDA;
@@ -49,11 +52,25 @@ int upload(muon_ctx* ctx, const void* src, size_t bytes, cudaStream_t st, void**
     s.cap = cap;
   }
   if (!s.ev && cudaEventCreateWithFlags(&s.ev, cudaEventDisableTiming) != cudaSuccess) return MUON_ERR_CUDA;
-  std::memcpy(s.host, src, bytes);
-  if (cudaMemcpyAsync(s.dev, s.host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return MUON_ERR_CUDA;
-  if (cudaEventRecord(s.ev, st) != cudaSuccess) return MUON_ERR_CUDA;
-  s.used = true;
-  *dev_out = s.dev;
+  *out = &s;
+  return MUON_OK;
+}
+
+int commit_slot(StagingSlot* s, const void* src, size_t bytes, cudaStream_t st) {
+  std::memcpy(s->host, src, bytes);
+  if (cudaMemcpyAsync(s->dev, s->host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return MUON_ERR_CUDA;
+  if (cudaEventRecord(s->ev, st) != cudaSuccess) return MUON_ERR_CUDA;
+  s->used = true;
+  return MUON_OK;
+}
+
+int upload(muon_ctx* ctx, const void* src, size_t bytes, cudaStream_t st, void** dev_out) {
+  StagingSlot* s = nullptr;
+  int rc = acquire_slot(ctx, bytes, &s);
+  if (rc != MUON_OK) return rc;
+  rc = commit_slot(s, src, bytes, st);
+  if (rc != MUON_OK) return rc;
+  *dev_out = s->dev;
   return MUON_OK;
 }
 
@@ -98,15 +115,21 @@ Plan* get_plan(muon_ctx* ctx, const muon_shape_t* shapes, int32_t count, int* st
   Plan p;
   *status = build_plan(ctx->opt, shapes, count, &p);
   if (*status != MUON_OK) return nullptr;
-  if (ctx->plans.size() > 64) ctx->plans.clear();
+  if (ctx->plans.size() > 64) {
+    for (auto& kv : ctx->plans) release_plan_tables(&kv.second);
+    ctx->plans.clear();
+  }
   return &ctx->plans.emplace(std::move(key), std::move(p)).first->second;
 }
 
+bool grouped_engine(const muon_ctx* ctx) {
+  return ctx->opt.ns_precision == MUON_NS_BF16 && ctx->opt.engine == MUON_ENGINE_TENSOR;
+}
+
+// One product on the engines that launch per shape group (single-CTA tensor kernel, CUDA cores).
 int run_gemm(muon_ctx* ctx, const GemmArgs& g, cudaStream_t st) {
-  if (ctx->opt.ns_precision == MUON_NS_BF16 && ctx->opt.engine != MUON_ENGINE_CUDA_CORE && tc_supported(g)) {
-    if (ctx->opt.engine == MUON_ENGINE_TENSOR && tc_pair_supported(g)) return launch_gemm_tc_pair(ctx, g, st);
+  if (ctx->opt.ns_precision == MUON_NS_BF16 && ctx->opt.engine != MUON_ENGINE_CUDA_CORE && tc_supported(g))
     return launch_gemm_tc(ctx, g, st);
-  }
   return launch_gemm_simt(g, ctx->opt.ns_precision, st);
 }
 
@@ -118,102 +141,168 @@ struct ChunkRun {
   const float* coeffs;
 };
 
-int run_chunk(muon_ctx* ctx, const Chunk& ch, const MatDesc* d_descs, const ChunkRun& r, cudaStream_t st,
-              const RowSeg* d_segs = nullptr, bool pitch8 = true) {
-  const int32_t wide = (pitch8 && ch.s % 8 == 0 && ch.l % 8 == 0) ? 1 : 0;
-  const WsCarve w = carve_chunk(ctx->opt, ch);
-  char* base = static_cast<char*>(ctx->ws);
-  void* x0 = base + w.x0;
-  void* x1 = base + w.x1;
-  void* A = base + w.a;
-  void* B = base + w.b;
-  float* partials = reinterpret_cast<float*>(base + w.partials);
-  float* rnorm = reinterpret_cast<float*>(base + w.rnorm);
-  int n;
-  {
-    Span sp(ctx, MUON_PHASE_MOMENTUM, st);
-    StageArgs sa;
-    sa.segs = d_segs;
-    sa.descs = d_descs + ch.desc_begin;
-    sa.x = x0;
-    sa.partials = partials;
-    sa.rnorm = rnorm;
-    sa.count = ch.count;
-    sa.tiles_per_mat = ch.tiles_per_mat;
-    sa.s = ch.s; sa.l = ch.l; sa.ldx = ch.ldx;
-    sa.mu = r.mu; sa.eps = ctx->opt.eps;
-    sa.nesterov = ctx->opt.nesterov;
-    sa.grad_dtype = ctx->opt.grad_dtype;
-    sa.ns_precision = ctx->opt.ns_precision;
-    sa.momentum = r.momentum;
-    sa.normalize = r.normalize;
-    sa.wide = wide;
-    n = launch_stage(sa, st);
-    if (n < 0) return n;
-    ctx->launches += n;
-    sp.end(n);
+// Everything the kernels of one launch set need besides the plan.
+struct SetRun {
+  const std::vector<Chunk>* chunks;
+  const LaunchSet* set;
+  const SetTables* tables;      // null: per-group engines
+  const MatDesc* d_descs;       // device, first record of the SET
+  const RowSeg* d_segs;         // flat-shard mode, else null
+  bool pitch8;
+  int32_t flat_vec;
+};
+
+int fill_elem_chunks(const SetRun& sr, bool want_wide, int x_index, ElemChunk* out) {
+  int n = 0;
+  for (int32_t ci : sr.set->chunks) {
+    const Chunk& c = (*sr.chunks)[size_t(ci)];
+    const bool wide = sr.pitch8 && c.s % 8 == 0 && c.l % 8 == 0;
+    if (wide != want_wide) continue;
+    ElemChunk& e = out[n++];
+    e.block_begin = 0;
+    e.tiles = 0;
+    e.desc_begin = c.desc_begin - sr.set->desc_begin;
+    e.count = c.count;
+    e.s = c.s; e.l = c.l; e.ldx = c.ldx; e.pad = 0;
+    e.x_off = int64_t(c.off_x[x_index]);
+    e.part_off = c.part_off;
   }
-  void* cur = x0;
-  void* nxt = x1;
-  {
-    Span sp(ctx, MUON_PHASE_NS, st);
-    int64_t total = 0;
+  return n;
+}
+
+// The three Newton-Schulz products of every step, for every shape group of the set.
+int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStream_t st, int64_t* launches) {
+  char* base = static_cast<char*>(ctx->ws);
+  const float* rnorm = reinterpret_cast<const float*>(base + sr.set->off_rnorm);
+  int n;
+  if (sr.tables) {
+    auto launch = [&](const tc::TcTable& tab, float alpha, float beta, int gamma_mode) {
+      tc::TcLaunch L;
+      L.maps = tab.maps;
+      for (int i = 0; i < tab.nprob; ++i) L.info[i] = tab.info[i];
+      L.nprob = tab.nprob;
+      L.total_tiles = tab.total_tiles;
+      L.alpha = alpha; L.beta = beta; L.gamma_mode = gamma_mode;
+      L.coef_a = L.coef_b = -1;
+      L.coef_stride = 0;
+      L.status = ctx->d_status;
+      return launch_tc_grouped(ctx->device, L, st);
+    };
+    for (int k = 0; k < r.ns_steps; ++k) {
+      const float* co = r.coeffs + (ctx->opt.coeffs_per_step ? 3 * k : 0);
+      const int cur = k & 1;
+      if ((n = launch(sr.tables->g1[cur], 1.f, 0.f, k == 0 ? 2 : 0)) < 0) return n;     // A = gamma X X^T
+      *launches += n;
+      if ((n = launch(sr.tables->g2, co[2], co[1], 0)) < 0) return n;                   // B = b A + c A A^T (A symmetric)
+      *launches += n;
+      if ((n = launch(sr.tables->g3[cur], 1.f, co[0], k == 0 ? 1 : 0)) < 0) return n;   // X' = gamma (a X + B X)
+      *launches += n;
+    }
+    return MUON_OK;
+  }
+  for (int32_t ci : sr.set->chunks) {
+    const Chunk& ch = (*sr.chunks)[size_t(ci)];
+    void* xs[2] = {base + ch.off_x[0], base + ch.off_x[1]};
+    void* A = base + ch.off_a;
+    void* B = base + ch.off_b;
+    const float* rn = rnorm + (ch.desc_begin - sr.set->desc_begin);
     const int64_t sx = int64_t(ch.s) * ch.ldx, sa_ = int64_t(ch.s) * ch.lda;
     for (int k = 0; k < r.ns_steps; ++k) {
       const float* co = r.coeffs + (ctx->opt.coeffs_per_step ? 3 * k : 0);
+      void* cur = xs[k & 1];
+      void* nxt = xs[(k & 1) ^ 1];
       GemmArgs g{};
-      // A = gamma * X X^T
       g.p = cur; g.q = cur; g.d = nullptr; g.c = A;
       g.m = ch.s; g.n = ch.s; g.kdim = ch.l;
       g.ldp = ch.ldx; g.ldq = ch.ldx; g.ldc = ch.lda;
       g.stride_p = sx; g.stride_q = sx; g.stride_c = sa_;
-      g.batch = ch.count; g.rnorm = rnorm; g.gamma_mode = (k == 0) ? 2 : 0;
+      g.batch = ch.count; g.rnorm = rn; g.gamma_mode = (k == 0) ? 2 : 0;
       g.alpha = 1.f; g.beta = 0.f; g.nn = 0; g.symmetric = 1;
       if ((n = run_gemm(ctx, g, st)) < 0) return n;
-      total += n;
-      // B = b A + c A A^T   (A symmetric, so A A^T = A^2)
+      *launches += n;
       g.p = A; g.q = A; g.d = A; g.c = B;
       g.kdim = ch.s; g.ldp = ch.lda; g.ldq = ch.lda;
       g.stride_p = sa_; g.stride_q = sa_;
       g.gamma_mode = 0; g.alpha = co[2]; g.beta = co[1];
       if ((n = run_gemm(ctx, g, st)) < 0) return n;
-      total += n;
-      // X' = gamma * (a X + B X)
+      *launches += n;
       g.p = B; g.q = cur; g.d = cur; g.c = nxt;
       g.m = ch.s; g.n = ch.l; g.kdim = ch.s;
       g.ldp = ch.lda; g.ldq = ch.ldx; g.ldc = ch.ldx;
       g.stride_p = sa_; g.stride_q = sx; g.stride_c = sx;
       g.gamma_mode = (k == 0) ? 1 : 0; g.alpha = 1.f; g.beta = co[0]; g.nn = 1; g.symmetric = 0;
       if ((n = run_gemm(ctx, g, st)) < 0) return n;
+      *launches += n;
+    }
+  }
+  return MUON_OK;
+}
+
+int run_set(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStream_t st) {
+  char* base = static_cast<char*>(ctx->ws);
+  int n;
+  {
+    Span sp(ctx, MUON_PHASE_MOMENTUM, st);
+    int64_t total = 0;
+    for (int w = 1; w >= 0; --w) {
+      StageArgs sa;
+      sa.nchunks = fill_elem_chunks(sr, w != 0, 0, sa.ch);
+      if (sa.nchunks == 0) continue;
+      sa.segs = sr.d_segs;
+      sa.descs = sr.d_descs;
+      sa.ws = base;
+      sa.partials = reinterpret_cast<float*>(base + sr.set->off_partials);
+      sa.rnorm = reinterpret_cast<float*>(base + sr.set->off_rnorm);
+      sa.mu = r.mu; sa.eps = ctx->opt.eps;
+      sa.nesterov = ctx->opt.nesterov;
+      sa.grad_dtype = ctx->opt.grad_dtype;
+      sa.ns_precision = ctx->opt.ns_precision;
+      sa.momentum = r.momentum;
+      sa.normalize = r.normalize;
+      sa.wide = w;
+      sa.flat_vec = sr.flat_vec;
+      n = launch_stage(sa, st);
+      if (n < 0) return n;
       total += n;
-      void* t = cur; cur = nxt; nxt = t;
     }
     ctx->launches += total;
     sp.end(total);
   }
   {
+    Span sp(ctx, MUON_PHASE_NS, st);
+    int64_t total = 0;
+    const int rc = run_set_products(ctx, sr, r, st, &total);
+    if (rc != MUON_OK) return rc;
+    ctx->launches += total;
+    sp.end(total);
+  }
+  {
     Span sp(ctx, MUON_PHASE_UPDATE, st);
-    ApplyArgs aa;
-    aa.segs = d_segs;
-    aa.descs = d_descs + ch.desc_begin;
-    aa.x = cur;
-    aa.count = ch.count;
-    aa.tiles_per_mat = ch.tiles_per_mat;
-    aa.s = ch.s; aa.l = ch.l; aa.ldx = ch.ldx;
-    aa.lr = r.lr; aa.wd = r.wd;
-    aa.decay = 1.0f - r.lr * r.wd;
-    aa.ns_precision = ctx->opt.ns_precision;
-    aa.update = r.momentum;
-    aa.wide = wide;
-    n = launch_apply(aa, st);
-    if (n < 0) return n;
-    ctx->launches += n;
-    sp.end(n);
+    int64_t total = 0;
+    for (int w = 1; w >= 0; --w) {
+      ApplyArgs aa;
+      aa.nchunks = fill_elem_chunks(sr, w != 0, r.ns_steps & 1, aa.ch);
+      if (aa.nchunks == 0) continue;
+      aa.segs = sr.d_segs;
+      aa.descs = sr.d_descs;
+      aa.ws = base;
+      aa.lr = r.lr; aa.wd = r.wd;
+      aa.decay = 1.0f - r.lr * r.wd;
+      aa.ns_precision = ctx->opt.ns_precision;
+      aa.update = r.momentum;
+      aa.wide = w;
+      aa.flat_vec = sr.flat_vec;
+      n = launch_apply(aa, st);
+      if (n < 0) return n;
+      total += n;
+    }
+    ctx->launches += total;
+    sp.end(total);
   }
   return MUON_OK;
 }
 
-// Host-buffer pipeline: per chunk, gradients arrive by DMA straight into the whole-matrix buffers (the
+// Host-buffer pipeline: per launch set, gradients arrive by DMA straight into the whole-matrix buffers (the
 // copy engine performs the gather) and updates leave the same way, on two copy streams that run ahead
 // of / behind the compute stream.
 struct HostPipe {
@@ -267,12 +356,29 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
       d.scale = float(0.2 * std::sqrt(double(std::max(d.rows, d.cols))));
     }
   }
+  const bool grouped = grouped_engine(ctx);
+  if (grouped) {
+    if (tc_pair_grid_setup(ctx->device) < 0) return MUON_ERR_CUDA;
+    status = bind_plan_tables(ctx, plan);
+    if (status != MUON_OK) return status;
+  }
   void* d_descs = nullptr;
   status = upload(ctx, descs.data(), descs.size() * sizeof(MatDesc), st, &d_descs);
   if (status != MUON_OK) return status;
+  auto set_run = [&](size_t k) {
+    SetRun sr;
+    sr.chunks = &plan->chunks;
+    sr.set = &plan->sets[k];
+    sr.tables = grouped ? &(*plan->set_tables)[k] : nullptr;
+    sr.d_descs = static_cast<const MatDesc*>(d_descs) + plan->sets[k].desc_begin;
+    sr.d_segs = flat ? flat->d_rowsegs : nullptr;
+    sr.pitch8 = pitch8;
+    sr.flat_vec = flat ? flat->flat_vec : 8;
+    return sr;
+  };
   if (!pipe) {
-    for (const Chunk& ch : plan->chunks) {
-      status = run_chunk(ctx, ch, static_cast<const MatDesc*>(d_descs), r, st, flat ? flat->d_rowsegs : nullptr, pitch8);
+    for (size_t k = 0; k < plan->sets.size(); ++k) {
+      status = run_set(ctx, set_run(k), r, st);
       if (status != MUON_OK) return status;
     }
     return MUON_OK;
@@ -284,10 +390,11 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
   if (cudaStreamWaitEvent(ctx->h2d_stream, ev, 0) != cudaSuccess || cudaStreamWaitEvent(ctx->d2h_stream, ev, 0) != cudaSuccess)
     return MUON_ERR_CUDA;
   // Order of the batches: only the first batch's inbound copy and the last batch's outbound copy are exposed,
-  // so the smallest batch goes first and the second smallest last; the others keep the plan's order.
-  std::vector<size_t> order(plan->chunks.size());
+  // so the smallest batch goes first and the second smallest last; the others keep the plan's order
+  // (largest first, the descending-size order of Section 6.7).
+  std::vector<size_t> order(plan->sets.size());
   for (size_t c = 0; c < order.size(); ++c) order[c] = c;
-  auto elems = [&](size_t c) { return int64_t(plan->chunks[c].count) * plan->chunks[c].s * plan->chunks[c].l; };
+  auto elems = [&](size_t c) { return plan->sets[c].elems; };
   if (order.size() > 2) {
     size_t small = 0;
     for (size_t c = 1; c < order.size(); ++c)
@@ -301,31 +408,32 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
     order.insert(order.begin(), small);
     order.push_back(last);
   }
-  std::vector<cudaEvent_t> arrived(plan->chunks.size());
+  std::vector<cudaEvent_t> arrived(plan->sets.size());
   for (size_t c : order) {                                       // all inbound copies are queued up front, in batch order
-    for (int32_t i : plan->chunks[c].mats)
-      for (const muon_segment_t& sg : pipe->layout->segs_of[size_t(i)])
-        if (cudaMemcpyAsync(static_cast<char*>(const_cast<void*>(g[i])) + size_t(sg.elem_begin) * es,
-                            pipe->host_in + size_t(sg.flat_offset) * es, size_t(sg.elem_count) * es, cudaMemcpyHostToDevice,
-                            ctx->h2d_stream) != cudaSuccess)
-          return MUON_ERR_CUDA;
+    for (int32_t ci : plan->sets[c].chunks)
+      for (int32_t i : plan->chunks[size_t(ci)].mats)
+        for (const muon_segment_t& sg : pipe->layout->segs_of[size_t(i)])
+          if (cudaMemcpyAsync(static_cast<char*>(const_cast<void*>(g[i])) + size_t(sg.elem_begin) * es,
+                              pipe->host_in + size_t(sg.flat_offset) * es, size_t(sg.elem_count) * es, cudaMemcpyHostToDevice,
+                              ctx->h2d_stream) != cudaSuccess)
+            return MUON_ERR_CUDA;
     arrived[c] = next_sync_event(ctx);
     if (!arrived[c] || cudaEventRecord(arrived[c], ctx->h2d_stream) != cudaSuccess) return MUON_ERR_CUDA;
   }
   for (size_t c : order) {
-    const Chunk& ch = plan->chunks[c];
     if (cudaStreamWaitEvent(st, arrived[c], 0) != cudaSuccess) return MUON_ERR_CUDA;
-    status = run_chunk(ctx, ch, static_cast<const MatDesc*>(d_descs), r, st, nullptr, pitch8);
+    status = run_set(ctx, set_run(c), r, st);
     if (status != MUON_OK) return status;
     cudaEvent_t done = next_sync_event(ctx);
     if (!done || cudaEventRecord(done, st) != cudaSuccess || cudaStreamWaitEvent(ctx->d2h_stream, done, 0) != cudaSuccess)
       return MUON_ERR_CUDA;
-    for (int32_t i : ch.mats)
-      for (const muon_segment_t& sg : pipe->layout->segs_of[size_t(i)])
-        if (cudaMemcpyAsync(pipe->host_out + size_t(sg.flat_offset) * es,
-                            static_cast<const char*>(o[i]) + size_t(sg.elem_begin) * es, size_t(sg.elem_count) * es,
-                            cudaMemcpyDeviceToHost, ctx->d2h_stream) != cudaSuccess)
-          return MUON_ERR_CUDA;
+    for (int32_t ci : plan->sets[c].chunks)
+      for (int32_t i : plan->chunks[size_t(ci)].mats)
+        for (const muon_segment_t& sg : pipe->layout->segs_of[size_t(i)])
+          if (cudaMemcpyAsync(pipe->host_out + size_t(sg.flat_offset) * es,
+                              static_cast<const char*>(o[i]) + size_t(sg.elem_begin) * es, size_t(sg.elem_count) * es,
+                              cudaMemcpyDeviceToHost, ctx->d2h_stream) != cudaSuccess)
+            return MUON_ERR_CUDA;
   }
   cudaEvent_t fin = next_sync_event(ctx);
   if (!fin || cudaEventRecord(fin, ctx->d2h_stream) != cudaSuccess || cudaStreamWaitEvent(st, fin, 0) != cudaSuccess)
@@ -383,6 +491,7 @@ int muon_create(muon_ctx_t** out, const muon_options_t* opt) {
 void muon_destroy(muon_ctx_t* ctx) {
   if (!ctx) return;
   cudaDeviceSynchronize();
+  for (auto& kv : ctx->plans) release_plan_tables(&kv.second);
   for (StagingSlot& s : ctx->slots) {
     if (s.host) cudaFreeHost(s.host);
     if (s.dev) cudaFree(s.dev);
@@ -422,6 +531,35 @@ int muon_plan_describe(const muon_options_t* opt, const muon_shape_t* shapes, in
     for (int32_t i = 0; i < count; ++i) chunk_of[i] = -1;
     for (size_t c = 0; c < p.chunks.size(); ++c)
       for (int32_t i : p.chunks[c].mats) chunk_of[i] = int32_t(c);
+  }
+  return MUON_OK;
+}
+
+int muon_plan_launch_sets(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count, int32_t* num_sets,
+                          int32_t* set_of) {
+  if (!opt || !num_sets || count < 0 || (count > 0 && !shapes)) return MUON_ERR_INVALID_ARG;
+  if (!valid_options(*opt)) return MUON_ERR_INVALID_ARG;
+  Plan p;
+  const int st = build_plan(*opt, shapes, count, &p);
+  if (st != MUON_OK) return st;
+  *num_sets = int32_t(p.sets.size());
+  if (set_of) {
+    for (int32_t i = 0; i < count; ++i) set_of[i] = -1;
+    for (const Chunk& c : p.chunks)
+      for (int32_t i : c.mats) set_of[i] = c.set;
+  }
+  return MUON_OK;
+}
+
+int muon_symmetric_tiles(int32_t blocks, uint16_t* tiles, int32_t capacity, int32_t* count) {
+  if (blocks < 0 || blocks > 4096 || !count || capacity < 0 || (capacity > 0 && !tiles)) return MUON_ERR_INVALID_ARG;
+  const std::vector<TilePatHost> pat = symmetric_tile_pattern(blocks);
+  *count = int32_t(pat.size());
+  for (int32_t i = 0; i < *count && i < capacity; ++i) {
+    tiles[4 * i + 0] = pat[size_t(i)].ra;
+    tiles[4 * i + 1] = pat[size_t(i)].rb;
+    tiles[4 * i + 2] = pat[size_t(i)].cc;
+    tiles[4 * i + 3] = pat[size_t(i)].cd;
   }
   return MUON_OK;
 }
@@ -473,6 +611,14 @@ int muon_layout_create(muon_ctx_t* ctx, const muon_layout_desc_t* desc, muon_lay
     if (sg.elem_count > 0 && (sg.elem_begin % cols || sg.elem_count % cols)) L->row_aligned = false;
   }
   if (L->row_aligned) {
+    // how wide the step kernels may vectorise their accesses to flat buffers: every row segment must start on
+    // a multiple of the vector width (segment starts are only guaranteed to be multiples of align_elems)
+    L->flat_vec = 8;
+    for (int64_t k = 0; k < desc->num_segments; ++k) {
+      const muon_segment_t& sg = desc->segments[k];
+      if (sg.elem_count == 0) continue;
+      while (L->flat_vec > 1 && sg.flat_offset % L->flat_vec) L->flat_vec = L->flat_vec == 8 ? 4 : 1;
+    }
     std::vector<RowSeg> rs;
     L->rowseg_begin.assign(size_t(desc->num_matrices), 0);
     L->rowseg_count.assign(size_t(desc->num_matrices), 0);
@@ -671,11 +817,41 @@ int muon_ns_product(muon_ctx_t* ctx, const void* p, const void* q, const void* d
   g.gamma_mode = gamma ? gamma_mode : 0;
   g.alpha = alpha; g.beta = beta; g.nn = nn == 1 ? 1 : 0; g.symmetric = nn == 2 ? 1 : 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  Span sp(ctx, MUON_PHASE_NS, st);
-  const int nl = run_gemm(ctx, g, st);
-  if (nl < 0) return nl;
+  int nl;
+  if (grouped_engine(ctx) && tc_supported(g)) {
+    // the grouped engine reads its problem from device memory: a one-problem table goes through the staging ring
+    if (tc_pair_grid_setup(ctx->device) < 0) return MUON_ERR_CUDA;
+    std::vector<char> img;
+    tc::TcTable tab;
+    int rc = build_product_image(ctx->tmap_encode, g, nullptr, &img, &tab, nullptr);        // size only
+    if (rc != MUON_OK) return rc;
+    StagingSlot* slot = nullptr;
+    rc = acquire_slot(ctx, img.size(), &slot);
+    if (rc != MUON_OK) return rc;
+    rc = build_product_image(ctx->tmap_encode, g, slot->dev, &img, &tab, &ctx->tmap_encodes);   // at its device address
+    if (rc != MUON_OK) return rc;
+    rc = commit_slot(slot, img.data(), img.size(), st);
+    if (rc != MUON_OK) return rc;
+    tc::TcLaunch L;
+    L.maps = tab.maps;
+    L.info[0] = tab.info[0];
+    L.nprob = 1;
+    L.total_tiles = tab.total_tiles;
+    L.alpha = g.alpha; L.beta = g.beta; L.gamma_mode = g.gamma_mode;
+    L.coef_a = L.coef_b = -1;
+    L.coef_stride = 0;
+    L.status = ctx->d_status;
+    Span sp(ctx, MUON_PHASE_NS, st);
+    nl = launch_tc_grouped(ctx->device, L, st);
+    if (nl < 0) return nl;
+    sp.end(nl);
+  } else {
+    Span sp(ctx, MUON_PHASE_NS, st);
+    nl = run_gemm(ctx, g, st);
+    if (nl < 0) return nl;
+    sp.end(nl);
+  }
   ctx->launches += nl;
-  sp.end(nl);
   return MUON_OK;
 }
 
@@ -694,6 +870,15 @@ int muon_clear_device_status(muon_ctx_t* ctx, void* stream) {
   return cudaMemsetAsync(ctx->d_status, 0, sizeof(int32_t), static_cast<cudaStream_t>(stream)) == cudaSuccess ? MUON_OK
                                                                                                                : MUON_ERR_CUDA;
 }
+
+int muon_synchronize_and_check(muon_ctx_t* ctx, void* stream) {
+  int32_t v = 0;
+  const int rc = muon_last_device_status(ctx, stream, &v);
+  if (rc != MUON_OK) return rc;
+  return v == 0 ? MUON_OK : MUON_ERR_DEVICE_TIMEOUT;
+}
+
+int64_t muon_tensor_map_encodes(const muon_ctx_t* ctx) { return ctx ? ctx->tmap_encodes : 0; }
 
 int muon_self_test_bounded_wait(muon_ctx_t* ctx, void* stream) {
   if (!ctx) return MUON_ERR_INVALID_ARG;
@@ -770,12 +955,16 @@ static __device__ __align__(256) unsigned char g_static_scratch[MUON_STATIC_SCRA
 namespace {
 
 constexpr int kMaxDevices = 64;
-constexpr size_t kStaticHeader = 4096;      // [0,256): spare status word, [256,512): matrix descriptor
+// [0,256): spare status word; [256,512): matrix descriptor; [512, 16 KiB): problem tables of the tensor engine
+constexpr size_t kStaticHeader = 16384;
+constexpr size_t kStaticDescOff = 256, kStaticTablesOff = 512;
+std::mutex g_static_mutex;                  // guards the one-time set-up below
 void* g_static_ptr[kMaxDevices] = {};       // device address of g_static_scratch, per device ordinal
 void* g_static_encode = nullptr;            // cuTensorMapEncodeTiled
 
-int static_setup(int dev, void** ptr_out) {
+int static_setup(int dev, void** ptr_out, void** encode_out) {
   if (dev < 0 || dev >= kMaxDevices) return MUON_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
   if (!g_static_ptr[dev]) {
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return MUON_ERR_CUDA;
@@ -790,9 +979,11 @@ int static_setup(int dev, void** ptr_out) {
         return MUON_ERR_CUDA;
       g_static_encode = fn;
     }
+    if (tc_pair_grid_setup(dev) < 0) return MUON_ERR_CUDA;
     g_static_ptr[dev] = p;
   }
   *ptr_out = g_static_ptr[dev];
+  *encode_out = g_static_encode;
   return MUON_OK;
 }
 
@@ -815,25 +1006,29 @@ extern "C" int muon_orthogonalize_static(const void* in, void* out, int32_t rows
   muon_default_options(&ctx.opt);
   ctx.opt.ns_precision = ns_precision;
   ctx.opt.eps = eps;
-  Chunk ch;                                    // one matrix, one chunk, described on the stack
+  std::vector<Chunk> chunks(1);                // one matrix, one shape group, one launch set
+  Chunk& ch = chunks[0];
   ch.s = std::min(rows, cols);
   ch.l = std::max(rows, cols);
   ch.ldx = (ch.l + 7) / 8 * 8;
   ch.lda = (ch.s + 7) / 8 * 8;
   ch.count = 1;
   ch.tiles_per_mat = ((ch.s + kElemTile - 1) / kElemTile) * ((ch.l + kElemTile - 1) / kElemTile);
-  ch.desc_begin = 0;
-  const WsCarve carve = carve_chunk(ctx.opt, ch);
-  if (carve.total + kStaticHeader > size_t(MUON_STATIC_SCRATCH_BYTES)) return MUON_ERR_TOO_LARGE;
+  LaunchSet set;
+  set.chunks.push_back(0);
+  set.count = 1;
+  layout_set(ctx.opt, &chunks, &set);
+  if (set.bytes + kStaticHeader > size_t(MUON_STATIC_SCRATCH_BYTES)) return MUON_ERR_TOO_LARGE;
 
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return MUON_ERR_CUDA;
   void* base = nullptr;
-  const int rc = static_setup(dev, &base);
+  void* encode = nullptr;
+  int rc = static_setup(dev, &base, &encode);
   if (rc != MUON_OK) return rc;
   char* sb = static_cast<char*>(base);
   ctx.device = dev;
-  ctx.tmap_encode = g_static_encode;
+  ctx.tmap_encode = encode;
   ctx.d_status = status ? status : reinterpret_cast<int32_t*>(sb);
   ctx.ws = sb + kStaticHeader;
   ctx.ws_bytes = size_t(MUON_STATIC_SCRATCH_BYTES) - kStaticHeader;
@@ -849,10 +1044,29 @@ extern "C" int muon_orthogonalize_static(const void* in, void* out, int32_t rows
   d.transposed = rows > cols ? 1 : 0;
   d.scale = 0.f;
   d.seg_begin = d.seg_count = 0;
-  MatDesc* d_desc = reinterpret_cast<MatDesc*>(sb + 256);
-  // Pageable source: the runtime stages the 48 bytes before returning, so `d` may go out of scope.
-  if (cudaMemcpyAsync(d_desc, &d, sizeof(d), cudaMemcpyHostToDevice, st) != cudaSuccess) return MUON_ERR_CUDA;
+  // The descriptor and the problem tables reach the device as kernel arguments (no copy whose host source could
+  // go out of scope, no staging buffer).
+  MatDesc* d_desc = reinterpret_cast<MatDesc*>(sb + kStaticDescOff);
+  if (launch_poke(d_desc, &d, sizeof(d), st) < 0) return MUON_ERR_CUDA;
+  SetImage img;
+  const bool grouped = grouped_engine(&ctx);
+  if (grouped) {
+    rc = build_set_image(encode, ctx.ws, chunks, set, sb + kStaticTablesOff, &img, nullptr);
+    if (rc != MUON_OK) return rc;
+    if (img.bytes.size() > kStaticHeader - kStaticTablesOff) return MUON_ERR_TOO_LARGE;
+    img.bytes.resize((img.bytes.size() + 15) / 16 * 16, 0);
+    for (size_t off = 0; off < img.bytes.size(); off += 3072)
+      if (launch_poke(sb + kStaticTablesOff + off, img.bytes.data() + off, std::min<size_t>(3072, img.bytes.size() - off), st) < 0)
+        return MUON_ERR_CUDA;
+  }
   ChunkRun r{0, (flags & MUON_ORTHO_NO_NORMALIZE) ? 0 : 1, 0.f, 0.f, 0.f, ns_steps, coeffs};
-  return run_chunk(&ctx, ch, d_desc, r, st);
+  SetRun sr;
+  sr.chunks = &chunks;
+  sr.set = &set;
+  sr.tables = grouped ? &img.tables : nullptr;
+  sr.d_descs = d_desc;
+  sr.d_segs = nullptr;
+  sr.pitch8 = cols % 8 == 0;
+  sr.flat_vec = 8;
+  return run_set(&ctx, sr, r, st);
 }
-

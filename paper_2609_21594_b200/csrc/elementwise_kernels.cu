@@ -7,6 +7,7 @@
 // All three are HBM-bound.  Reductions use a fixed shuffle/shared-memory tree and per-tile
 // partial sums, never floating-point atomics, so results are bit-identical run to run.
 #include <algorithm>
+#include <cstring>
 
 #include "internal.h"
 
@@ -79,22 +80,41 @@ __device__ __forceinline__ float block_sum_256(float v, float* red) {
   return t;  // valid in thread 0
 }
 
+// Which shape group of the launch a block belongs to, and where inside it.
+struct BlockPos {
+  int ci, mat_local, tile;
+};
+template <typename Args>
+__device__ __forceinline__ BlockPos locate_block(const Args& a) {
+  int ci = 0;
+  for (int i = 1; i < a.nchunks; ++i)
+    if (int(blockIdx.x) >= a.ch[i].block_begin) ci = i;
+  const int local = int(blockIdx.x) - a.ch[ci].block_begin;
+  BlockPos p;
+  p.ci = ci;
+  p.mat_local = local / a.ch[ci].tiles;
+  p.tile = local - p.mat_local * a.ch[ci].tiles;
+  return p;
+}
+
 // GT: gradient/input element type; XT: NS element type; MOM: momentum rule on/off.
 // Thread (ty = tid/16, tx = tid%16) handles 4 consecutive columns tx*4.. of rows ty, ty+16, ty+32, ty+48.
 template <typename GT, typename XT, bool MOM, bool FLAT>
 __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
   __shared__ XT tile[T][PADT];
   __shared__ float red[8];
-  const int mat = blockIdx.x / a.tiles_per_mat;
-  const int t = blockIdx.x - mat * a.tiles_per_mat;
-  const MatDesc d = a.descs[mat];
+  const BlockPos bp = locate_block(a);
+  const ElemChunk ch = a.ch[bp.ci];
+  const int t = bp.tile, ldx = ch.ldx;
+  const MatDesc d = a.descs[ch.desc_begin + bp.mat_local];
   const int tiles_c = (d.cols + T - 1) / T;
   const int r0 = (t / tiles_c) * T, c0 = (t % tiles_c) * T;
   const GT* __restrict__ G = static_cast<const GT*>(d.g);
   float* __restrict__ M = static_cast<float*>(d.m);
-  XT* __restrict__ X = static_cast<XT*>(a.x) + size_t(mat) * a.s * a.ldx;
+  XT* __restrict__ X = reinterpret_cast<XT*>(a.ws + ch.x_off) + size_t(bp.mat_local) * ch.s * ldx;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  const bool vec = ((d.cols | int(d.ld)) & 3) == 0;
+  // 16-byte (fp32) / 8-byte (bf16) accesses need columns, pitch and, in flat-shard mode, every segment offset in fours
+  const bool vec = ((d.cols | int(d.ld)) & 3) == 0 && (!FLAT || a.flat_vec >= 4);
   float sum = 0.f;
   RowCursor<FLAT> cur;
   cur.init(d, a.segs, min(r0 + ty, d.rows - 1));
@@ -151,7 +171,7 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
         if (i < nv) sum += q * q;
       }
       if (!d.transposed) {
-        XT* dst = X + size_t(r) * a.ldx + c;   // ldx % 8 == 0 and c % 4 == 0: 8/16-byte aligned
+        XT* dst = X + size_t(r) * ldx + c;     // ldx % 8 == 0 and c % 4 == 0: 8/16-byte aligned
         if (nv == 4) {
           if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(xv);
           else *reinterpret_cast<float4*>(dst) = *reinterpret_cast<const float4*>(xv);
@@ -175,7 +195,7 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
         alignas(16) XT xv[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) xv[i] = tile[rr + i][cc];
-        XT* dst = X + size_t(c) * a.ldx + r;
+        XT* dst = X + size_t(c) * ldx + r;
         const int nv = min(4, d.rows - r);
         if (nv == 4) {
           if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(xv);
@@ -187,23 +207,30 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
     }
   }
   const float tot = block_sum_256(sum, red);
-  if (threadIdx.x == 0) a.partials[blockIdx.x] = tot;
+  if (threadIdx.x == 0) a.partials[ch.part_off + int64_t(bp.mat_local) * ch.tiles + t] = tot;
 }
 
-// One block per matrix: fixed-order sum of the tile partials in double, then r = 1/(sqrt(.)+eps).
-__global__ void __launch_bounds__(256) norm_kernel(const float* __restrict__ partials, float* __restrict__ rnorm,
-                                                   int tiles_per_mat, float eps, int normalize) {
+// One block per matrix of the launch: fixed-order sum of the tile partials in double, then r = 1/(sqrt(.)+eps).
+__global__ void __launch_bounds__(256) norm_kernel(StageArgs a) {
   __shared__ double red[256];
-  const float* p = partials + size_t(blockIdx.x) * tiles_per_mat;
+  int ci = 0, first = 0;
+  for (int i = 0; i < a.nchunks; ++i) {
+    if (int(blockIdx.x) >= first + a.ch[i].count) first += a.ch[i].count;
+    else { ci = i; break; }
+  }
+  const ElemChunk ch = a.ch[ci];
+  const int mat_local = int(blockIdx.x) - first;
+  const float* p = a.partials + ch.part_off + int64_t(mat_local) * ch.tiles;
   double acc = 0.0;
-  for (int i = threadIdx.x; i < tiles_per_mat; i += 256) acc += double(p[i]);
+  for (int i = threadIdx.x; i < ch.tiles; i += 256) acc += double(p[i]);
   red[threadIdx.x] = acc;
   __syncthreads();
   for (int o = 128; o > 0; o >>= 1) {
     if (int(threadIdx.x) < o) red[threadIdx.x] += red[threadIdx.x + o];
     __syncthreads();
   }
-  if (threadIdx.x == 0) rnorm[blockIdx.x] = normalize ? float(1.0 / (sqrt(red[0]) + double(eps))) : 1.0f;
+  if (threadIdx.x == 0)
+    a.rnorm[ch.desc_begin + mat_local] = a.normalize ? float(1.0 / (sqrt(red[0]) + double(a.eps))) : 1.0f;
 }
 
 // XT: NS element type; UPD: 1 = weight update, 0 = plain store of O into d.w (element type XT).
@@ -212,15 +239,16 @@ __global__ void __launch_bounds__(256) norm_kernel(const float* __restrict__ par
 template <typename XT, bool UPD, bool FLAT>
 __global__ void __launch_bounds__(256, FLAT ? 5 : 6) apply_kernel(ApplyArgs a) {
   __shared__ XT tile[T][PADT];
-  const int mat = blockIdx.x / a.tiles_per_mat;
-  const int t = blockIdx.x - mat * a.tiles_per_mat;
-  const MatDesc d = a.descs[mat];
+  const BlockPos bp = locate_block(a);
+  const ElemChunk ch = a.ch[bp.ci];
+  const int t = bp.tile, ldx = ch.ldx;
+  const MatDesc d = a.descs[ch.desc_begin + bp.mat_local];
   const int tiles_c = (d.cols + T - 1) / T;
   const int r0 = (t / tiles_c) * T, c0 = (t % tiles_c) * T;
-  const XT* __restrict__ X = static_cast<const XT*>(a.x) + size_t(mat) * a.s * a.ldx;
+  const XT* __restrict__ X = reinterpret_cast<const XT*>(a.ws + ch.x_off) + size_t(bp.mat_local) * ch.s * ldx;
   float* __restrict__ W = static_cast<float*>(d.w);
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  const bool vec = ((d.cols | int(d.ld)) & 3) == 0;
+  const bool vec = ((d.cols | int(d.ld)) & 3) == 0 && (!FLAT || a.flat_vec >= 4);
   const int cc = tx * 4, c = c0 + cc;
   const int nv = min(4, d.cols - c);
   float w[4][4];
@@ -260,7 +288,7 @@ __global__ void __launch_bounds__(256, FLAT ? 5 : 6) apply_kernel(ApplyArgs a) {
       const int cc2 = ty + pass * 16, rr = tx * 4;
       const int c2 = c0 + cc2, r = r0 + rr;
       if (c2 < d.cols && r < d.rows) {
-        const XT* src = X + size_t(c2) * a.ldx + r;
+        const XT* src = X + size_t(c2) * ldx + r;
         const int nr = min(4, d.rows - r);
         alignas(16) XT tv[4];
         if (nr == 4) {
@@ -287,7 +315,7 @@ __global__ void __launch_bounds__(256, FLAT ? 5 : 6) apply_kernel(ApplyArgs a) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) xv[pass][i] = XConv<XT>::from(0.f);
       if (r < d.rows && nv > 0) {
-        const XT* src = X + size_t(r) * a.ldx + c;
+        const XT* src = X + size_t(r) * ldx + c;
         if (nv == 4) {
           if (sizeof(XT) == 2) *reinterpret_cast<uint2*>(xv[pass]) = __ldcs(reinterpret_cast<const uint2*>(src));
           else *reinterpret_cast<float4*>(xv[pass]) = __ldcs(reinterpret_cast<const float4*>(src));
@@ -360,19 +388,20 @@ __device__ __forceinline__ uint32_t wide_tile_addr(int c_local, int r_local) {  
 __host__ __device__ inline int wide_tiles(int rows, int cols) { return ((rows + WR - 1) / WR) * ((cols + WC - 1) / WC); }
 
 template <typename GT, bool MOM, bool FLAT>
-__global__ void __launch_bounds__(256, 6) stage_wide_kernel(StageArgs a, int tiles_wide) {
+__global__ void __launch_bounds__(256, 6) stage_wide_kernel(StageArgs a) {
   __shared__ __align__(16) unsigned char tsm[WC * 128];
   __shared__ float red[8];
-  const int mat = blockIdx.x / tiles_wide;
-  const int t = blockIdx.x - mat * tiles_wide;
-  const MatDesc d = a.descs[mat];
+  const BlockPos bp = locate_block(a);
+  const ElemChunk ch = a.ch[bp.ci];
+  const int t = bp.tile, ldx = ch.ldx;
+  const MatDesc d = a.descs[ch.desc_begin + bp.mat_local];
   const int tiles_c = (d.cols + WC - 1) / WC;
   float sum = 0.f;
   if (t < wide_tiles(d.rows, d.cols)) {                      // block-uniform: the grid is sized for the larger orientation
     const int r0 = (t / tiles_c) * WR, c0 = (t % tiles_c) * WC;
     const GT* __restrict__ G = static_cast<const GT*>(d.g);
     float* __restrict__ M = static_cast<float*>(d.m);
-    __nv_bfloat16* __restrict__ X = static_cast<__nv_bfloat16*>(a.x) + size_t(mat) * a.s * a.ldx;
+    __nv_bfloat16* __restrict__ X = reinterpret_cast<__nv_bfloat16*>(a.ws + ch.x_off) + size_t(bp.mat_local) * ch.s * ldx;
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     const int c = c0 + 8 * tx;
     RowCursor<FLAT> cur;
@@ -419,7 +448,7 @@ __global__ void __launch_bounds__(256, 6) stage_wide_kernel(StageArgs a, int til
             sum += q1 * q1;
           }
           if (!d.transposed) {
-            *reinterpret_cast<uint4*>(X + size_t(r) * a.ldx + c) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            *reinterpret_cast<uint4*>(X + size_t(r) * ldx + c) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -437,24 +466,25 @@ __global__ void __launch_bounds__(256, 6) stage_wide_kernel(StageArgs a, int til
         const int oc = (threadIdx.x >> 3) + 32 * pass, og = threadIdx.x & 7;
         const int cc = c0 + oc, r = r0 + 8 * og;
         if (cc < d.cols && r < d.rows)
-          *reinterpret_cast<uint4*>(X + size_t(cc) * a.ldx + r) = *reinterpret_cast<const uint4*>(tsm + wide_tile_addr(oc, 8 * og));
+          *reinterpret_cast<uint4*>(X + size_t(cc) * ldx + r) = *reinterpret_cast<const uint4*>(tsm + wide_tile_addr(oc, 8 * og));
       }
     }
   }
   const float tot = block_sum_256(sum, red);
-  if (threadIdx.x == 0) a.partials[blockIdx.x] = tot;
+  if (threadIdx.x == 0) a.partials[ch.part_off + int64_t(bp.mat_local) * ch.tiles + t] = tot;
 }
 
 template <bool UPD, bool FLAT>
-__global__ void __launch_bounds__(256) apply_wide_kernel(ApplyArgs a, int tiles_wide) {
+__global__ void __launch_bounds__(256, 6) apply_wide_kernel(ApplyArgs a) {
   __shared__ __align__(16) unsigned char tsm[WC * 128];
-  const int mat = blockIdx.x / tiles_wide;
-  const int t = blockIdx.x - mat * tiles_wide;
-  const MatDesc d = a.descs[mat];
+  const BlockPos bp = locate_block(a);
+  const ElemChunk ch = a.ch[bp.ci];
+  const int t = bp.tile, ldx = ch.ldx;
+  const MatDesc d = a.descs[ch.desc_begin + bp.mat_local];
   if (t >= wide_tiles(d.rows, d.cols)) return;               // block-uniform
   const int tiles_c = (d.cols + WC - 1) / WC;
   const int r0 = (t / tiles_c) * WR, c0 = (t % tiles_c) * WC;
-  const __nv_bfloat16* __restrict__ X = static_cast<const __nv_bfloat16*>(a.x) + size_t(mat) * a.s * a.ldx;
+  const __nv_bfloat16* __restrict__ X = reinterpret_cast<const __nv_bfloat16*>(a.ws + ch.x_off) + size_t(bp.mat_local) * ch.s * ldx;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   const int c = c0 + 8 * tx;
   const bool col_ok = c < d.cols;
@@ -474,7 +504,7 @@ __global__ void __launch_bounds__(256) apply_wide_kernel(ApplyArgs a, int tiles_
       const int oc = (threadIdx.x >> 3) + 32 * pass, og = threadIdx.x & 7;
       const int cc = c0 + oc, r = r0 + 8 * og;
       if (cc < d.cols && r < d.rows)
-        *reinterpret_cast<uint4*>(tsm + wide_tile_addr(oc, 8 * og)) = __ldcs(reinterpret_cast<const uint4*>(X + size_t(cc) * a.ldx + r));
+        *reinterpret_cast<uint4*>(tsm + wide_tile_addr(oc, 8 * og)) = __ldcs(reinterpret_cast<const uint4*>(X + size_t(cc) * ldx + r));
     }
     __syncthreads();
   }
@@ -486,7 +516,7 @@ __global__ void __launch_bounds__(256) apply_wide_kernel(ApplyArgs a, int tiles_
     if (!col_ok || r >= d.rows) continue;
     uint32_t pk[4];
     if (!d.transposed) {
-      const uint4 v = __ldcs(reinterpret_cast<const uint4*>(X + size_t(r) * a.ldx + c));
+      const uint4 v = __ldcs(reinterpret_cast<const uint4*>(X + size_t(r) * ldx + c));
       pk[0] = v.x; pk[1] = v.y; pk[2] = v.z; pk[3] = v.w;
     } else {
 #pragma unroll
@@ -547,33 +577,52 @@ static void launch_stage_t(const StageArgs& a, unsigned g, cudaStream_t st) {
 }
 
 template <bool FLAT>
-static void launch_stage_wide_t(const StageArgs& a, unsigned g, int tw, cudaStream_t st) {
+static void launch_stage_wide_t(const StageArgs& a, unsigned g, cudaStream_t st) {
   if (a.momentum) {
-    if (a.grad_dtype == MUON_DTYPE_BF16) stage_wide_kernel<__nv_bfloat16, true, FLAT><<<g, 256, 0, st>>>(a, tw);
-    else stage_wide_kernel<float, true, FLAT><<<g, 256, 0, st>>>(a, tw);
+    if (a.grad_dtype == MUON_DTYPE_BF16) stage_wide_kernel<__nv_bfloat16, true, FLAT><<<g, 256, 0, st>>>(a);
+    else stage_wide_kernel<float, true, FLAT><<<g, 256, 0, st>>>(a);
   } else {
-    stage_wide_kernel<__nv_bfloat16, false, FLAT><<<g, 256, 0, st>>>(a, tw);
+    stage_wide_kernel<__nv_bfloat16, false, FLAT><<<g, 256, 0, st>>>(a);
   }
 }
 
 // Tiles per matrix of the wide kernels: a chunk mixes both orientations of its core shape, the grid takes the larger count.
 static int wide_tiles_of_chunk(int s, int l) { return std::max(wide_tiles(s, l), wide_tiles(l, s)); }
 
-int launch_stage(const StageArgs& a, cudaStream_t st) {
-  const bool wide = a.wide && a.ns_precision == MUON_NS_BF16;
-  const int tiles = wide ? wide_tiles_of_chunk(a.s, a.l) : a.tiles_per_mat;
-  const int64_t blocks = int64_t(a.count) * tiles;
+// Fills block_begin / tiles of every shape group of the launch; returns the grid size or < 0.
+template <typename Args>
+static int64_t finish_chunks(Args* a, bool wide) {
+  int64_t blocks = 0;
+  int matrices = 0;
+  for (int i = 0; i < a->nchunks; ++i) {
+    ElemChunk& c = a->ch[i];
+    c.tiles = wide ? wide_tiles_of_chunk(c.s, c.l) : ((c.s + T - 1) / T) * ((c.l + T - 1) / T);
+    if (blocks > 0x7fffffffLL) return -1;
+    c.block_begin = int32_t(blocks);
+    blocks += int64_t(c.count) * c.tiles;
+    matrices += c.count;
+  }
+  return blocks > 0x7fffffffLL ? -1 : blocks;
+}
+
+int launch_stage(const StageArgs& a0, cudaStream_t st) {
+  StageArgs a = a0;
+  if (a.nchunks < 1 || a.nchunks > kMaxElemChunks) return MUON_ERR_INVALID_ARG;
+  const bool wide = a.wide && a.ns_precision == MUON_NS_BF16 && (!a.segs || a.flat_vec >= 8);
+  const int64_t blocks = finish_chunks(&a, wide);
+  if (blocks < 0) return MUON_ERR_UNSUPPORTED;
   if (blocks == 0) return 0;
-  if (blocks > 0x7fffffffLL) return MUON_ERR_UNSUPPORTED;
   if (wide) {
-    if (a.segs) launch_stage_wide_t<true>(a, unsigned(blocks), tiles, st);
-    else launch_stage_wide_t<false>(a, unsigned(blocks), tiles, st);
+    if (a.segs) launch_stage_wide_t<true>(a, unsigned(blocks), st);
+    else launch_stage_wide_t<false>(a, unsigned(blocks), st);
   } else {
     if (a.segs) launch_stage_t<true>(a, unsigned(blocks), st);
     else launch_stage_t<false>(a, unsigned(blocks), st);
   }
   if (cudaGetLastError() != cudaSuccess) return MUON_ERR_CUDA;
-  norm_kernel<<<unsigned(a.count), 256, 0, st>>>(a.partials, a.rnorm, tiles, a.eps, a.normalize);
+  int matrices = 0;
+  for (int i = 0; i < a.nchunks; ++i) matrices += a.ch[i].count;
+  norm_kernel<<<unsigned(matrices), 256, 0, st>>>(a);
   return cudaGetLastError() == cudaSuccess ? 2 : MUON_ERR_CUDA;
 }
 
@@ -589,25 +638,44 @@ static void launch_apply_t(const ApplyArgs& a, unsigned g, cudaStream_t st) {
   }
 }
 
-int launch_apply(const ApplyArgs& a, cudaStream_t st) {
-  const bool wide = a.wide && a.ns_precision == MUON_NS_BF16;
-  const int tiles = wide ? wide_tiles_of_chunk(a.s, a.l) : a.tiles_per_mat;
-  const int64_t blocks = int64_t(a.count) * tiles;
+int launch_apply(const ApplyArgs& a0, cudaStream_t st) {
+  ApplyArgs a = a0;
+  if (a.nchunks < 1 || a.nchunks > kMaxElemChunks) return MUON_ERR_INVALID_ARG;
+  const bool wide = a.wide && a.ns_precision == MUON_NS_BF16 && (!a.segs || a.flat_vec >= 8);
+  const int64_t blocks = finish_chunks(&a, wide);
+  if (blocks < 0) return MUON_ERR_UNSUPPORTED;
   if (blocks == 0) return 0;
-  if (blocks > 0x7fffffffLL) return MUON_ERR_UNSUPPORTED;
   const unsigned g = unsigned(blocks);
   if (wide) {
     if (a.update) {
-      if (a.segs) apply_wide_kernel<true, true><<<g, 256, 0, st>>>(a, tiles);
-      else apply_wide_kernel<true, false><<<g, 256, 0, st>>>(a, tiles);
+      if (a.segs) apply_wide_kernel<true, true><<<g, 256, 0, st>>>(a);
+      else apply_wide_kernel<true, false><<<g, 256, 0, st>>>(a);
     } else {
-      if (a.segs) apply_wide_kernel<false, true><<<g, 256, 0, st>>>(a, tiles);
-      else apply_wide_kernel<false, false><<<g, 256, 0, st>>>(a, tiles);
+      if (a.segs) apply_wide_kernel<false, true><<<g, 256, 0, st>>>(a);
+      else apply_wide_kernel<false, false><<<g, 256, 0, st>>>(a);
     }
   } else {
     if (a.segs) launch_apply_t<true>(a, g, st);
     else launch_apply_t<false>(a, g, st);
   }
+  return cudaGetLastError() == cudaSuccess ? 1 : MUON_ERR_CUDA;
+}
+
+// ---- poke: small host data -> device memory, carried by the kernel's argument buffer
+struct PokeBlob {
+  uint4 v[192];      // 3 KiB
+};
+__global__ void __launch_bounds__(192) poke_kernel(uint4* dst, const PokeBlob b, int n16) {
+  if (int(threadIdx.x) < n16) dst[threadIdx.x] = b.v[threadIdx.x];
+}
+
+int launch_poke(void* dst, const void* src, size_t bytes, cudaStream_t st) {
+  if (bytes == 0) return 0;
+  if (bytes > sizeof(PokeBlob) || (reinterpret_cast<uintptr_t>(dst) & 15u)) return MUON_ERR_INVALID_ARG;
+  PokeBlob b;
+  std::memset(&b, 0, sizeof(b));
+  std::memcpy(&b, src, bytes);
+  poke_kernel<<<1, 192, 0, st>>>(static_cast<uint4*>(dst), b, int((bytes + 15) / 16));
   return cudaGetLastError() == cudaSuccess ? 1 : MUON_ERR_CUDA;
 }
 

@@ -36,30 +36,50 @@ struct alignas(16) RowSeg {
   int64_t flat_offset;
 };
 
-// One batched Newton-Schulz invocation: `count` matrices of one core shape (s <= l).
+// One shape group's share of a batched Newton-Schulz invocation: `count` matrices of one core shape (s <= l).
 struct Chunk {
-  int32_t s, l;          // core shape: s = min(rows, cols), l = max(rows, cols)
-  int32_t ldx, lda;      // leading dimensions (elements) of X [s x ldx] and of A, B [s x lda]
-  int32_t count;
-  int32_t tiles_per_mat; // elementwise 64x64 tiles per matrix
-  int32_t desc_begin;    // index of the first MatDesc of this chunk in the uploaded table
-  std::vector<int32_t> mats;  // caller indices, in caller order
+  int32_t s = 0, l = 0;  // core shape: s = min(rows, cols), l = max(rows, cols)
+  int32_t ldx = 0, lda = 0;      // leading dimensions (elements) of X [s x ldx] and of A, B [s x lda]
+  int32_t count = 0;
+  int32_t tiles_per_mat = 0;     // elementwise 64x64 tiles per matrix
+  int32_t desc_begin = 0;        // index of the first MatDesc of this chunk in the uploaded table
+  int32_t set = 0;               // launch set this chunk belongs to
+  size_t off_x[2] = {0, 0}, off_a = 0, off_b = 0;   // byte offsets of the chunk's buffers in the workspace
+  int64_t part_off = 0;          // float index of the chunk's tile partial sums inside the set's partial-sum area
+  std::vector<int32_t> mats;     // caller indices, in caller order
 };
+
+// Chunks that are resident in the workspace together (at most chunk_elems elements in total): every
+// product of a Newton-Schulz step is ONE launch over all of them.
+struct LaunchSet {
+  std::vector<int32_t> chunks;      // indices into Plan::chunks; their MatDescs are contiguous
+  int32_t desc_begin = 0, count = 0;
+  size_t off_partials = 0, off_rnorm = 0, bytes = 0;
+  int64_t elems = 0;
+};
+
+struct SetTables;   // tensor-core tables of one launch set (tc_tables.h)
 
 struct Plan {
   std::vector<Chunk> chunks;
+  std::vector<LaunchSet> sets;
   size_t ws_bytes = 0;
   int32_t live = 0;      // matrices with rows > 0 and cols > 0
-};
-
-// Carving of the caller's workspace for the largest chunk.
-struct WsCarve {
-  size_t x0, x1, a, b, partials, rnorm, total;
+  // tensor-core tables: built when the plan first runs on a workspace, rebuilt when the workspace moves
+  void* d_tables = nullptr;
+  const void* tables_ws = nullptr;
+  std::vector<SetTables>* set_tables = nullptr;   // owned; one entry per launch set
 };
 
 size_t elem_bytes_of_ns(int ns_precision);
 int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t count, Plan* plan);
-WsCarve carve_chunk(const muon_options_t& opt, const Chunk& c);
+// Lays the chunks of one launch set out in a workspace (fills Chunk::off_*, part_off and the set's offsets).
+void layout_set(const muon_options_t& opt, std::vector<Chunk>* chunks, LaunchSet* set);
+// Tile list of a symmetric product over nb x nb blocks of 128: every unordered pair of blocks exactly once.
+struct TilePatHost {
+  uint16_t ra, rb, cc, cd;
+};
+std::vector<TilePatHost> symmetric_tile_pattern(int nb);
 int validate_layout_host(const muon_layout_desc_t* d);
 
 // Copy work item of the gather/scatter kernel.
@@ -94,6 +114,7 @@ struct muon_layout {
   int device = 0;
   std::vector<std::vector<muon_segment_t>> segs_of;   // host copy of the segment table, grouped by matrix
   bool row_aligned = false;                           // every segment holds whole rows: the flat buffers can be addressed in place
+  int32_t flat_vec = 1;                               // largest of 8, 4, 1 that divides every row segment's flat offset
   muon::RowSeg* d_rowsegs = nullptr;                  // device, all matrices' row segments, sorted by row inside a matrix
   std::vector<int32_t> rowseg_begin, rowseg_count;    // per matrix: its range in d_rowsegs
 };
@@ -113,6 +134,7 @@ struct muon_ctx {
   double phase_ms[MUON_NUM_PHASES] = {0, 0, 0, 0, 0};
   int64_t phase_launches[MUON_NUM_PHASES] = {0, 0, 0, 0, 0};
   int64_t launches = 0;
+  int64_t tmap_encodes = 0;                        // tensor maps encoded so far (plan binding and the per-launch engines)
   void* tmap_encode = nullptr;                     // cuTensorMapEncodeTiled, resolved at run time
   cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;   // copy streams of the host-buffer path (created on first use)
   std::vector<cudaEvent_t> sync_events;            // untimed events that order the copy streams against the caller's stream
@@ -125,33 +147,53 @@ namespace muon {
 int launch_copy(const CopyItem* items, int64_t num_items, void* flat, void* const* d_mats, int elem_size,
                 bool scatter, cudaStream_t st);
 
+// One shape group inside an elementwise launch.
+struct ElemChunk {
+  int32_t block_begin;   // first block of this chunk in the launch
+  int32_t tiles;         // blocks per matrix
+  int32_t desc_begin;    // first MatDesc / rnorm entry, relative to the launch set
+  int32_t count;
+  int32_t s, l, ldx, pad;
+  int64_t x_off;         // byte offset in the workspace of the X iterate this launch writes (stage) or reads (apply)
+  int64_t part_off;      // float index of the chunk's partial sums
+};
+constexpr int kMaxElemChunks = 8;
+
 struct StageArgs {
   const RowSeg* segs;     // device row-segment table (flat-shard mode), else null
-  const MatDesc* descs;   // device, first record of the chunk
-  void* x;                // device, chunk X buffer (bf16 or fp32)
-  float* partials;        // device, count*tiles_per_mat
-  float* rnorm;           // device, count
-  int32_t count, tiles_per_mat, s, l, ldx;
+  const MatDesc* descs;   // device, first record of the launch set
+  char* ws;               // device, workspace base
+  float* partials;        // device, the set's partial sums
+  float* rnorm;           // device, one per matrix of the set
   float mu, eps;
   int32_t nesterov, grad_dtype, ns_precision;
   int32_t momentum;       // 1: full momentum rule; 0: plain staging of the input (orthogonalize)
   int32_t normalize;      // 0: rnorm = 1
   int32_t wide;           // 1: rows, cols and every row pitch are multiples of 8: the 8-elements-per-thread kernels apply
+  int32_t flat_vec;       // flat-shard mode: every segment offset is a multiple of this many elements (8, 4 or 1)
+  int32_t nchunks;
+  ElemChunk ch[kMaxElemChunks];
 };
 int launch_stage(const StageArgs& a, cudaStream_t st);
 
 struct ApplyArgs {
   const RowSeg* segs;     // device row-segment table (flat-shard mode), else null
   const MatDesc* descs;
-  const void* x;          // final NS iterate
-  int32_t count, tiles_per_mat, s, l, ldx;
+  const char* ws;
   float lr, wd;
   float decay;            // 1 - lr*wd, computed once on the host so that every update route uses the same value
   int32_t ns_precision;
   int32_t update;         // 1: W <- W(1-lr*wd) - lr*scale*O ; 0: write O into descs[i].w in the NS element type
   int32_t wide;           // as in StageArgs
+  int32_t flat_vec;
+  int32_t nchunks;
+  ElemChunk ch[kMaxElemChunks];
 };
 int launch_apply(const ApplyArgs& a, cudaStream_t st);
+
+// Writes up to 3 KiB of host data into device memory with a kernel (the data travels as a kernel argument):
+// no staging buffer, no host-to-device copy that could outlive its source.
+int launch_poke(void* dst, const void* src, size_t bytes, cudaStream_t st);
 
 // C[k] = gamma_k * (beta * D[k] + alpha * op(P[k], Q[k])),  op = P Q^T (nn=0) or P Q (nn=1)
 struct GemmArgs {
@@ -167,10 +209,8 @@ struct GemmArgs {
   int32_t symmetric;   // op is P P^T with symmetric result (kernels may exploit it)
 };
 int launch_gemm_simt(const GemmArgs& a, int ns_precision, cudaStream_t st);
-int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st);   // tcgen05 engine (bf16 only)
+int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st);   // tcgen05 engine, single-CTA kernel (bf16 only)
 bool tc_supported(const GemmArgs& a);
-int launch_gemm_tc_pair(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st);   // two-CTA (cta_group::2) variant
-bool tc_pair_supported(const GemmArgs& a);
 int launch_bounded_wait_probe(muon_ctx* ctx, cudaStream_t st);            // a wait that must expire (self-test)
 
 }  // namespace muon

@@ -74,7 +74,7 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;            // swizzled tiles need 1024-byte alignment
   uint8_t* gen_base = smem_raw + (base - raw);
-  const uint32_t epi_base = base + STAGES * STAGE_BYTES;    // two epilogue staging buffers follow the ring
+  const uint32_t epi_base = base + STAGES * STAGE_BYTES;    // the epilogue staging buffers follow the ring
   constexpr int BAR_OFF = STAGES * STAGE_BYTES + EPI_BUFS * EPI_BYTES;
   const uint32_t bars = base + BAR_OFF;                     // barrier block follows the buffers
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + BAR_OFF + 128);
@@ -191,19 +191,35 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
     EpilogueState est;
     uint32_t tile_it = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_it) {
-      const Tile tl = decode_tile(t, a);
-      const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-      const bool mirror = a.symmetric && tl.n0 >= tl.m0 + BM;   // tile lies strictly above the diagonal
-      const uint32_t taddr = tmem_base + acc * uint32_t(BN) + (uint32_t(quad * 32) << 16);
-      const EpiTile cur{tl.mat, tl.m0, tl.n0, true};
-      EpiTile nxt{0, 0, 0, false};
-      if (t + int(gridDim.x) < total_tiles) {
-        const Tile tn = decode_tile(t + int(gridDim.x), a);
-        nxt = EpiTile{tn.mat, tn.m0, tn.n0, true};
+    auto epi_of = [&](const Tile& tl) {
+      EpiTile e;
+      e.map_d = &map_d; e.map_c = &map_c;
+      e.d = a.d; e.c = a.c;
+      e.stride_c = a.stride_c;
+      e.ldc = a.ldc; e.m = a.m; e.n = a.n;
+      e.mat = tl.mat;
+      e.rblk = tl.m0 / BM;
+      e.cblk0 = tl.n0 / 128;
+      e.cblk1 = tl.n0 + 128 < a.n ? tl.n0 / 128 + 1 : -1;
+      e.mirror0 = e.mirror1 = a.symmetric && tl.n0 >= tl.m0 + BM;       // tile lies strictly above the diagonal
+      e.alpha = a.alpha; e.beta = a.beta; e.gamma = 1.f;
+      if (a.gamma_mode) {
+        const float r = a.rnorm[tl.mat];
+        e.gamma = a.gamma_mode == 1 ? r : r * r;
       }
-      ok = epilogue_tile(a, &map_d, &map_c, cur, nxt, mirror, taddr, epi_base, dfull_bar(0), egroup_bar, tfull_bar(int(acc)),
-                         aph, abort_flag, est, quad, lane);
+      e.valid = true;
+      return e;
+    };
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_it) {
+      const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+      const uint32_t taddr = tmem_base + acc * uint32_t(BN) + (uint32_t(quad * 32) << 16);
+      const EpiTile cur = epi_of(decode_tile(t, a));
+      EpiTile nxt;
+      nxt.valid = false;
+      nxt.d = nullptr;
+      if (t + int(gridDim.x) < total_tiles) nxt = epi_of(decode_tile(t + int(gridDim.x), a));
+      ok = epilogue_tile(cur, nxt, taddr, epi_base, dfull_bar(0), egroup_bar, tfull_bar(int(acc)), aph, abort_flag, est, quad,
+                         lane);
       if (!ok) break;
       tc_fence_before();
       __syncwarp();
@@ -292,6 +308,7 @@ int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st) {
   CUtensorMap map_c, map_d;
   if (!encode_map(ctx->tmap_encode, &map_c, a.c, a.n, a.m, a.batch, a.ldc, a.stride_c, BM)) return MUON_ERR_CUDA;
   if (!encode_map(ctx->tmap_encode, &map_d, a.d ? a.d : a.c, a.n, a.m, a.batch, a.ldc, a.stride_c, BM)) return MUON_ERR_CUDA;
+  ctx->tmap_encodes += 4;
   TcArgs t;
   t.d = static_cast<const __nv_bfloat16*>(a.d);
   t.c = static_cast<__nv_bfloat16*>(a.c);

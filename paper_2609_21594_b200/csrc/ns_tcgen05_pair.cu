@@ -1,22 +1,29 @@
-// Paired-CTA tensor-core kernel for the Newton-Schulz products (Eq. 1): the same operation as
-// ns_tcgen05.cu, computed by clusters of two CTAs that drive one tcgen05.mma.cta_group::2 of shape
-// M256 x N256 x K16 together.
+// Paired-CTA tensor-core engine for the Newton-Schulz products (Eq. 1), grouped over heterogeneous
+// shapes: ONE launch computes the same product (A = X X^T, B = bA + cA A^T or X' = aX + B X) for every
+// shape group that is resident in the workspace (the shape-fused batching of Section 6.6, taken one
+// step further: not one batched kernel per core shape but one per product for all core shapes).
 //
 //   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k]^T)   (nn = 0)      C[k] = ... P[k] Q[k]   (nn = 1)
 //
-// A pair owns a 256 x 256 output tile.  CTA r of the pair (r = 0, 1) owns rows [128 r, 128 r + 128):
-// it loads those 128 rows of P and HALF of the Q tile (128 of the 256 columns of the output) per
-// 64-wide k-block -- 32 KiB per stage instead of 48 KiB, so five stages and a three-buffer epilogue ring fit and the bytes that cross
-// L2 -> shared memory per flop drop by a third.  The leader (r = 0) issues every MMA; the hardware
-// reads each CTA's own P rows and both CTAs' Q halves.  Each CTA keeps its 128 x 256 fp32 accumulator
-// in its own TMEM (double-buffered) and runs its own epilogue.
+// The launch reads a table of problems from global memory (tensor maps encoded once per plan, shapes,
+// tile counts) and walks one global tile list with persistent clusters of two CTAs.  A tile is given in
+// 128-row / 128-column blocks: CTA r of the pair owns row block (ra, rb)[r] and loads those 128 rows of P;
+// the tile spans column blocks cc and cd (N = 256) or cc alone (N = 128), and CTA r stages half of the
+// N columns of Q per 64-wide k-block.  The leader (r = 0) issues tcgen05.mma.cta_group::2 of shape
+// M256 x N x K16; each CTA keeps its 128 x N fp32 accumulator in its own TMEM (double-buffered) and runs
+// its own epilogue.  Symmetric products (P = Q, C = C^T) come with an explicit per-matrix tile list that
+// covers every unordered pair of blocks exactly once, so no block of the triangle is computed twice and a
+// ragged last block costs a 128-wide tile instead of a 256-wide one; off-diagonal blocks are mirrored.
 //
-// Synchronisation (all waits bounded, as in the single-CTA kernel):
+// Synchronisation (all waits bounded):
 //   full[s]    leader only.  The leader's producer arms it with the bytes of BOTH CTAs; both producers'
 //              TMA loads complete on it (cta_group::2 form, no multicast).
 //   empty[s]   in each CTA; the leader's tcgen05.commit arrives on both (commit multicast).
 //   tfull[a]   in each CTA; commit multicast after a tile's last k-block.
 //   tempty[a]  leader only, 8 arrivals: the four epilogue warps of each CTA (remote arrive).
+//   drain      in each CTA; the issuer's last commit, awaited before TMEM is freed.
+// A role that gives up sets the abort flag of BOTH CTAs (remote store), records a code in the status word
+// and leaves; everybody else notices the flag inside its own bounded wait.
 #include "tc_common.cuh"
 
 namespace muon {
@@ -25,13 +32,14 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128;          // rows per CTA; the pair covers 256
-constexpr int BN = 256;          // columns of the pair's tile
-constexpr int BNH = 128;         // columns of Q each CTA stages
 constexpr int BK = 64;
 constexpr int UK = 16;
-constexpr int STAGES = 5;
-constexpr int A_BYTES = BM * BK * 2;          // 16 KiB
-constexpr int B_BYTES = BNH * BK * 2;         // 16 KiB
+#ifndef MUON_PAIR_STAGES
+#define MUON_PAIR_STAGES 5
+#endif
+constexpr int STAGES = MUON_PAIR_STAGES;
+constexpr int A_BYTES = BM * BK * 2;          // 16 KiB: this CTA's rows of P
+constexpr int B_BYTES = 128 * BK * 2;         // 16 KiB: this CTA's half of the Q tile
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BUFS * EPI_BYTES + 1024 + 256;
 constexpr int TMEM_COLS = 512;
@@ -53,6 +61,9 @@ __device__ __forceinline__ void cluster_sync_all() {
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
 }
 // TMA load whose completion bytes are credited to a barrier that may live in the peer CTA.
 __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int c0,
@@ -81,32 +92,75 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
 }
 
 struct Tile {
-  int mat, m0, n0;   // m0: first row of the PAIR's tile
+  int prob;      // index into the launch's problem list
+  int mat;
+  int ra, rb;    // row block of CTA 0 / CTA 1 (rb = -1: none)
+  int cc, cd;    // column blocks (cd = -1: the tile is 128 columns wide)
 };
-// Tiles are 256 x 256.  Dense: row blocks vary fastest.  Symmetric: block row I needs block columns J >= I.
-__device__ __forceinline__ Tile decode_tile(int t, const TcArgs& a) {
+
+__device__ __forceinline__ Tile decode_tile(int t, const TcLaunch& L) {
+  int pi = 0;
+  for (int i = 1; i < L.nprob; ++i)
+    if (t >= L.info[i].tile_begin) pi = i;
+  const TcProbInfo& p = L.info[pi];
   Tile r;
-  r.mat = t / a.tiles_per_mat;
-  int u = t - r.mat * a.tiles_per_mat;
-  if (!a.symmetric) {
-    r.n0 = (u / a.tiles_m) * BN;
-    r.m0 = (u % a.tiles_m) * (2 * BM);
-    return r;
+  r.prob = pi;
+  const int u = t - p.tile_begin;
+  r.mat = u / p.tiles_per_mat;
+  const int v = u - r.mat * p.tiles_per_mat;
+  if (p.pattern) {
+    const uint2 raw = __ldg(reinterpret_cast<const uint2*>(p.pattern + v));
+    const uint32_t ra = raw.x & 0xffffu, rb = raw.x >> 16, cc = raw.y & 0xffffu, cd = raw.y >> 16;
+    r.ra = int(ra);
+    r.rb = rb == kNoBlock ? -1 : int(rb);
+    r.cc = int(cc);
+    r.cd = cd == kNoBlock ? -1 : int(cd);
+  } else {   // dense: row pairs vary fastest, so concurrent pairs share the Q tile
+    const int j = v / p.row_pairs, i = v - j * p.row_pairs;
+    r.ra = 2 * i;
+    r.rb = 2 * i + 1 < p.rblocks ? 2 * i + 1 : -1;
+    r.cc = 2 * j;
+    r.cd = 2 * j + 1 < p.cblocks ? 2 * j + 1 : -1;
   }
-  int i = 0;
-  while (u >= a.tiles_n - i) {
-    u -= a.tiles_n - i;
-    ++i;
-  }
-  r.m0 = i * (2 * BM);
-  r.n0 = (i + u) * BN;
   return r;
 }
 
-template <bool NN>
+__device__ __forceinline__ EpiTile make_epi(const Tile& tl, int rank, const TcLaunch& L) {
+  EpiTile e;
+  const TcProbInfo& p = L.info[tl.prob];
+  e.map_d = &L.maps[tl.prob].d;
+  e.map_c = &L.maps[tl.prob].c;
+  e.d = p.d;
+  e.c = p.c;
+  e.stride_c = p.stride_c;
+  e.ldc = p.ldc; e.m = p.m; e.n = p.n;
+  e.mat = tl.mat;
+  e.rblk = rank ? tl.rb : tl.ra;
+  e.cblk0 = tl.cc; e.cblk1 = tl.cd;
+  const bool sym = p.symmetric != 0 && p.mirror_out != 0;
+  // when the whole of a symmetric result is wanted, a block (r, c) is also written as (c, r) unless it lies on
+  // the diagonal or this very tile computes (c, r) itself (the diagonal 2 x 2 tiles)
+  const bool in_cols = e.rblk == tl.cc || e.rblk == tl.cd;
+  e.mirror0 = sym && tl.cc != e.rblk && !(in_cols && (tl.cc == tl.ra || tl.cc == tl.rb));
+  e.mirror1 = sym && tl.cd != e.rblk && !(in_cols && (tl.cd == tl.ra || tl.cd == tl.rb));
+  e.valid = e.rblk >= 0;
+  e.alpha = L.alpha; e.beta = L.beta; e.gamma = 1.f;
+  if (e.valid) {
+    if (L.gamma_mode) {
+      const float r = p.rnorm[tl.mat];
+      e.gamma = L.gamma_mode == 1 ? r : r * r;
+    }
+    if (p.coef) {
+      const float* co = p.coef + size_t(tl.mat) * L.coef_stride;
+      if (L.coef_a >= 0) e.alpha = co[L.coef_a];
+      if (L.coef_b >= 0) e.beta = co[L.coef_b];
+    }
+  }
+  return e;
+}
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
-ns_product_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q,
-                       const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_c, const TcArgs a) {
+ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -122,13 +176,19 @@ ns_product_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
   auto tempty_bar = [&](int i) { return bars + uint32_t(2 * STAGES + 2 + i) * 8u; };
   auto dfull_bar = [&](int i) { return bars + uint32_t(2 * STAGES + 4 + i) * 8u; };
   const uint32_t egroup_bar = bars + uint32_t(2 * STAGES + 4 + EPI_BUFS) * 8u;
+  const uint32_t drain_bar = bars + uint32_t(2 * STAGES + 5 + EPI_BUFS) * 8u;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();
   const bool leader_cta = rank == 0;
   const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-  const int total_tiles = a.batch * a.tiles_per_mat;
-  const int num_kb = (a.kdim + BK - 1) / BK;
+  const int total_tiles = L.total_tiles;
+  const uint32_t peer_abort = map_to_cta(base + BAR_OFF + 200, rank ^ 1u);
+  auto give_up = [&](int code) {                 // tell both CTAs of the pair, then the host
+    *abort_flag = 1;
+    st_cluster_u32(peer_abort, 1u);
+    atomicExch(L.status, code);
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -141,6 +201,7 @@ ns_product_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
     }
     for (int i = 0; i < EPI_BUFS; ++i) mbar_init(dfull_bar(i), 1);
     mbar_init(egroup_bar, 4);
+    mbar_init(drain_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -161,73 +222,99 @@ ns_product_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      const int mrow = int(rank) * BM;           // this CTA's rows inside the pair's tile
-      const int ncol = int(rank) * BNH;          // this CTA's half of the Q tile
       for (int t = pair_id; t < total_tiles && ok; t += num_pairs) {
-        const Tile tl = decode_tile(t, a);
+        const Tile tl = decode_tile(t, L);
+        const TcProbInfo& p = L.info[tl.prob];
+        const TcMaps* mp = L.maps + tl.prob;
+        const bool nn = p.nn != 0;
+        const bool narrow = tl.cd < 0;
+        const int num_kb = (p.kdim + BK - 1) / BK;
+        // this CTA's 128 rows of P (a missing row block reads beyond the matrix: zero fill)
+        const int rblk = rank ? tl.rb : tl.ra;
+        const int prow = rblk >= 0 ? rblk * BM : p.rblocks * BM;
+        // this CTA's half of the N columns: a whole column block of a 256-wide tile, half a block of a 128-wide one
+        const int qcol = narrow ? tl.cc * 128 + int(rank) * 64 : (rank ? tl.cd : tl.cc) * 128;
+        const uint32_t stage_tx = narrow ? 2 * (A_BYTES + B_BYTES / 2) : 2 * STAGE_BYTES;
+        // half-stored symmetric operands: k-blocks left of the tile's own block pair are read transposed
+        const int p_flip_kb = p.p_half ? (tl.ra >> 1) * 4 : 0;      // k-blocks [0, p_flip_kb) of P come MN-major
+        const int q_flip_kb = nn ? num_kb : (p.q_half ? (tl.cc >> 1) * 4 : 0);
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = int(it % STAGES);
           const uint32_t ph = (it / STAGES) & 1u;
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t sa = base + uint32_t(s) * STAGE_BYTES, sb = sa + A_BYTES;
-          if (leader_cta) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);
+          if (leader_cta) mbar_expect_tx(full_bar(s), stage_tx);
           const uint32_t fb = map_to_cta(full_bar(s), 0);
           const int k0 = kb * BK;
-          tma_load_3d_pair(sa, &map_p, fb, k0, tl.m0 + mrow, tl.mat);
-          if (!NN) {
-            tma_load_3d_pair(sb, &map_q, fb, k0, tl.n0 + ncol, tl.mat);
-          } else {
-#pragma unroll
-            for (int j = 0; j < BNH / 64; ++j)
-              tma_load_3d_pair(sb + uint32_t(j) * (64 * BK * 2), &map_q, fb, tl.n0 + ncol + 64 * j, k0, tl.mat);
+          if (kb >= p_flip_kb) {                       // 128 rows of P x 64 k
+            tma_load_3d_pair(sa, &mp->p, fb, k0, prow, tl.mat);
+          } else {                                     // the same block read from its mirror image: 64 k-rows x 64 columns, twice
+            tma_load_3d_pair(sa, &mp->ph, fb, prow, k0, tl.mat);
+            tma_load_3d_pair(sa + 64 * BK * 2, &mp->ph, fb, prow + 64, k0, tl.mat);
+          }
+          if (kb >= q_flip_kb) {                       // 128 rows of Q, or the 64 a 128-wide tile needs
+            tma_load_3d_pair(sb, narrow ? &mp->qh : &mp->q, fb, k0, qcol, tl.mat);
+          } else {                                     // 64 k-rows x 64 columns, twice for a 256-wide tile
+            tma_load_3d_pair(sb, &mp->qh, fb, qcol, k0, tl.mat);
+            if (!narrow) tma_load_3d_pair(sb + 64 * BK * 2, &mp->qh, fb, qcol + 64, k0, tl.mat);
           }
         }
       }
-      if (!ok) {
-        *abort_flag = 1;
-        atomicExch(a.status, 11);
-      }
+      if (!ok) give_up(11);
       if (leader_cta) {   // every armed stage (both CTAs' bytes) has landed before shared memory is released
         const uint32_t issued = it;
         for (uint32_t j = (issued > STAGES ? issued - STAGES : 0); j < issued; ++j) {
           const int s = int(j % STAGES);
           const uint32_t ph = (j / STAGES) & 1u;
-          if (!mbar_wait(full_bar(s), ph, abort_flag, false, WAIT_CYCLES / 8)) atomicExch(a.status, 12);
+          if (!mbar_wait(full_bar(s), ph, abort_flag, false, WAIT_CYCLES / 8)) atomicExch(L.status, 12);
         }
       }
+      if (*abort_flag)    // loads this CTA issued for a stage the leader never armed: give them time to land
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
-    if (lane == 0 && leader_cta) {
-      constexpr uint32_t idesc = make_idesc(NN, 2 * BM, BN);
-      uint32_t it = 0, tile_it = 0;
-      bool ok = true;
-      for (int t = pair_id; t < total_tiles && ok; t += num_pairs, ++tile_it) {
-        const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-        if (!mbar_wait(tempty_bar(int(acc)), aph ^ 1u, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * uint32_t(BN);
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
-          const int s = int(it % STAGES);
-          const uint32_t ph = (it / STAGES) & 1u;
-          if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+    if (lane == 0) {
+      if (leader_cta) {
+        uint32_t it = 0, tile_it = 0;
+        bool ok = true;
+        for (int t = pair_id; t < total_tiles && ok; t += num_pairs, ++tile_it) {
+          const Tile tl = decode_tile(t, L);
+          const TcProbInfo& p = L.info[tl.prob];
+          const bool nn = p.nn != 0;
+          const int num_kb = (p.kdim + BK - 1) / BK;
+          const int umma_n = tl.cd >= 0 ? 256 : 128;
+          const int p_flip_kb = p.p_half ? (tl.ra >> 1) * 4 : 0;
+          const int q_flip_kb = nn ? num_kb : (p.q_half ? (tl.cc >> 1) * 4 : 0);
+          const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+          if (!mbar_wait(tempty_bar(int(acc)), aph ^ 1u, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = base + uint32_t(s) * STAGE_BYTES, sb = sa + A_BYTES;
+          const uint32_t d_tmem = tmem_base + acc * 256u;
+          for (int kb = 0; kb < num_kb; ++kb, ++it) {
+            const int s = int(it % STAGES);
+            const uint32_t ph = (it / STAGES) & 1u;
+            if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sa = base + uint32_t(s) * STAGE_BYTES, sb = sa + A_BYTES;
+            const bool a_mn = kb < p_flip_kb, b_mn = kb < q_flip_kb;
+            const uint32_t idesc = make_idesc(b_mn, 2 * BM, umma_n, a_mn);
 #pragma unroll
-          for (int k = 0; k < BK / UK; ++k) {
-            const uint64_t ad = make_desc(sa + uint32_t(k) * (UK * 2), 16, 1024);
-            const uint64_t bd = NN ? make_desc(sb + uint32_t(k) * (UK * 128), 64 * BK * 2, 1024)
-                                   : make_desc(sb + uint32_t(k) * (UK * 2), 16, 1024);
-            tc_mma_pair(d_tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            for (int k = 0; k < BK / UK; ++k) {
+              // K-major: 16 k = 32 bytes along a 128-byte row; MN-major: 16 k-rows of 128 bytes, 64-element chunks 8 KiB apart
+              const uint64_t ad = a_mn ? make_desc(sa + uint32_t(k) * (UK * 128), 64 * BK * 2, 1024)
+                                       : make_desc(sa + uint32_t(k) * (UK * 2), 16, 1024);
+              const uint64_t bd = b_mn ? make_desc(sb + uint32_t(k) * (UK * 128), 64 * BK * 2, 1024)
+                                       : make_desc(sb + uint32_t(k) * (UK * 2), 16, 1024);
+              tc_mma_pair(d_tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            }
+            tc_commit_pair(empty_bar(s));
           }
-          tc_commit_pair(empty_bar(s));
+          if (ok) tc_commit_pair(tfull_bar(int(acc)));
         }
-        if (ok) tc_commit_pair(tfull_bar(int(acc)));
+        if (!ok) give_up(13);
+        tc_commit_pair(drain_bar);       // arrives in both CTAs once every MMA issued above has finished
       }
-      if (!ok) {
-        *abort_flag = 1;
-        atomicExch(a.status, 13);
-      }
+      if (!mbar_wait(drain_bar, 0, abort_flag, false, WAIT_CYCLES / 8)) atomicExch(L.status, 15);
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps (per CTA: its 128 rows)
@@ -235,19 +322,27 @@ ns_product_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
     EpilogueState est;
     uint32_t tile_it = 0;
     bool ok = true;
-    for (int t = pair_id; t < total_tiles && ok; t += num_pairs, ++tile_it) {
-      const Tile tl = decode_tile(t, a);
+    bool have = pair_id < total_tiles;
+    Tile tl;
+    if (have) tl = decode_tile(pair_id, L);
+    for (int t = pair_id; have && ok; t += num_pairs, ++tile_it) {
       const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-      const bool mirror = a.symmetric && tl.n0 > tl.m0;          // pair tile strictly above the diagonal block
-      const uint32_t taddr = tmem_base + acc * uint32_t(BN) + (uint32_t(quad * 32) << 16);
-      const EpiTile cur{tl.mat, tl.m0 + int(rank) * BM, tl.n0, true};
-      EpiTile nxt{0, 0, 0, false};
-      if (t + num_pairs < total_tiles) {
-        const Tile tn = decode_tile(t + num_pairs, a);
-        nxt = EpiTile{tn.mat, tn.m0 + int(rank) * BM, tn.n0, true};
+      const uint32_t taddr = tmem_base + acc * 256u + (uint32_t(quad * 32) << 16);
+      const EpiTile cur = make_epi(tl, int(rank), L);
+      EpiTile nxt;
+      nxt.valid = false;
+      nxt.d = nullptr;
+      have = t + num_pairs < total_tiles;
+      if (have) {
+        tl = decode_tile(t + num_pairs, L);
+        nxt = make_epi(tl, int(rank), L);
       }
-      ok = epilogue_tile(a, &map_d, &map_c, cur, nxt, mirror, taddr, epi_base, dfull_bar(0), egroup_bar, tfull_bar(int(acc)),
-                         aph, abort_flag, est, quad, lane);
+      if (cur.valid) {
+        ok = epilogue_tile(cur, nxt, taddr, epi_base, dfull_bar(0), egroup_bar, tfull_bar(int(acc)), aph, abort_flag, est, quad,
+                           lane);
+      } else {                                     // no rows for this CTA: hand the accumulator straight back
+        ok = mbar_wait(tfull_bar(int(acc)), aph, abort_flag);
+      }
       if (!ok) break;
       tc_fence_before();
       __syncwarp();
@@ -258,10 +353,7 @@ ns_product_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
       if (!ok)                                      // a prefetched D chunk may still be landing: give it (bounded) time
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
     }
-    if (!ok && lane == 0) {
-      *abort_flag = 1;
-      atomicExch(a.status, 14);
-    }
+    if (!ok && lane == 0) give_up(14);
   }
   tc_fence_before();
   __syncthreads();
@@ -279,50 +371,25 @@ int g_num_sms[kMaxDevices] = {};
 
 }  // namespace
 
-bool tc_pair_supported(const GemmArgs& a) {
-  // The pair kernel pays off once a matrix has at least one full 256-row tile; smaller ones keep the single-CTA kernel.
-  return a.m > 128;
+int tc_pair_grid_setup(int device) {
+  if (device < 0 || device >= kMaxDevices) return MUON_ERR_UNSUPPORTED;
+  if (!g_num_sms[device]) {
+    if (cudaFuncSetAttribute(ns_product_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+      return MUON_ERR_CUDA;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 2) return MUON_ERR_CUDA;
+    g_num_sms[device] = sms;
+  }
+  return g_num_sms[device];
 }
 
-int launch_gemm_tc_pair(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st) {
-  if (!ctx->tmap_encode) return MUON_ERR_CUDA;
-  if (ctx->device < 0 || ctx->device >= kMaxDevices) return MUON_ERR_UNSUPPORTED;
-  if (!g_num_sms[ctx->device]) {
-    if (cudaFuncSetAttribute(ns_product_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(ns_product_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
-      return MUON_ERR_CUDA;
-    cudaDeviceProp prop;
-    if (cudaGetDeviceProperties(&prop, ctx->device) != cudaSuccess) return MUON_ERR_CUDA;
-    g_num_sms[ctx->device] = prop.multiProcessorCount;
-  }
-  CUtensorMap map_p, map_q, map_c, map_d;
-  if (!encode_map(ctx->tmap_encode, &map_p, a.p, a.kdim, a.m, a.batch, a.ldp, a.stride_p, BM)) return MUON_ERR_CUDA;
-  if (!a.nn) {
-    if (!encode_map(ctx->tmap_encode, &map_q, a.q, a.kdim, a.n, a.batch, a.ldq, a.stride_q, BNH)) return MUON_ERR_CUDA;
-  } else {
-    if (!encode_map(ctx->tmap_encode, &map_q, a.q, a.n, a.kdim, a.batch, a.ldq, a.stride_q, BK)) return MUON_ERR_CUDA;
-  }
-  if (!encode_map(ctx->tmap_encode, &map_c, a.c, a.n, a.m, a.batch, a.ldc, a.stride_c, BM)) return MUON_ERR_CUDA;
-  if (!encode_map(ctx->tmap_encode, &map_d, a.d ? a.d : a.c, a.n, a.m, a.batch, a.ldc, a.stride_c, BM)) return MUON_ERR_CUDA;
-  TcArgs t;
-  t.d = static_cast<const __nv_bfloat16*>(a.d);
-  t.c = static_cast<__nv_bfloat16*>(a.c);
-  t.m = a.m; t.n = a.n; t.kdim = a.kdim; t.ldc = a.ldc;
-  t.stride_c = a.stride_c;
-  t.batch = a.batch;
-  t.tiles_m = (a.m + 2 * BM - 1) / (2 * BM);
-  t.tiles_n = (a.n + BN - 1) / BN;
-  t.symmetric = a.symmetric ? 1 : 0;
-  t.tiles_per_mat = t.symmetric ? t.tiles_n * (t.tiles_n + 1) / 2 : t.tiles_m * t.tiles_n;
-  t.rnorm = a.rnorm;
-  t.gamma_mode = a.gamma_mode;
-  t.alpha = a.alpha; t.beta = a.beta;
-  t.status = ctx->d_status;
-  const int64_t tiles = int64_t(t.tiles_per_mat) * t.batch;
-  const int64_t pairs = g_num_sms[ctx->device] / 2;
-  const unsigned grid = unsigned(2 * (tiles < pairs ? tiles : pairs));
-  if (a.nn) ns_product_pair_kernel<true><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, map_d, map_c, t);
-  else ns_product_pair_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_p, map_q, map_d, map_c, t);
+int launch_tc_grouped(int device, const tc::TcLaunch& L, cudaStream_t st) {
+  if (L.total_tiles <= 0) return 0;
+  const int sms = tc_pair_grid_setup(device);
+  if (sms < 0) return sms;
+  const int64_t pairs = sms / 2;
+  const unsigned grid = unsigned(2 * (L.total_tiles < pairs ? L.total_tiles : pairs));
+  ns_product_pair_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(L);
   return cudaGetLastError() == cudaSuccess ? 1 : MUON_ERR_CUDA;
 }
 

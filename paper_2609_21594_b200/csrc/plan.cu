@@ -1,5 +1,6 @@
 // Host-side planning: shape-fused batching (Section 6.6), workspace carving, layout validation.
 #include <algorithm>
+#include <iterator>
 #include <map>
 #include <numeric>
 
@@ -14,9 +15,13 @@ size_t elem_bytes_of_ns(int ns_precision) { return ns_precision == MUON_NS_FP32 
 // Matrices sharing a core shape (s, l) form one group (tensors of shape [A,B], [A,1,B], [N,A,B]
 // share the (A,B) group, Section 6.6); a tall matrix joins the group of its transpose because the
 // iteration runs on the transpose anyway.  Each group is cut into chunks of at most chunk_elems
-// elements (the 2^29-element batching cap of Section 6.6), never fewer than one matrix.
+// elements (the 2^29-element batching cap of Section 6.6), never fewer than one matrix.  Chunks are
+// then packed into launch sets of at most chunk_elems elements in total (first fit, largest chunk
+// first): the chunks of a set are resident in the workspace together and share every launch, so a
+// set -- not a chunk -- is the unit the cap bounds.
 int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t count, Plan* plan) {
   plan->chunks.clear();
+  plan->sets.clear();
   plan->ws_bytes = 0;
   plan->live = 0;
   std::map<std::pair<int32_t, int32_t>, std::vector<int32_t>> groups;
@@ -35,7 +40,7 @@ int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t co
     plan->live++;
   }
   const int64_t cap = opt.chunk_elems > 0 ? opt.chunk_elems : (int64_t(1) << 29);
-  int32_t desc_begin = 0;
+  std::vector<Chunk> chunks;
   for (const auto& key : order) {
     const std::vector<int32_t>& idx = groups[key];
     const int64_t per = int64_t(key.first) * key.second;
@@ -57,28 +62,98 @@ int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t co
       ch.count = int32_t(ch.mats.size());
       const int32_t ts = (ch.s + kElemTile - 1) / kElemTile, tl = (ch.l + kElemTile - 1) / kElemTile;
       ch.tiles_per_mat = ts * tl;
+      chunks.push_back(std::move(ch));
+    }
+  }
+  // first-fit decreasing into launch sets (stable for equal sizes, so the result is a pure function of the shape list)
+  auto elems_of = [](const Chunk& c) { return int64_t(c.count) * c.s * c.l; };
+  std::vector<size_t> by_size(chunks.size());
+  std::iota(by_size.begin(), by_size.end(), size_t(0));
+  std::stable_sort(by_size.begin(), by_size.end(), [&](size_t a, size_t b) { return elems_of(chunks[a]) > elems_of(chunks[b]); });
+  std::vector<std::vector<size_t>> bins;
+  std::vector<int64_t> fill;
+  for (size_t ci : by_size) {
+    const int64_t e = elems_of(chunks[ci]);
+    size_t k = 0;
+    while (k < bins.size() && (fill[k] + e > cap || bins[k].size() >= size_t(kMaxElemChunks))) ++k;
+    if (k == bins.size()) {
+      bins.emplace_back();
+      fill.push_back(0);
+    }
+    bins[k].push_back(ci);
+    fill[k] += e;
+  }
+  // final order: set by set, descriptors contiguous inside a set
+  int32_t desc_begin = 0;
+  for (size_t k = 0; k < bins.size(); ++k) {
+    LaunchSet set;
+    set.desc_begin = desc_begin;
+    set.elems = fill[k];
+    for (size_t ci : bins[k]) {
+      Chunk ch = std::move(chunks[ci]);
+      ch.set = int32_t(k);
       ch.desc_begin = desc_begin;
       desc_begin += ch.count;
-      plan->ws_bytes = std::max(plan->ws_bytes, carve_chunk(opt, ch).total);
+      set.chunks.push_back(int32_t(plan->chunks.size()));
       plan->chunks.push_back(std::move(ch));
     }
+    set.count = desc_begin - set.desc_begin;
+    layout_set(opt, &plan->chunks, &set);
+    plan->ws_bytes = std::max(plan->ws_bytes, set.bytes);
+    plan->sets.push_back(std::move(set));
   }
   return MUON_OK;
 }
 
-WsCarve carve_chunk(const muon_options_t& opt, const Chunk& c) {
+// Workspace of a launch set: per chunk X0, X1 [K, s, ldx] and A, B [K, s, lda] in the NS element type
+// (every piece 256-byte aligned), then the set's tile partial sums and one reciprocal norm per matrix.
+void layout_set(const muon_options_t& opt, std::vector<Chunk>* chunks, LaunchSet* set) {
   const size_t eb = elem_bytes_of_ns(opt.ns_precision);
-  const size_t xb = up(size_t(c.count) * c.s * c.ldx * eb, 256);
-  const size_t ab = up(size_t(c.count) * c.s * c.lda * eb, 256);
-  WsCarve w;
-  w.x0 = 0;
-  w.x1 = w.x0 + xb;
-  w.a = w.x1 + xb;
-  w.b = w.a + ab;
-  w.partials = w.b + ab;
-  w.rnorm = w.partials + up(size_t(c.count) * c.tiles_per_mat * sizeof(float), 256);
-  w.total = w.rnorm + up(size_t(c.count) * sizeof(float), 256);
-  return w;
+  size_t off = 0;
+  int64_t parts = 0;
+  for (int32_t ci : set->chunks) {
+    Chunk& c = (*chunks)[size_t(ci)];
+    const size_t xb = up(size_t(c.count) * c.s * c.ldx * eb, 256);
+    const size_t ab = up(size_t(c.count) * c.s * c.lda * eb, 256);
+    c.off_x[0] = off;
+    c.off_x[1] = off + xb;
+    c.off_a = off + 2 * xb;
+    c.off_b = c.off_a + ab;
+    off = c.off_b + ab;
+    c.part_off = parts;
+    // the wide elementwise kernels use 64 x 128 tiles (never more per matrix than the 64 x 64 count), so
+    // tiles_per_mat partial sums per matrix cover both tilings
+    parts += int64_t(c.count) * c.tiles_per_mat;
+  }
+  set->off_partials = off;
+  off += up(size_t(parts) * sizeof(float), 256);
+  set->off_rnorm = off;
+  off += up(size_t(set->count) * sizeof(float), 256);
+  set->bytes = off;
+}
+
+// Symmetric product over nb x nb blocks of 128 rows/columns.  Needed: every unordered pair {x, y}, x <= y,
+// once (the epilogue mirrors off-diagonal blocks).  A tile is {ra, rb} x {cc, cd} (256 wide, four blocks) or
+// {ra, rb} x {cc} (128 wide, two blocks).  256-wide tiles feed the tensor cores best (a 128-wide tile moves
+// three quarters of the operand bytes for half the flops), so the list uses them wherever four useful blocks
+// can be had, accepts one redundant block per diagonal 2 x 2 tile (1/(nb+1) of the work), and spends 128-wide
+// tiles only on a last odd column, which a 256-wide tile would compute half empty:
+//   column pairs (2j, 2j+1):  row pairs (2i, 2i+1), i < j: four needed blocks each;
+//                             the diagonal tile {2j, 2j+1} x {2j, 2j+1}: three needed blocks, one computed twice;
+//   last column L when nb is odd: {2i, 2i+1} x {L}, and {L, -} x {L} with an idle second CTA.
+std::vector<TilePatHost> symmetric_tile_pattern(int nb) {
+  std::vector<TilePatHost> tiles;
+  const uint16_t none = 0xFFFFu;
+  const int pairs = nb / 2;
+  for (int j = 0; j < pairs; ++j)
+    for (int i = 0; i <= j; ++i)
+      tiles.push_back(TilePatHost{uint16_t(2 * i), uint16_t(2 * i + 1), uint16_t(2 * j), uint16_t(2 * j + 1)});
+  if (nb % 2) {
+    const int L = nb - 1;
+    for (int i = 0; i < pairs; ++i) tiles.push_back(TilePatHost{uint16_t(2 * i), uint16_t(2 * i + 1), uint16_t(L), none});
+    tiles.push_back(TilePatHost{uint16_t(L), none, uint16_t(L), none});
+  }
+  return tiles;
 }
 
 int validate_layout_host(const muon_layout_desc_t* d) {

@@ -2,9 +2,7 @@
 // mbarrier / TMA / tcgen05, shared-memory and instruction descriptors.  Internal to the library.
 #pragma once
 
-#include <cuda.h>
-
-#include "internal.h"
+#include "tc_tables.h"
 
 namespace muon {
 namespace tc {
@@ -127,23 +125,36 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint
   return d;
 }
 
-// Instruction descriptor for kind::f16: fp32 accumulator, bf16 A and B, A K-major, B K- or MN-major.
-__host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major, int umma_m, int umma_n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(b_mn_major ? 1 : 0) << 16) | (uint32_t(umma_n >> 3) << 17) |
-         (uint32_t(umma_m >> 4) << 24);
+// Instruction descriptor for kind::f16: fp32 accumulator, bf16 A and B, each K- or MN-major.
+__host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major, int umma_m, int umma_n, bool a_mn_major = false) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(a_mn_major ? 1 : 0) << 15) | (uint32_t(b_mn_major ? 1 : 0) << 16) |
+         (uint32_t(umma_n >> 3) << 17) | (uint32_t(umma_m >> 4) << 24);
 }
 
 
-// ------------------------------------------------------------------ epilogue of one 128 x 256 accumulator tile
-constexpr int EPI_TILE_N = 256;
+// ------------------------------------------------------------------ epilogue of one 128-row accumulator tile
 constexpr int EPI_ROWS = 128;
 constexpr int EPI_COLS = 64;                         // columns per chunk (one 128-byte swizzle row of bf16)
 constexpr int EPI_BYTES = EPI_ROWS * EPI_COLS * 2;   // 16 KiB staging buffer
-constexpr int EPI_BUFS = 3;                          // ring of staging buffers: chunk g uses buffer g % 3
+#ifndef MUON_EPI_BUFS
+#define MUON_EPI_BUFS 3
+#endif
+constexpr int EPI_BUFS = MUON_EPI_BUFS;              // ring of staging buffers: chunk g uses buffer g % EPI_BUFS
 
-// Where a tile of C lives: matrix, first row of this CTA's 128 rows, first column.
+// What the four epilogue warps of a CTA need to know about one accumulator tile: 128 rows (row block
+// `rblk`) times one or two 128-column blocks (`cblk0` in TMEM columns [0,128), `cblk1` in [128,256);
+// cblk1 < 0 = the tile is 128 columns wide).  valid = this CTA has rows to write for the tile.
 struct EpiTile {
-  int mat, m0, n0;
+  const CUtensorMap* map_d;
+  const CUtensorMap* map_c;
+  const __nv_bfloat16* d;    // aux matrix D (may be null)
+  __nv_bfloat16* c;
+  int64_t stride_c;
+  int32_t ldc, m, n;
+  int32_t mat, rblk;
+  int32_t cblk0, cblk1;
+  bool mirror0, mirror1;     // also write the 128 x 128 block transposed (symmetric products, off-diagonal blocks)
+  float alpha, beta, gamma;
   bool valid;
 };
 
@@ -151,19 +162,26 @@ struct EpiTile {
 struct EpilogueState {
   uint32_t g = 0;            // chunks processed so far
   uint32_t eph = 0;          // phase of the group rendezvous
+  uint32_t dph = 0;          // bit b: phase of the D-chunk barrier of staging buffer b
   bool d_in_flight = false;  // the D load of chunk g has already been issued (prefetched during chunk g-1)
 };
 
-// Thread = one accumulator row (TMEM lane).  The tile leaves in four 64-column chunks through a ring of three
+__device__ __forceinline__ int epi_chunk_col(const EpiTile& t, int cb) {          // first column of chunk cb, or -1
+  const int blk = cb < 2 ? t.cblk0 : t.cblk1;
+  if (blk < 0) return -1;
+  const int c0 = blk * 128 + (cb & 1) * EPI_COLS;
+  return c0 < t.n ? c0 : -1;
+}
+
+// Thread = one accumulator row (TMEM lane).  The tile leaves in 64-column chunks through a ring of three
 // 128B-swizzled staging buffers: TMA brings the D chunk in (requested one chunk ahead, across tile boundaries,
 // so its latency hides behind the previous chunk), every thread turns its own row of D into its row of C in
-// place (one bf16 rounding of gamma*(beta*D + alpha*acc)), TMA stores the chunk; a strictly upper tile of a
+// place (one bf16 rounding of gamma*(beta*D + alpha*acc)), TMA stores the chunk; an off-diagonal block of a
 // symmetric product is also written transposed with plain stores (64 contiguous bytes per warp instruction).
 // `next` is the tile this CTA processes afterwards (for the prefetch).  Returns false when a bounded wait expired.
-__device__ __forceinline__ bool epilogue_tile(const TcArgs& a, const CUtensorMap* map_d, const CUtensorMap* map_c,
-                                              const EpiTile& cur, const EpiTile& next, bool mirror, uint32_t taddr,
-                                              uint32_t epi_base, uint32_t dfull_bar0, uint32_t egroup_bar, uint32_t tfull_bar,
-                                              uint32_t aph, volatile int* abort_flag, EpilogueState& st, int quad, int lane) {
+__device__ __forceinline__ bool epilogue_tile(const EpiTile& cur, const EpiTile& next, uint32_t taddr, uint32_t epi_base,
+                                              uint32_t dfull_bar0, uint32_t egroup_bar, uint32_t tfull_bar, uint32_t aph,
+                                              volatile int* abort_flag, EpilogueState& st, int quad, int lane) {
   const bool leader = quad == 2 && lane == 0;        // warp 2 is the first epilogue warp
   const int lrow = quad * 32 + lane;
   auto group_sync = [&]() -> bool {                  // rendezvous of the four warps on an mbarrier: bounded like every wait
@@ -173,42 +191,42 @@ __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, const CUtensorMap
     st.eph ^= 1u;
     return done;
   };
-  const int mat = cur.mat, m0 = cur.m0, n0 = cur.n0;
-  float gamma = 1.f;
-  if (a.gamma_mode) {
-    const float r = a.rnorm[mat];
-    gamma = a.gamma_mode == 1 ? r : r * r;
-  }
+  const int mat = cur.mat, m0 = cur.rblk * EPI_ROWS;
+  const float alpha = cur.alpha, beta = cur.beta, gamma = cur.gamma;
   const int row = m0 + lrow;
-  const bool row_ok = row < a.m;
-  __nv_bfloat16* cmat = a.c + size_t(mat) * a.stride_c;
+  const bool row_ok = row < cur.m;
+  __nv_bfloat16* cmat = cur.c + size_t(mat) * cur.stride_c;
+  const bool next_d = next.valid && next.d != nullptr;
   bool acc_ready = false;
 #pragma unroll 1
-  for (int cb = 0; cb < EPI_TILE_N / EPI_COLS; ++cb, ++st.g) {
-    const int c0 = n0 + cb * EPI_COLS;
-    if (c0 >= a.n) break;                             // uniform over the group
+  for (int cb = 0; cb < 4; ++cb) {
+    const int c0 = epi_chunk_col(cur, cb);
+    if (c0 < 0) continue;                             // uniform over the group
     const uint32_t b = st.g % EPI_BUFS;
     const uint32_t ebuf = epi_base + b * EPI_BYTES;
     const uint32_t dbar = dfull_bar0 + b * 8u;
-    // the chunk after this one: the next chunk of this tile, or the first chunk of the next tile
-    const bool more_here = cb + 1 < EPI_TILE_N / EPI_COLS && c0 + EPI_COLS < a.n;
-    const bool have_next = more_here || next.valid;
+    // the chunk after this one: the next valid chunk of this tile, or the first chunk of the next tile
+    int nc0 = -1;
+    for (int k = cb + 1; k < 4 && nc0 < 0; ++k) nc0 = epi_chunk_col(cur, k);
+    const bool more_here = nc0 >= 0;
+    const bool prefetch = cur.d ? (more_here || next_d) : false;
     if (leader) {
-      if (a.d) {
-        if (!st.d_in_flight) {                        // only the very first chunk of a CTA is not prefetched
-          tma_wait_read<2>();                         // buffer b was last read by the store of chunk g-3
+      if (cur.d) {
+        if (!st.d_in_flight) {                        // a chunk that nobody prefetched (the first of a CTA, or after a tile without D)
+          tma_wait_read<EPI_BUFS - 1>();              // buffer b was last read by the store of chunk g - EPI_BUFS
           mbar_expect_tx(dbar, EPI_BYTES);
-          tma_load_3d(ebuf, map_d, dbar, c0, m0, mat);
+          tma_load_3d(ebuf, cur.map_d, dbar, c0, m0, mat);
         }
-        if (have_next) {
+        if (prefetch) {
           const uint32_t nb = (st.g + 1) % EPI_BUFS;
-          tma_wait_read<1>();                         // buffer nb was last read by the store of chunk g-2
+          tma_wait_read<EPI_BUFS - 2>();              // buffer nb was last read by the store of chunk g + 1 - EPI_BUFS
           mbar_expect_tx(dfull_bar0 + nb * 8u, EPI_BYTES);
-          if (more_here) tma_load_3d(epi_base + nb * EPI_BYTES, map_d, dfull_bar0 + nb * 8u, c0 + EPI_COLS, m0, mat);
-          else tma_load_3d(epi_base + nb * EPI_BYTES, map_d, dfull_bar0 + nb * 8u, next.n0, next.m0, next.mat);
+          if (more_here) tma_load_3d(epi_base + nb * EPI_BYTES, cur.map_d, dfull_bar0 + nb * 8u, nc0, m0, mat);
+          else tma_load_3d(epi_base + nb * EPI_BYTES, next.map_d, dfull_bar0 + nb * 8u, epi_chunk_col(next, 0),
+                           next.rblk * EPI_ROWS, next.mat);
         }
       } else {
-        tma_wait_read<2>();                           // buffer b was last read by the store of chunk g-3
+        tma_wait_read<EPI_BUFS - 1>();                // buffer b was last read by the store of chunk g - EPI_BUFS
       }
     }
     if (!acc_ready) {
@@ -216,31 +234,33 @@ __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, const CUtensorMap
       tc_fence_after();
       acc_ready = true;
     }
-    if (a.d) {
-      if (!mbar_wait(dbar, (st.g / EPI_BUFS) & 1u, abort_flag)) return false;
+    if (cur.d) {
+      if (!mbar_wait(dbar, (st.dph >> b) & 1u, abort_flag)) return false;
+      st.dph ^= 1u << b;
     } else {
       if (!group_sync()) return false;                // the leader's wait_group above frees the buffer for everyone
     }
-    st.d_in_flight = a.d && have_next;
+    st.d_in_flight = prefetch;
     uint32_t v[64];
     tc_ld32(taddr + uint32_t(cb * EPI_COLS), *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
     tc_ld32(taddr + uint32_t(cb * EPI_COLS + 32), *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
     tc_wait_ld();
+    const bool mirror = cb < 2 ? cur.mirror0 : cur.mirror1;
     const uint32_t srow = ebuf + uint32_t(lrow) * 128u;
 #pragma unroll
     for (int q = 0; q < 8; ++q) {                     // 16-byte piece q of the row sits at piece q ^ (row & 7)
       const uint32_t addr = srow + (uint32_t(q ^ (lrow & 7)) << 4);
       uint32_t d0 = 0, d1 = 0, d2 = 0, d3 = 0;
-      if (a.d) asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3) : "r"(addr));
+      if (cur.d) asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3) : "r"(addr));
       const uint32_t dd[4] = {d0, d1, d2, d3};
       uint32_t oo[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        float x0 = a.alpha * __uint_as_float(v[q * 8 + 2 * e]), x1 = a.alpha * __uint_as_float(v[q * 8 + 2 * e + 1]);
-        if (a.d) {
+        float x0 = alpha * __uint_as_float(v[q * 8 + 2 * e]), x1 = alpha * __uint_as_float(v[q * 8 + 2 * e + 1]);
+        if (cur.d) {
           const __nv_bfloat162 dp = *reinterpret_cast<const __nv_bfloat162*>(&dd[e]);
-          x0 += a.beta * __low2float(dp);
-          x1 += a.beta * __high2float(dp);
+          x0 += beta * __low2float(dp);
+          x1 += beta * __high2float(dp);
         }
         const __nv_bfloat162 o = __floats2bfloat162_rn(gamma * x0, gamma * x1);
         oo[e] = *reinterpret_cast<const uint32_t*>(&o);
@@ -251,38 +271,20 @@ __device__ __forceinline__ bool epilogue_tile(const TcArgs& a, const CUtensorMap
         for (int e = 0; e < 4; ++e) {
           const int c = c0 + q * 8 + 2 * e;
           const __nv_bfloat162 o = *reinterpret_cast<const __nv_bfloat162*>(&oo[e]);
-          if (c < a.n) cmat[size_t(c) * a.ldc + row] = __low2bfloat16(o);
-          if (c + 1 < a.n) cmat[size_t(c + 1) * a.ldc + row] = __high2bfloat16(o);
+          if (c < cur.n) cmat[size_t(c) * cur.ldc + row] = __low2bfloat16(o);
+          if (c + 1 < cur.n) cmat[size_t(c + 1) * cur.ldc + row] = __high2bfloat16(o);
         }
       }
     }
     fence_async_smem();                               // generic-proxy writes -> visible to the TMA store
     if (!group_sync()) return false;                  // everyone is done with the buffer (reads of D, writes of C)
     if (leader) {
-      tma_store_3d(map_c, ebuf, c0, m0, mat);         // rows/columns beyond the matrix are clipped
+      tma_store_3d(cur.map_c, ebuf, c0, m0, mat);     // rows/columns beyond the matrix are clipped
       tma_commit();
     }
+    ++st.g;
   }
   return true;
-}
-
-// ------------------------------------------------------------------ host: tensor maps
-typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// 3-D map over a batch of row-major matrices: dims (cols, rows, batch), box (64, box_rows, 1), 128B swizzle.
-inline bool encode_map(void* fn, CUtensorMap* map, const void* ptr, int cols, int rows, int batch, int ld, int64_t stride,
-                int box_rows) {
-  const cuuint64_t dims[3] = {cuuint64_t(cols), cuuint64_t(rows), cuuint64_t(batch)};
-  const cuuint64_t strides[2] = {cuuint64_t(ld) * 2u, cuuint64_t(stride) * 2u};
-  const cuuint32_t box[3] = {64u, cuuint32_t(box_rows), 1u};
-  const cuuint32_t estr[3] = {1u, 1u, 1u};
-  const CUresult r = reinterpret_cast<EncodeFn>(fn)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims,
-                                                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
 }
 
 }  // namespace tc

@@ -1,0 +1,122 @@
+// Problem tables of the grouped tensor-core engine and the host helpers that fill them.  Internal to the library.
+#pragma once
+
+#include <cuda.h>
+
+#include "internal.h"
+
+namespace muon {
+namespace tc {
+
+// One tile of the paired engine, in units of 128-row / 128-column blocks: CTA 0 of the pair computes row
+// block ra, CTA 1 row block rb, both against column blocks cc (accumulator columns 0..127) and cd (128..255).
+// kNoBlock in rb: CTA 1 has nothing to do; in cd: the tile is 128 columns wide (UMMA N = 128).
+struct TilePat {
+  uint16_t ra, rb, cc, cd;
+};
+constexpr uint16_t kNoBlock = 0xFFFFu;
+
+// Tensor maps of one batched product of a grouped launch.  They are encoded once, when the plan is bound to a
+// workspace, and stay in device memory (the TMA unit reads them from there).
+struct alignas(128) TcMaps {
+  CUtensorMap p;     // P: 128-row boxes
+  CUtensorMap ph;    // P: 64 x 64 boxes (transposed reads of a half-stored symmetric P)
+  CUtensorMap q;     // Q: 128-row boxes (nn = 0) or 64 k-rows x 64 columns (nn = 1)
+  CUtensorMap qh;    // Q: 64 x 64 boxes (128-wide tiles; transposed reads of a half-stored symmetric Q)
+  CUtensorMap d, c;  // aux matrix and result: 128 rows x 64 columns
+};
+
+// Everything else about the product travels by value with the launch (constant bank: decoding a tile costs no
+// global-memory round trip on the MMA issuer's critical path).
+struct TcProbInfo {
+  const __nv_bfloat16* d;    // aux matrix (may be null)
+  __nv_bfloat16* c;
+  const float* rnorm;        // per matrix (gamma modes 1, 2)
+  const float* coef;         // per matrix coefficient rows [batch][coef_stride] or null
+  const TilePat* pattern;    // explicit tile list per matrix (symmetric products); null: dense 2 x 2 block grid
+  int64_t stride_c;
+  int32_t m, n, kdim, ldc;
+  int32_t batch, tiles_per_mat, tile_begin, row_pairs;
+  int32_t symmetric, nn, rblocks, cblocks;
+  // Half-stored symmetric matrices.  The Newton-Schulz products never need the whole of A or B in memory: a
+  // symmetric result is written only where tiles compute it -- block (r, c) with (r >> 1) <= (c >> 1) in
+  // 128-blocks -- and a consumer that needs block (r, k) below that line reads block (k, r) instead and feeds
+  // it to the tensor core as an MN-major operand (the transpose costs nothing).
+  int32_t mirror_out;        // 1: also write the transposed blocks (stand-alone symmetric product: full C)
+  int32_t p_half, q_half;    // operand P / Q is such a half-stored symmetric matrix
+  int32_t pad;
+};
+constexpr int kMaxProblems = kMaxElemChunks;
+
+// By-value arguments of one grouped launch.
+struct TcLaunch {
+  const TcMaps* maps;        // device, one per problem
+  TcProbInfo info[kMaxProblems];
+  int32_t nprob, total_tiles;
+  float alpha, beta;
+  int32_t gamma_mode;        // 0: 1, 1: r, 2: r*r
+  int32_t coef_a, coef_b;    // index into a matrix's coefficient row that replaces alpha / beta (-1: keep the scalar)
+  int32_t coef_stride;
+  int32_t* status;
+};
+
+// Host view of one product launch of a launch set: the device maps plus the by-value problem records.
+struct TcTable {
+  const TcMaps* maps = nullptr;
+  TcProbInfo info[kMaxProblems];
+  int32_t nprob = 0, total_tiles = 0;
+};
+
+// ------------------------------------------------------------------ host: tensor maps
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 3-D map over a batch of row-major matrices: dims (cols, rows, batch), box (64, box_rows, 1), 128B swizzle.
+inline bool encode_map(void* fn, CUtensorMap* map, const void* ptr, int cols, int rows, int batch, int ld, int64_t stride,
+                int box_rows) {
+  const cuuint64_t dims[3] = {cuuint64_t(cols), cuuint64_t(rows), cuuint64_t(batch)};
+  const cuuint64_t strides[2] = {cuuint64_t(ld) * 2u, cuuint64_t(stride) * 2u};
+  const cuuint32_t box[3] = {64u, cuuint32_t(box_rows), 1u};
+  const cuuint32_t estr[3] = {1u, 1u, 1u};
+  const CUresult r = reinterpret_cast<EncodeFn>(fn)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims,
+                                                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+}  // namespace tc
+
+// Tables of one launch set (tensor-core engine): for each product the problem list, longest k first.
+struct SetTables {
+  tc::TcTable g1[2];   // A = X X^T, reading X iterate 0 / 1
+  tc::TcTable g2;      // B = bA + c A A^T
+  tc::TcTable g3[2];   // X' = aX + B X, reading iterate 0 / 1 and writing the other
+};
+
+// Launches the paired engine: tensor maps in device memory, everything else by value.
+int launch_tc_grouped(int device, const tc::TcLaunch& L, cudaStream_t st);
+// Number of SMs of the device (> 0), after making the paired kernel launchable there; < 0 on error.
+int tc_pair_grid_setup(int device);
+
+// Builds (or rebuilds, when the workspace moved) the tables of every launch set of `plan`:
+// tensor maps over the workspace buffers (device memory), tile lists, per-product problem lists.
+int bind_plan_tables(muon_ctx* ctx, Plan* plan);
+void release_plan_tables(Plan* plan);
+
+// Host image of the device part of the tables of ONE launch set (tile lists and tensor maps) laid out for device
+// address `dev_base`; used by bind_plan_tables and by the allocation-free entry point, which places the image in
+// its built-in scratch.
+struct SetImage {
+  std::vector<char> bytes;
+  SetTables tables;       // device addresses inside refer to dev_base + offset
+};
+int build_set_image(void* encode_fn, const void* ws, const std::vector<Chunk>& chunks, const LaunchSet& set,
+                    const void* dev_base, SetImage* out, int64_t* encodes);
+
+// Single stand-alone product (muon_ns_product): device image (maps and tile list) plus the by-value table.
+int build_product_image(void* encode_fn, const GemmArgs& g, const void* dev_base, std::vector<char>* bytes, tc::TcTable* table,
+                        int64_t* encodes);
+
+}  // namespace muon

@@ -23,8 +23,10 @@ def test_expired_wait_is_reported_and_the_context_survives():
     ctx.muon_self_test_bounded_wait()
     assert ctx.muon_last_device_status() == 100           # the wait gave up and said so
     assert time.perf_counter() - t0 < 5.0                  # ... within its limit, not after a hang
+    assert ctx.muon_synchronize_and_check() == mb.ERR_DEVICE_TIMEOUT   # the opt-in synchronous check turns it into a status
     ctx.muon_clear_device_status()
     assert ctx.muon_last_device_status() == 0
+    assert ctx.muon_synchronize_and_check() == mb.OK
     # the device and the context are fine: a normal orthogonalisation still matches the oracle
     shape = (256, 384)
     x, v = bf16_input(wl.grad_np("after_timeout", 0, 0, shape))

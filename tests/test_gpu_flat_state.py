@@ -76,6 +76,28 @@ def test_flat_state_one_llama_layer():
     _case(mb, shapes, wl.layout_per_param(shapes, 8), "flatllama", two_steps=False)
 
 
+@pytest.mark.parametrize("align", [1, 2, 4])
+def test_flat_state_with_segment_offsets_that_are_not_vector_aligned(align):
+    """A row-aligned layout may start a segment on any multiple of align_elems.  With align 1, 2 or 4 a small odd
+    matrix ahead of a 64 x 64 one leaves the latter's rows at offsets that are no multiple of 8 (or 4) elements:
+    the step kernels must then give up their 16-byte accesses on the flat buffers, not fault or mis-read."""
+    from paper_2609_21594_b200 import binding as mb
+
+    shapes = [(3, 5), (64, 64), (7, 9), (128, 256), (256, 128)]
+    lay = wl.layout_per_param(shapes, 2, align=align)
+    offs = {s.flat_offset % 8 for s in lay.segments if shapes[s.matrix][1] % 8 == 0}
+    assert any(o != 0 for o in offs)                     # the interesting case really occurs
+    W, Wn = _case(mb, shapes, lay, f"flatalign{align}")
+    # ... and the shared result is right: two oracle steps on the 64 x 64 matrix
+    Wo, Mo = Wn[1].astype(np.float64), wl.grad_np(f"flatalign{align}", 9, 1, shapes[1]).astype(np.float64)
+    for step in range(2):
+        g = wl.bf16_bits_to_f32(wl.to_bf16_bits(wl.grad_np(f"flatalign{align}", step, 1, shapes[1]))).astype(np.float64)
+        Wprev = Wo
+        Wo, Mo, _ = orc.muon_step(Wo, g, Mo, LR, MU, WD, 5, QUINTIC, 1e-7, True, "bf16")
+    # teacher forcing is not needed at this size: two steps stay well inside the tolerance on dW of the last step
+    assert rel(host_f64(W[1]) - Wprev, Wo - Wprev) <= 3e-2
+
+
 def test_flat_state_needs_whole_row_segments():
     from paper_2609_21594_b200 import binding as mb
 

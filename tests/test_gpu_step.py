@@ -458,6 +458,41 @@ def test_ns_ragged_multi_tile_shapes(engine):
     ctx.close()
 
 
+def test_one_launch_per_product_for_all_shape_groups_and_no_encoding_in_steady_state():
+    """The tensor engine runs each Newton-Schulz product as one kernel over every shape group that is resident
+    together: the d=256 layer (two core shapes) takes 3 * 5 product launches, not 30, and after the first step on
+    a workspace no tensor map is encoded again."""
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, "bf16", "tensor")
+    shapes = wl.shapes_tiny()
+    ctx.ensure_workspace(shapes)
+    ins = [bf16_input(wl.grad_np("grouped", 0, i, s))[0] for i, s in enumerate(shapes)]
+    outs = [torch.empty_like(t) for t in ins]
+    ctx.muon_orthogonalize_batched(ins, outs, shapes, 5, QUINTIC)          # binds the plan: encodes once
+    torch.cuda.synchronize()
+    enc0 = ctx.muon_tensor_map_encodes()
+    assert enc0 > 0
+    ctx.muon_profile_enable(True)
+    ctx.muon_profile_reset()
+    n0 = ctx.muon_launch_count()
+    for _ in range(3):
+        ctx.muon_orthogonalize_batched(ins, outs, shapes, 5, QUINTIC)
+    torch.cuda.synchronize()
+    ph = ctx.muon_profile_read()
+    ctx.muon_profile_enable(False)
+    assert ph["ns"][1] == 3 * 15                                           # product launches: 15 per call
+    assert ctx.muon_launch_count() - n0 == 3 * (15 + 2 + 1)                # + stage, norm, apply (one wide launch each)
+    assert ctx.muon_tensor_map_encodes() == enc0                           # steady state: nothing encoded
+    # a new workspace address re-binds once
+    ctx.muon_set_workspace(torch.empty(mb.muon_workspace_bytes(ctx.opt, shapes) + 4096, dtype=torch.uint8, device="cuda"))
+    ctx.muon_orthogonalize_batched(ins, outs, shapes, 5, QUINTIC)
+    torch.cuda.synchronize()
+    assert ctx.muon_tensor_map_encodes() == 2 * enc0
+    assert ctx.muon_last_device_status() == 0
+    ctx.close()
+
+
 def test_many_small_heterogeneous_matrices():
     """1500 small matrices of a dozen interleaved shapes (several shape groups, tall and wide mixed in one group,
     batches far larger than the SM count): every 50th one is checked against the oracle, all must be finite and

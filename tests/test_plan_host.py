@@ -1,0 +1,104 @@
+"""Host-side planning logic of the library, checked on a CPU: the tile lists of the symmetric products and
+the packing of shape groups into launch sets.  Both are pure host arithmetic behind the C ABI."""
+import itertools
+
+import numpy as np
+import pytest
+
+from paper_2609_21594_b200 import binding as mb
+from paper_2609_21594_b200 import workloads as wl
+
+NONE = 0xFFFF
+
+
+def _blocks_of(tiles):
+    """Every (row block, column block) a tile list computes, in order."""
+    out = []
+    for ra, rb, cc, cd in tiles:
+        for r in (ra, rb):
+            for c in (cc, cd):
+                if r != NONE and c != NONE:
+                    out.append((r, c))
+    return out
+
+
+@pytest.mark.parametrize("nb", list(range(0, 41)) + [56, 112])
+def test_symmetric_tiles_cover_every_unordered_block_pair(nb):
+    tiles = mb.muon_symmetric_tiles(nb)
+    blocks = _blocks_of(tiles)
+    for ra, rb, cc, cd in tiles:
+        assert ra != NONE and cc != NONE and ra < nb and cc < nb
+        assert rb == NONE or (rb < nb and rb != ra)
+        assert cd == NONE or (cd < nb and cd != cc)
+    # brute force over every block the list computes
+    seen = {}
+    for r, c in blocks:
+        seen[(min(r, c), max(r, c))] = seen.get((min(r, c), max(r, c)), 0) + 1
+    want = {(x, y) for x in range(nb) for y in range(x, nb)}
+    assert set(seen) == want                                     # nothing missing, nothing outside the matrix
+    # the only pairs computed twice are (2j, 2j+1): the lower-left block of a diagonal 2 x 2 tile
+    twice = sorted(k for k, v in seen.items() if v > 1)
+    assert all(v <= 2 for v in seen.values())
+    assert twice == [(2 * j, 2 * j + 1) for j in range(nb // 2)]
+    # each ordered block position is written by at most one tile (a mirrored block is written by its source tile)
+    assert len(set(blocks)) == len(blocks)
+    # a last odd column is covered by 128-wide tiles, everything else by 256-wide ones
+    narrow = [t for t in tiles if t[3] == NONE]
+    assert len(narrow) == (nb // 2 + 1 if nb % 2 else 0)
+    assert all(t[2] == nb - 1 for t in narrow)
+    half_empty = [t for t in tiles if t[1] == NONE]
+    assert len(half_empty) == nb % 2
+    # cost in 128 x 128 block products: the triangle, one redundant block per diagonal tile, one idle half at most
+    paid = sum(2 * (1 if t[3] == NONE else 2) for t in tiles)
+    assert paid == nb * (nb + 1) // 2 + nb // 2 + nb % 2
+
+
+def test_symmetric_tiles_cost_at_the_benchmark_sizes():
+    def cost(nb):                                  # in 256 x 256 tile equivalents
+        return sum(0.5 if t[3] == NONE else 1.0 for t in mb.muon_symmetric_tiles(nb))
+    assert cost(32) == 136                         # 4096 rows: the plain upper triangle of 2 x 2 tiles
+    assert cost(11) == 18                          # 1408 rows: 15 full tiles + 6 half-width ones (21 before)
+    assert cost(16) == 36 and cost(8) == 10 and cost(2) == 1
+
+
+def test_launch_sets_pack_shape_groups_under_the_cap():
+    opt = mb.muon_default_options()
+    cap = 1 << 29
+
+    def sets_of(shapes):
+        n, set_of = mb.muon_plan_launch_sets(opt, shapes)
+        nch, chunk_of = mb.muon_plan_describe(opt, shapes)
+        elems = np.zeros(n, dtype=np.int64)
+        chunks_in = [set() for _ in range(n)]
+        for (m, k), s, c in zip(shapes, set_of, chunk_of):
+            if s >= 0:
+                elems[s] += m * k
+                chunks_in[s].add(c)
+        return n, nch, elems, chunks_in
+
+    n, nch, elems, chunks_in = sets_of(wl.shapes_tiny())
+    assert n == 1 and nch == 2                    # both core shapes of the d=256 layer share every launch
+    n, nch, elems, chunks_in = sets_of(wl.shapes_1b())
+    assert nch == 4 and n == 2 and (elems <= cap).all()
+    n, nch, elems, chunks_in = sets_of(wl.shapes_moe())
+    assert nch == 6 and n == 5 and (elems <= cap).all()      # the attention group rides with one expert chunk
+    n, nch, elems, chunks_in = sets_of(wl.shapes_llama8b())
+    assert nch == 14 and n == 14                  # every Llama-3-8B chunk already fills the cap on its own
+    # a chunk belongs to exactly one set
+    all_chunks = list(itertools.chain.from_iterable(chunks_in))
+    assert len(all_chunks) == len(set(all_chunks)) == nch
+    # one matrix larger than the cap still gets a set of its own
+    big = mb.muon_default_options(chunk_elems=1000)
+    n, set_of = mb.muon_plan_launch_sets(big, [(64, 64), (8, 8), (8, 8), (100, 100)])
+    assert n == 3 and set_of[1] == set_of[2] and len({set_of[0], set_of[1], set_of[3]}) == 3
+    n, set_of = mb.muon_plan_launch_sets(opt, [(0, 5), (3, 4)])
+    assert n == 1 and set_of == [-1, 0]
+
+
+def test_workspace_is_the_largest_launch_set():
+    opt = mb.muon_default_options()
+    # tiny: both groups resident together: 2 X + 2 A for each, bf16
+    need = mb.muon_workspace_bytes(opt, wl.shapes_tiny())
+    x = (4 * 256 * 256 + 2 * 256 * 1024) * 2
+    a = (4 * 256 * 256 + 2 * 256 * 256) * 2
+    assert 2 * x + 2 * a <= need <= 2 * x + 2 * a + 16384
