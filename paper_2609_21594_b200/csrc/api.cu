@@ -178,8 +178,10 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
   if (sr.tables) {
     auto launch = [&](const tc::TcTable& tab, float alpha, float beta, int gamma_mode) {
       tc::TcLaunch L;
-      L.maps = tab.maps;
-      for (int i = 0; i < tab.nprob; ++i) L.info[i] = tab.info[i];
+      for (int i = 0; i < tab.nprob; ++i) {
+        L.maps[i] = tab.maps[i];
+        L.info[i] = tab.info[i];
+      }
       L.nprob = tab.nprob;
       L.total_tiles = tab.total_tiles;
       L.alpha = alpha; L.beta = beta; L.gamma_mode = gamma_mode;
@@ -833,7 +835,7 @@ int muon_ns_product(muon_ctx_t* ctx, const void* p, const void* q, const void* d
     rc = commit_slot(slot, img.data(), img.size(), st);
     if (rc != MUON_OK) return rc;
     tc::TcLaunch L;
-    L.maps = tab.maps;
+    L.maps[0] = tab.maps[0];
     L.info[0] = tab.info[0];
     L.nprob = 1;
     L.total_tiles = tab.total_tiles;

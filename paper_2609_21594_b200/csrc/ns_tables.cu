@@ -100,9 +100,7 @@ int build_set_image(void* encode_fn, const void* ws, const std::vector<Chunk>& c
   const float* rnorm_base = reinterpret_cast<const float*>(wsb + set.off_rnorm);
   SetTables T;
   for (int kind = 0; kind < 5; ++kind) {     // 0,1: G1 reading X0/X1; 2: G2; 3,4: G3 reading X0/X1
-    const size_t off = ib.reserve(size_t(n) * sizeof(TcMaps), 128);
     TcTable& tab = kind < 2 ? T.g1[kind] : kind == 2 ? T.g2 : T.g3[kind - 3];
-    tab.maps = static_cast<const TcMaps*>(ib.dev(off));
     tab.nprob = n;
     int32_t tile_begin = 0;
     const std::vector<int>& order = kind < 2 ? by_l : by_s;
@@ -161,7 +159,7 @@ int build_set_image(void* encode_fn, const void* ws, const std::vector<Chunk>& c
       const int64_t tiles = int64_t(p.tiles_per_mat) * p.batch;
       if (tile_begin + tiles > 0x3fffffffLL) return MUON_ERR_UNSUPPORTED;
       tile_begin += int32_t(tiles);
-      std::memcpy(ib.bytes.data() + off + size_t(j) * sizeof(TcMaps), &m, sizeof(m));
+      tab.maps[j] = m;
       tab.info[j] = p;
     }
     tab.total_tiles = tile_begin;
@@ -176,7 +174,6 @@ int build_product_image(void* encode_fn, const GemmArgs& g, const void* dev_base
   if (!encode_fn) return MUON_ERR_CUDA;
   ImageBuilder ib;
   ib.dev_base = static_cast<const char*>(dev_base);
-  const size_t off = ib.reserve(sizeof(TcMaps), 128);
   TcMaps m;
   std::memset(&m, 0, sizeof(m));
   TcProbInfo p;
@@ -216,8 +213,7 @@ int build_product_image(void* encode_fn, const GemmArgs& g, const void* dev_base
   }
   const int64_t tiles = int64_t(p.tiles_per_mat) * p.batch;
   if (tiles > 0x3fffffffLL) return MUON_ERR_UNSUPPORTED;
-  std::memcpy(ib.bytes.data() + off, &m, sizeof(m));
-  table->maps = static_cast<const TcMaps*>(ib.dev(off));
+  table->maps[0] = m;
   table->info[0] = p;
   table->nprob = 1;
   table->total_tiles = int32_t(tiles);

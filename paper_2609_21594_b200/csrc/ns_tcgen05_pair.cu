@@ -44,6 +44,11 @@ constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BUFS * EPI_BYTES + 1024 + 256;
 constexpr int TMEM_COLS = 512;
 constexpr int NUM_THREADS = 192;
+// constant parts of the shared-memory matrix descriptors (see make_desc): K-major (LBO 16, SBO 1024) and
+// MN-major (LBO 8 KiB between 64-element chunks, SBO 1024), 128-byte swizzle
+constexpr uint64_t DESC_HI_K = (uint64_t(16 >> 4) << 16) | (uint64_t(1024 >> 4) << 32) | (uint64_t(1) << 46) | (uint64_t(2) << 61);
+constexpr uint64_t DESC_HI_MN =
+    (uint64_t((64 * BK * 2) >> 4) << 16) | (uint64_t(1024 >> 4) << 32) | (uint64_t(1) << 46) | (uint64_t(2) << 61);
 
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
@@ -159,6 +164,83 @@ __device__ __forceinline__ EpiTile make_epi(const Tile& tl, int rank, const TcLa
   return e;
 }
 
+// ---- main-loop bodies, specialised at compile time on how the two operands are read (K-major as stored, or
+// MN-major = transposed): the producer and the MMA issuer are single threads whose loop must stay short, so
+// a tile's k-range is cut into at most three pieces with fixed operand forms instead of deciding per k-block.
+struct LoopCtx {
+  uint32_t base, bars;          // shared-memory addresses of the stage ring and of the barrier block
+  volatile int* abort_flag;
+  uint32_t it;                  // k-blocks processed so far by this role (ring position and phase)
+};
+__device__ __forceinline__ uint32_t full_bar_of(const LoopCtx& c, int s) { return c.bars + uint32_t(s) * 8u; }
+__device__ __forceinline__ uint32_t empty_bar_of(const LoopCtx& c, int s) { return c.bars + uint32_t(STAGES + s) * 8u; }
+
+struct LoadArgs {
+  const TcMaps* mp;
+  int mat, prow, qcol;
+  uint32_t stage_tx;
+  bool leader_cta, narrow;
+};
+
+template <bool A_MN, bool B_MN>
+__device__ __forceinline__ bool produce_range(LoopCtx& c, const LoadArgs& a, int kb_begin, int kb_end) {
+  for (int kb = kb_begin; kb < kb_end; ++kb, ++c.it) {
+    const int s = int(c.it % STAGES);
+    const uint32_t ph = (c.it / STAGES) & 1u;
+    if (!mbar_wait(empty_bar_of(c, s), ph ^ 1u, c.abort_flag)) return false;
+    const uint32_t sa = c.base + uint32_t(s) * STAGE_BYTES, sb = sa + A_BYTES;
+    if (a.leader_cta) mbar_expect_tx(full_bar_of(c, s), a.stage_tx);
+    const uint32_t fb = map_to_cta(full_bar_of(c, s), 0);
+    const int k0 = kb * BK;
+    if (!A_MN) {                                   // 128 rows of P x 64 k
+      tma_load_3d_pair(sa, &a.mp->p, fb, k0, a.prow, a.mat);
+    } else {                                       // the same block read from its mirror image: 64 k-rows x 64 columns, twice
+      tma_load_3d_pair(sa, &a.mp->ph, fb, a.prow, k0, a.mat);
+      tma_load_3d_pair(sa + 64 * BK * 2, &a.mp->ph, fb, a.prow + 64, k0, a.mat);
+    }
+    if (!B_MN) {                                   // 128 rows of Q, or the 64 a 128-wide tile needs
+      tma_load_3d_pair(sb, a.narrow ? &a.mp->qh : &a.mp->q, fb, k0, a.qcol, a.mat);
+    } else {                                       // 64 k-rows x 64 columns, twice for a 256-wide tile
+      tma_load_3d_pair(sb, &a.mp->qh, fb, a.qcol, k0, a.mat);
+      if (!a.narrow) tma_load_3d_pair(sb + 64 * BK * 2, &a.mp->qh, fb, a.qcol + 64, k0, a.mat);
+    }
+  }
+  return true;
+}
+
+// A shared-memory descriptor is a constant high part (layout, strides) plus the start address in 16-byte units.
+// K-major: 16 k = 32 bytes along a 128-byte row; MN-major: 16 k-rows of 128 bytes each.
+template <bool A_MN, bool B_MN>
+__device__ __forceinline__ bool issue_range(LoopCtx& c, uint32_t d_tmem, uint32_t idesc_base, int kb_begin, int kb_end) {
+  constexpr uint32_t idesc_major = (A_MN ? 1u << 15 : 0u) | (B_MN ? 1u << 16 : 0u);
+  constexpr uint64_t a_hi = A_MN ? DESC_HI_MN : DESC_HI_K, b_hi = B_MN ? DESC_HI_MN : DESC_HI_K;
+  constexpr uint32_t a_step = A_MN ? (UK * 128) >> 4 : (UK * 2) >> 4, b_step = B_MN ? (UK * 128) >> 4 : (UK * 2) >> 4;
+  const uint32_t idesc = idesc_base | idesc_major;
+  for (int kb = kb_begin; kb < kb_end; ++kb, ++c.it) {
+    const int s = int(c.it % STAGES);
+    const uint32_t ph = (c.it / STAGES) & 1u;
+    if (!mbar_wait(full_bar_of(c, s), ph, c.abort_flag)) return false;
+    tc_fence_after();
+    const uint32_t a0 = (c.base + uint32_t(s) * STAGE_BYTES) >> 4, b0 = a0 + (A_BYTES >> 4);
+#pragma unroll
+    for (int k = 0; k < BK / UK; ++k)
+      tc_mma_pair(d_tmem, a_hi | uint64_t(a0 + uint32_t(k) * a_step), b_hi | uint64_t(b0 + uint32_t(k) * b_step), idesc,
+                  (kb > 0 || k > 0) ? 1u : 0u);
+    tc_commit_pair(empty_bar_of(c, s));
+  }
+  return true;
+}
+
+// k-blocks [0, p_flip) read P transposed, [0, q_flip) read Q transposed: three pieces with fixed forms.
+#define MUON_FOR_K_PIECES(CALL)                                                              \
+  {                                                                                          \
+    const int lo_ = p_flip_kb < q_flip_kb ? p_flip_kb : q_flip_kb;                           \
+    const int hi_ = p_flip_kb < q_flip_kb ? q_flip_kb : p_flip_kb;                           \
+    if (ok && lo_ > 0) ok = CALL(true, true, 0, lo_);                                        \
+    if (ok && hi_ > lo_) ok = p_flip_kb > q_flip_kb ? CALL(true, false, lo_, hi_) : CALL(false, true, lo_, hi_); \
+    if (ok && num_kb > hi_) ok = CALL(false, false, hi_, num_kb);                            \
+  }
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
   extern __shared__ uint8_t smem_raw[];
@@ -220,12 +302,12 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (one per CTA)
     if (lane == 0) {
-      uint32_t it = 0;
+      LoopCtx lc{base, bars, abort_flag, 0u};
       bool ok = true;
       for (int t = pair_id; t < total_tiles && ok; t += num_pairs) {
         const Tile tl = decode_tile(t, L);
         const TcProbInfo& p = L.info[tl.prob];
-        const TcMaps* mp = L.maps + tl.prob;
+        const TcMaps* mp = &L.maps[tl.prob];
         const bool nn = p.nn != 0;
         const bool narrow = tl.cd < 0;
         const int num_kb = (p.kdim + BK - 1) / BK;
@@ -234,35 +316,22 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
         const int prow = rblk >= 0 ? rblk * BM : p.rblocks * BM;
         // this CTA's half of the N columns: a whole column block of a 256-wide tile, half a block of a 128-wide one
         const int qcol = narrow ? tl.cc * 128 + int(rank) * 64 : (rank ? tl.cd : tl.cc) * 128;
-        const uint32_t stage_tx = narrow ? 2 * (A_BYTES + B_BYTES / 2) : 2 * STAGE_BYTES;
+        LoadArgs la;
+        la.mp = mp; la.mat = tl.mat; la.prow = prow; la.qcol = qcol;
+        la.stage_tx = narrow ? 2 * (A_BYTES + B_BYTES / 2) : 2 * STAGE_BYTES;
+        la.leader_cta = leader_cta; la.narrow = narrow;
         // half-stored symmetric operands: k-blocks left of the tile's own block pair are read transposed
-        const int p_flip_kb = p.p_half ? (tl.ra >> 1) * 4 : 0;      // k-blocks [0, p_flip_kb) of P come MN-major
-        const int q_flip_kb = nn ? num_kb : (p.q_half ? (tl.cc >> 1) * 4 : 0);
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
-          const int s = int(it % STAGES);
-          const uint32_t ph = (it / STAGES) & 1u;
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t sa = base + uint32_t(s) * STAGE_BYTES, sb = sa + A_BYTES;
-          if (leader_cta) mbar_expect_tx(full_bar(s), stage_tx);
-          const uint32_t fb = map_to_cta(full_bar(s), 0);
-          const int k0 = kb * BK;
-          if (kb >= p_flip_kb) {                       // 128 rows of P x 64 k
-            tma_load_3d_pair(sa, &mp->p, fb, k0, prow, tl.mat);
-          } else {                                     // the same block read from its mirror image: 64 k-rows x 64 columns, twice
-            tma_load_3d_pair(sa, &mp->ph, fb, prow, k0, tl.mat);
-            tma_load_3d_pair(sa + 64 * BK * 2, &mp->ph, fb, prow + 64, k0, tl.mat);
-          }
-          if (kb >= q_flip_kb) {                       // 128 rows of Q, or the 64 a 128-wide tile needs
-            tma_load_3d_pair(sb, narrow ? &mp->qh : &mp->q, fb, k0, qcol, tl.mat);
-          } else {                                     // 64 k-rows x 64 columns, twice for a 256-wide tile
-            tma_load_3d_pair(sb, &mp->qh, fb, qcol, k0, tl.mat);
-            if (!narrow) tma_load_3d_pair(sb + 64 * BK * 2, &mp->qh, fb, qcol + 64, k0, tl.mat);
-          }
-        }
+        int p_flip_kb = p.p_half ? (tl.ra >> 1) * 4 : 0;            // k-blocks [0, p_flip_kb) of P come MN-major
+        int q_flip_kb = nn ? num_kb : (p.q_half ? (tl.cc >> 1) * 4 : 0);
+        p_flip_kb = p_flip_kb < num_kb ? p_flip_kb : num_kb;
+        q_flip_kb = q_flip_kb < num_kb ? q_flip_kb : num_kb;
+#define MUON_PRODUCE(AM, BM_, B0, B1) produce_range<AM, BM_>(lc, la, B0, B1)
+        MUON_FOR_K_PIECES(MUON_PRODUCE)
+#undef MUON_PRODUCE
       }
       if (!ok) give_up(11);
       if (leader_cta) {   // every armed stage (both CTAs' bytes) has landed before shared memory is released
-        const uint32_t issued = it;
+        const uint32_t issued = lc.it;
         for (uint32_t j = (issued > STAGES ? issued - STAGES : 0); j < issued; ++j) {
           const int s = int(j % STAGES);
           const uint32_t ph = (j / STAGES) & 1u;
@@ -276,39 +345,26 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
     if (lane == 0) {
       if (leader_cta) {
-        uint32_t it = 0, tile_it = 0;
+        LoopCtx lc{base, bars, abort_flag, 0u};
+        uint32_t tile_it = 0;
         bool ok = true;
         for (int t = pair_id; t < total_tiles && ok; t += num_pairs, ++tile_it) {
           const Tile tl = decode_tile(t, L);
           const TcProbInfo& p = L.info[tl.prob];
           const bool nn = p.nn != 0;
           const int num_kb = (p.kdim + BK - 1) / BK;
-          const int umma_n = tl.cd >= 0 ? 256 : 128;
-          const int p_flip_kb = p.p_half ? (tl.ra >> 1) * 4 : 0;
-          const int q_flip_kb = nn ? num_kb : (p.q_half ? (tl.cc >> 1) * 4 : 0);
+          const uint32_t idesc_base = make_idesc(false, 2 * BM, tl.cd >= 0 ? 256 : 128);
+          int p_flip_kb = p.p_half ? (tl.ra >> 1) * 4 : 0;
+          int q_flip_kb = nn ? num_kb : (p.q_half ? (tl.cc >> 1) * 4 : 0);
+          p_flip_kb = p_flip_kb < num_kb ? p_flip_kb : num_kb;
+          q_flip_kb = q_flip_kb < num_kb ? q_flip_kb : num_kb;
           const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
           if (!mbar_wait(tempty_bar(int(acc)), aph ^ 1u, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + acc * 256u;
-          for (int kb = 0; kb < num_kb; ++kb, ++it) {
-            const int s = int(it % STAGES);
-            const uint32_t ph = (it / STAGES) & 1u;
-            if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t sa = base + uint32_t(s) * STAGE_BYTES, sb = sa + A_BYTES;
-            const bool a_mn = kb < p_flip_kb, b_mn = kb < q_flip_kb;
-            const uint32_t idesc = make_idesc(b_mn, 2 * BM, umma_n, a_mn);
-#pragma unroll
-            for (int k = 0; k < BK / UK; ++k) {
-              // K-major: 16 k = 32 bytes along a 128-byte row; MN-major: 16 k-rows of 128 bytes, 64-element chunks 8 KiB apart
-              const uint64_t ad = a_mn ? make_desc(sa + uint32_t(k) * (UK * 128), 64 * BK * 2, 1024)
-                                       : make_desc(sa + uint32_t(k) * (UK * 2), 16, 1024);
-              const uint64_t bd = b_mn ? make_desc(sb + uint32_t(k) * (UK * 128), 64 * BK * 2, 1024)
-                                       : make_desc(sb + uint32_t(k) * (UK * 2), 16, 1024);
-              tc_mma_pair(d_tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-            }
-            tc_commit_pair(empty_bar(s));
-          }
+#define MUON_ISSUE(AM, BM_, B0, B1) issue_range<AM, BM_>(lc, d_tmem, idesc_base, B0, B1)
+          MUON_FOR_K_PIECES(MUON_ISSUE)
+#undef MUON_ISSUE
           if (ok) tc_commit_pair(tfull_bar(int(acc)));
         }
         if (!ok) give_up(13);

@@ -50,7 +50,7 @@ constexpr int kMaxProblems = kMaxElemChunks;
 
 // By-value arguments of one grouped launch.
 struct TcLaunch {
-  const TcMaps* maps;        // device, one per problem
+  TcMaps maps[kMaxProblems];
   TcProbInfo info[kMaxProblems];
   int32_t nprob, total_tiles;
   float alpha, beta;
@@ -62,7 +62,7 @@ struct TcLaunch {
 
 // Host view of one product launch of a launch set: the device maps plus the by-value problem records.
 struct TcTable {
-  const TcMaps* maps = nullptr;
+  TcMaps maps[kMaxProblems];
   TcProbInfo info[kMaxProblems];
   int32_t nprob = 0, total_tiles = 0;
 };
