@@ -35,23 +35,41 @@ template <> __device__ __forceinline__ float load_g<float>(const float* p) { ret
 // Where the rows of a matrix live inside the buffers w/g/m/o point at.  Dense or strided matrices are one
 // run of rows with pitch ld; in flat-shard mode a matrix is a few runs of whole rows (sorted by row, covering
 // every row) with pitch cols.  A thread's four rows almost always fall into one run, so the cursor keeps the
-// current run and only searches when a row leaves it.
+// current run and only searches when a row leaves it.  The block first copies the matrix's run table into
+// shared memory (one coalesced load instead of a chain of dependent global loads per thread); a table longer
+// than kSegCache is searched in global memory.
+constexpr int kSegCache = 32;
+
 template <bool FLAT>
 struct RowCursor {
   int row_begin, row_end;
   size_t base, pitch;
-  __device__ __forceinline__ void init(const MatDesc& d, const RowSeg* __restrict__ segs, int r) {
+  const RowSeg* table;      // the matrix's runs: shared-memory copy or global table
+  int count;
+  // every thread of the block must call this (it contains a barrier in flat-shard mode)
+  __device__ __forceinline__ void prepare(const MatDesc& d, const RowSeg* __restrict__ segs, RowSeg* cache) {
+    if (!FLAT) return;
+    count = d.seg_count;
+    if (count <= kSegCache) {
+      if (int(threadIdx.x) < count) cache[threadIdx.x] = segs[d.seg_begin + threadIdx.x];
+      __syncthreads();
+      table = cache;
+    } else {
+      table = segs + d.seg_begin;
+    }
+  }
+  __device__ __forceinline__ void init(const MatDesc& d, int r) {
     if (!FLAT) {
       row_begin = 0; row_end = d.rows; base = 0; pitch = size_t(d.ld);
     } else {
       pitch = size_t(d.cols);
-      seek(d, segs, r);
+      seek(r);
     }
   }
-  __device__ __forceinline__ void seek(const MatDesc& d, const RowSeg* __restrict__ segs, int r) {
+  __device__ __forceinline__ void seek(int r) {
     row_begin = 0; row_end = 0; base = 0;
-    for (int i = 0; i < d.seg_count; ++i) {
-      const RowSeg sg = segs[d.seg_begin + i];
+    for (int i = 0; i < count; ++i) {
+      const RowSeg sg = table[i];
       if (r < sg.row_begin + sg.row_count) {
         row_begin = sg.row_begin; row_end = sg.row_begin + sg.row_count; base = size_t(sg.flat_offset);
         return;
@@ -59,9 +77,9 @@ struct RowCursor {
     }
   }
   // element offset of (r, 0); r must be a valid row of the matrix
-  __device__ __forceinline__ size_t at(const MatDesc& d, const RowSeg* __restrict__ segs, int r) {
+  __device__ __forceinline__ size_t at(const MatDesc& d, int r) {
     if (!FLAT) return size_t(unsigned(r)) * unsigned(d.ld);
-    if (r >= row_end) seek(d, segs, r);
+    if (r >= row_end) seek(r);
     return base + size_t(r - row_begin) * pitch;
   }
 };
@@ -116,15 +134,17 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
   // 16-byte (fp32) / 8-byte (bf16) accesses need columns, pitch and, in flat-shard mode, every segment offset in fours
   const bool vec = ((d.cols | int(d.ld)) & 3) == 0 && (!FLAT || a.flat_vec >= 4);
   float sum = 0.f;
+  __shared__ RowSeg seg_cache[FLAT ? kSegCache : 1];
   RowCursor<FLAT> cur;
-  cur.init(d, a.segs, min(r0 + ty, d.rows - 1));
+  cur.prepare(d, a.segs, seg_cache);
+  cur.init(d, min(r0 + ty, d.rows - 1));
 #pragma unroll
   for (int pass = 0; pass < 4; ++pass) {
     const int rr = ty + pass * 16, cc = tx * 4;
     const int r = r0 + rr, c = c0 + cc;
     float u[4] = {0.f, 0.f, 0.f, 0.f};
     if (r < d.rows && c < d.cols) {
-      const size_t off = cur.at(d, a.segs, r) + c;
+      const size_t off = cur.at(d, r) + c;
       float g[4], m[4] = {0.f, 0.f, 0.f, 0.f};
       const int nv = min(4, d.cols - c);
       if (vec) {
@@ -254,13 +274,15 @@ __global__ void __launch_bounds__(256, FLAT ? 5 : 6) apply_kernel(ApplyArgs a) {
   float w[4][4];
   alignas(16) XT xv[4][4];
   size_t offs[FLAT ? 4 : 1];
+  __shared__ RowSeg seg_cache[FLAT ? kSegCache : 1];
   if (FLAT) {
     RowCursor<true> cur;
-    cur.init(d, a.segs, min(r0 + ty, d.rows - 1));
+    cur.prepare(d, a.segs, seg_cache);
+    cur.init(d, min(r0 + ty, d.rows - 1));
 #pragma unroll
     for (int pass = 0; pass < 4; ++pass) {
       const int r = r0 + ty + pass * 16;
-      offs[FLAT ? pass : 0] = r < d.rows ? cur.at(d, a.segs, r) + c : 0;
+      offs[FLAT ? pass : 0] = r < d.rows ? cur.at(d, r) + c : 0;
     }
   }
   // ---- loads: W (update mode), then O
@@ -404,14 +426,16 @@ __global__ void __launch_bounds__(256, 6) stage_wide_kernel(StageArgs a) {
     __nv_bfloat16* __restrict__ X = reinterpret_cast<__nv_bfloat16*>(a.ws + ch.x_off) + size_t(bp.mat_local) * ch.s * ldx;
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     const int c = c0 + 8 * tx;
+    __shared__ RowSeg seg_cache[FLAT ? kSegCache : 1];
     RowCursor<FLAT> cur;
-    cur.init(d, a.segs, min(r0 + ty, d.rows - 1));
+    cur.prepare(d, a.segs, seg_cache);
+    cur.init(d, min(r0 + ty, d.rows - 1));
     if (c < d.cols) {
 #pragma unroll
       for (int pass = 0; pass < 4; ++pass) {
         const int rl = ty + pass * 16, r = r0 + rl;
         if (r < d.rows) {
-          const size_t off = cur.at(d, a.segs, r) + size_t(c);
+          const size_t off = cur.at(d, r) + size_t(c);
           float g[8], m[8];
           if (sizeof(GT) == 2) {
             const uint4 raw = __ldcs(reinterpret_cast<const uint4*>(G + off));
@@ -489,13 +513,15 @@ __global__ void __launch_bounds__(256, 6) apply_wide_kernel(ApplyArgs a) {
   const int c = c0 + 8 * tx;
   const bool col_ok = c < d.cols;
   size_t offs[4];
+  __shared__ RowSeg seg_cache[FLAT ? kSegCache : 1];
   {
     RowCursor<FLAT> cur;
-    cur.init(d, a.segs, min(r0 + ty, d.rows - 1));
+    cur.prepare(d, a.segs, seg_cache);
+    cur.init(d, min(r0 + ty, d.rows - 1));
 #pragma unroll
     for (int pass = 0; pass < 4; ++pass) {
       const int r = r0 + ty + pass * 16;
-      offs[pass] = r < d.rows ? cur.at(d, a.segs, r) + size_t(c) : 0;
+      offs[pass] = r < d.rows ? cur.at(d, r) + size_t(c) : 0;
     }
   }
   if (d.transposed) {

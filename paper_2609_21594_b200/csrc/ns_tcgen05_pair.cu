@@ -170,7 +170,16 @@ __device__ __forceinline__ EpiTile make_epi(const Tile& tl, int rank, const TcLa
 struct LoopCtx {
   uint32_t base, bars;          // shared-memory addresses of the stage ring and of the barrier block
   volatile int* abort_flag;
-  uint32_t it;                  // k-blocks processed so far by this role (ring position and phase)
+  uint32_t it;                  // k-blocks processed so far by this role
+  uint32_t s, ph;               // ring position and phase of k-block `it` (kept incrementally: no division in the loop)
+  uint32_t full0_leader;        // cluster address of the leader CTA's full[0] barrier
+  __device__ __forceinline__ void advance() {
+    ++it;
+    if (++s == uint32_t(STAGES)) {
+      s = 0;
+      ph ^= 1u;
+    }
+  }
 };
 __device__ __forceinline__ uint32_t full_bar_of(const LoopCtx& c, int s) { return c.bars + uint32_t(s) * 8u; }
 __device__ __forceinline__ uint32_t empty_bar_of(const LoopCtx& c, int s) { return c.bars + uint32_t(STAGES + s) * 8u; }
@@ -184,13 +193,12 @@ struct LoadArgs {
 
 template <bool A_MN, bool B_MN>
 __device__ __forceinline__ bool produce_range(LoopCtx& c, const LoadArgs& a, int kb_begin, int kb_end) {
-  for (int kb = kb_begin; kb < kb_end; ++kb, ++c.it) {
-    const int s = int(c.it % STAGES);
-    const uint32_t ph = (c.it / STAGES) & 1u;
-    if (!mbar_wait(empty_bar_of(c, s), ph ^ 1u, c.abort_flag)) return false;
+  for (int kb = kb_begin; kb < kb_end; ++kb, c.advance()) {
+    const int s = int(c.s);
+    if (!mbar_wait(empty_bar_of(c, s), c.ph ^ 1u, c.abort_flag)) return false;
     const uint32_t sa = c.base + uint32_t(s) * STAGE_BYTES, sb = sa + A_BYTES;
     if (a.leader_cta) mbar_expect_tx(full_bar_of(c, s), a.stage_tx);
-    const uint32_t fb = map_to_cta(full_bar_of(c, s), 0);
+    const uint32_t fb = c.full0_leader + uint32_t(s) * 8u;
     const int k0 = kb * BK;
     if (!A_MN) {                                   // 128 rows of P x 64 k
       tma_load_3d_pair(sa, &a.mp->p, fb, k0, a.prow, a.mat);
@@ -216,10 +224,9 @@ __device__ __forceinline__ bool issue_range(LoopCtx& c, uint32_t d_tmem, uint32_
   constexpr uint64_t a_hi = A_MN ? DESC_HI_MN : DESC_HI_K, b_hi = B_MN ? DESC_HI_MN : DESC_HI_K;
   constexpr uint32_t a_step = A_MN ? (UK * 128) >> 4 : (UK * 2) >> 4, b_step = B_MN ? (UK * 128) >> 4 : (UK * 2) >> 4;
   const uint32_t idesc = idesc_base | idesc_major;
-  for (int kb = kb_begin; kb < kb_end; ++kb, ++c.it) {
-    const int s = int(c.it % STAGES);
-    const uint32_t ph = (c.it / STAGES) & 1u;
-    if (!mbar_wait(full_bar_of(c, s), ph, c.abort_flag)) return false;
+  for (int kb = kb_begin; kb < kb_end; ++kb, c.advance()) {
+    const int s = int(c.s);
+    if (!mbar_wait(full_bar_of(c, s), c.ph, c.abort_flag)) return false;
     tc_fence_after();
     const uint32_t a0 = (c.base + uint32_t(s) * STAGE_BYTES) >> 4, b0 = a0 + (A_BYTES >> 4);
 #pragma unroll
@@ -302,7 +309,7 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (one per CTA)
     if (lane == 0) {
-      LoopCtx lc{base, bars, abort_flag, 0u};
+      LoopCtx lc{base, bars, abort_flag, 0u, 0u, 0u, map_to_cta(full_bar(0), 0)};
       bool ok = true;
       for (int t = pair_id; t < total_tiles && ok; t += num_pairs) {
         const Tile tl = decode_tile(t, L);
@@ -345,7 +352,7 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
     if (lane == 0) {
       if (leader_cta) {
-        LoopCtx lc{base, bars, abort_flag, 0u};
+        LoopCtx lc{base, bars, abort_flag, 0u, 0u, 0u, 0u};
         uint32_t tile_it = 0;
         bool ok = true;
         for (int t = pair_id; t < total_tiles && ok; t += num_pairs, ++tile_it) {
