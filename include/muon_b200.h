@@ -175,6 +175,57 @@ int muon_materialize(muon_ctx_t* ctx, const void* flat_buf, const muon_layout_t*
 int muon_scatter(muon_ctx_t* ctx, void* flat_buf, const muon_layout_t* layout,
                  const void* const* matrices, void* stream);
 
+/* ------------------------------------------------------------------ owner-sharded step (several ranks)
+ * The pieces of the paper's shard-domain deduplication (Section 6.4, Figure "Two-level deduplication" (a)) and of
+ * its batch pipeline (Section 6.7, Algorithm 2), as calls a rank makes on the shard it holds.  The library does
+ * no communication: the caller moves the staged shards and the updates between ranks (all-gather in, broadcast
+ * out) and these calls do everything else.  One step of one batch on rank r of S:
+ *     muon_shard_momentum(layout, r, G_r, M_r, U_r)            momentum on the local shard; U_r is what the
+ *                                                              fused gather sends (step 1)
+ *     [all-gather U_0..U_{S-1} into one flat buffer]
+ *     muon_materialize_owned(flat U, layout, owned matrices)   only the owner materialises a matrix (step 2)
+ *     muon_orthogonalize_batched(owned matrices)               batched Newton-Schulz over core-shape groups
+ *     [broadcast every owner's updates]                        relay broadcast (step 3)
+ *     muon_shard_apply(layout, r, W_r, updates)                slice extraction and update with decay (step 4)
+ * Momentum and parameters stay sharded throughout.  Assembled this way the step is bit-identical to
+ * muon_step_batched on the whole matrices. */
+
+/* Host-only: compute-owner assignment and batching.  Matrices are packed into batches in descending size
+ * (Section 6.7: large matrices first; a batch is closed when the next matrix would take it beyond batch_elems
+ * elements; batch_elems <= 0: one batch), and inside a batch each matrix is assigned to exactly one of `ranks`
+ * owners by greedy balancing of its Newton-Schulz work, 3 s^2 l + s^3 (Section 6.4 step 2: "greedy size
+ * balancing"): matrices in descending work, each to the least-loaded rank, lowest rank on ties.  Deterministic;
+ * a batch's largest load is within 4/3 - 1/(3 ranks) of the best possible.  owner_of[i], batch_of[i] receive
+ * rank and batch of matrix i (-1 for empty matrices); *num_batches the number of batches. */
+int muon_owner_plan(const muon_shape_t* shapes, int32_t count, int32_t ranks, int64_t batch_elems,
+                    int32_t* owner_of, int32_t* batch_of, int32_t* num_batches);
+
+/* Shard-local momentum (Section 6.4 step 1, the part before the gather): for every element of shard `shard`
+ * of the layout,  M <- mu*M + G;  staged = cast(G + mu*M)  (opt.nesterov) or cast(M).
+ *   local_grads   : device, opt.grad_dtype, the shard_len elements of this shard (element 0 = flat offset
+ *                   shard*shard_len)
+ *   local_momenta : device, fp32, same extent, in/out
+ *   local_staged  : device, NS element type, same extent, out
+ * Padding elements are neither read nor written. */
+int muon_shard_momentum(muon_ctx_t* ctx, const muon_layout_t* layout, int32_t shard, const void* local_grads,
+                        void* local_momenta, void* local_staged, float mu, void* stream);
+
+/* muon_materialize / muon_scatter for a subset: entries of `matrices` that are NULL are skipped (an owner
+ * materialises only the matrices assigned to it, Section 6.4 step 2, and packs only its own updates, step 3). */
+int muon_materialize_owned(muon_ctx_t* ctx, const void* flat_buf, const muon_layout_t* layout,
+                           void* const* matrices, void* stream);
+int muon_scatter_owned(muon_ctx_t* ctx, void* flat_buf, const muon_layout_t* layout,
+                       const void* const* matrices, void* stream);
+
+/* Shard-local slice-and-apply (Section 6.4 step 4): for every element of shard `shard`,
+ *     W <- W (1 - lr*wd) - lr * 0.2 sqrt(max(rows, cols)) * O[matrix][element]
+ * where updates[i] is the whole rows x cols update of matrix i in the NS element type (the payload of the relay
+ * broadcast, wherever the caller received it); the slice this shard holds is taken from it on the fly.
+ *   local_params : device, fp32, the shard_len elements of this shard, in/out
+ *   updates      : host array [num_matrices] of device pointers; NULL = leave that matrix's slice alone */
+int muon_shard_apply(muon_ctx_t* ctx, const muon_layout_t* layout, int32_t shard, void* local_params,
+                     const void* const* updates, float lr, float wd, void* stream);
+
 /* muon_step_batched: one Muon update of `count` independent matrices (Section 2.3, Eq. 1;
  * the complete-matrix path of Algorithm 2: momentum, batched Newton-Schulz, apply):
  *     M <- mu*M + G;  u = G + mu*M (Nesterov) or M;  U = cast(u)

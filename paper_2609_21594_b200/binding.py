@@ -70,6 +70,12 @@ _sig = {
     "muon_layout_destroy": (None, [_vp]),
     "muon_materialize": (C.c_int, [_vp, _vp, _vp, C.POINTER(_vp), _vp]),
     "muon_scatter": (C.c_int, [_vp, _vp, _vp, C.POINTER(_vp), _vp]),
+    "muon_owner_plan": (C.c_int, [C.POINTER(Shape), C.c_int32, C.c_int32, C.c_int64, C.POINTER(C.c_int32), C.POINTER(C.c_int32),
+                                  C.POINTER(C.c_int32)]),
+    "muon_shard_momentum": (C.c_int, [_vp, _vp, C.c_int32, _vp, _vp, _vp, C.c_float, _vp]),
+    "muon_materialize_owned": (C.c_int, [_vp, _vp, _vp, C.POINTER(_vp), _vp]),
+    "muon_scatter_owned": (C.c_int, [_vp, _vp, _vp, C.POINTER(_vp), _vp]),
+    "muon_shard_apply": (C.c_int, [_vp, _vp, C.c_int32, _vp, C.POINTER(_vp), C.c_float, C.c_float, _vp]),
     "muon_step_batched": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(Shape), C.c_int32,
                                     C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
     "muon_step_batched_out": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(Shape),
@@ -174,6 +180,16 @@ def muon_symmetric_tiles(blocks: int) -> List[Tuple[int, int, int, int]]:
     buf = (C.c_uint16 * max(1, 4 * n.value))()
     _check(lib.muon_symmetric_tiles(blocks, buf, n.value, C.byref(n)), "muon_symmetric_tiles")
     return [(buf[4 * i], buf[4 * i + 1], buf[4 * i + 2], buf[4 * i + 3]) for i in range(n.value)]
+
+
+def muon_owner_plan(shapes, ranks: int, batch_elems: int = 0) -> Tuple[List[int], List[int], int]:
+    """(owner_of, batch_of, num_batches): compute owners and batches of the owner-sharded step (host only)."""
+    n = len(shapes)
+    owner = (C.c_int32 * max(1, n))()
+    batch = (C.c_int32 * max(1, n))()
+    nb = C.c_int32(0)
+    _check(lib.muon_owner_plan(_shapes(shapes), n, ranks, batch_elems, owner, batch, C.byref(nb)), "muon_owner_plan")
+    return [int(owner[i]) for i in range(n)], [int(batch[i]) for i in range(n)], int(nb.value)
 
 
 def make_layout_desc(layout, elem_size: int):
@@ -301,6 +317,23 @@ class Context:
     def muon_scatter(self, flat, layout: Layout, matrices, stream=None) -> None:
         _check(lib.muon_scatter(self.handle, flat.data_ptr(), layout.handle, _ptrs(matrices), _stream(stream)),
                "muon_scatter")
+
+    # -- owner-sharded step: the shard-local halves and the subset copies
+    def muon_shard_momentum(self, layout: Layout, shard: int, local_grads, local_momenta, local_staged, mu, stream=None) -> None:
+        _check(lib.muon_shard_momentum(self.handle, layout.handle, shard, local_grads.data_ptr(), local_momenta.data_ptr(),
+                                       local_staged.data_ptr(), mu, _stream(stream)), "muon_shard_momentum")
+
+    def muon_materialize_owned(self, flat, layout: Layout, matrices, stream=None) -> None:
+        _check(lib.muon_materialize_owned(self.handle, flat.data_ptr(), layout.handle, _ptrs(matrices), _stream(stream)),
+               "muon_materialize_owned")
+
+    def muon_scatter_owned(self, flat, layout: Layout, matrices, stream=None) -> None:
+        _check(lib.muon_scatter_owned(self.handle, flat.data_ptr(), layout.handle, _ptrs(matrices), _stream(stream)),
+               "muon_scatter_owned")
+
+    def muon_shard_apply(self, layout: Layout, shard: int, local_params, updates, lr, wd, stream=None) -> None:
+        _check(lib.muon_shard_apply(self.handle, layout.handle, shard, local_params.data_ptr(), _ptrs(updates), lr, wd,
+                                    _stream(stream)), "muon_shard_apply")
 
     # -- compute
     def muon_step_batched(self, params, grads, momenta, shapes, lr, mu, wd, ns_steps, coeffs, stream=None) -> None:

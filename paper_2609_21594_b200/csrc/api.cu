@@ -105,15 +105,16 @@ struct Span {
   }
 };
 
-Plan* get_plan(muon_ctx* ctx, const muon_shape_t* shapes, int32_t count, int* status) {
+Plan* get_plan(muon_ctx* ctx, const muon_shape_t* shapes, int32_t count, int* status, const uint8_t* odd_pitch = nullptr) {
   std::string key(reinterpret_cast<const char*>(shapes), size_t(count) * sizeof(muon_shape_t));
+  if (odd_pitch) key.append(reinterpret_cast<const char*>(odd_pitch), size_t(count));
   auto it = ctx->plans.find(key);
   if (it != ctx->plans.end()) {
     *status = MUON_OK;
     return &it->second;
   }
   Plan p;
-  *status = build_plan(ctx->opt, shapes, count, &p);
+  *status = build_plan(ctx->opt, shapes, count, &p, odd_pitch);
   if (*status != MUON_OK) return nullptr;
   if (ctx->plans.size() > 64) {
     for (auto& kv : ctx->plans) release_plan_tables(&kv.second);
@@ -148,7 +149,6 @@ struct SetRun {
   const SetTables* tables;      // null: per-group engines
   const MatDesc* d_descs;       // device, first record of the SET
   const RowSeg* d_segs;         // flat-shard mode, else null
-  bool pitch8;
   int32_t flat_vec;
 };
 
@@ -156,7 +156,7 @@ int fill_elem_chunks(const SetRun& sr, bool want_wide, int x_index, ElemChunk* o
   int n = 0;
   for (int32_t ci : sr.set->chunks) {
     const Chunk& c = (*sr.chunks)[size_t(ci)];
-    const bool wide = sr.pitch8 && c.s % 8 == 0 && c.l % 8 == 0;
+    const bool wide = c.pitch8 && c.s % 8 == 0 && c.l % 8 == 0;
     if (wide != want_wide) continue;
     ElemChunk& e = out[n++];
     e.block_begin = 0;
@@ -253,7 +253,7 @@ int run_set(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStream_t st)
       sa.segs = sr.d_segs;
       sa.descs = sr.d_descs;
       sa.ws = base;
-      sa.partials = reinterpret_cast<float*>(base + sr.set->off_partials);
+      sa.partials = reinterpret_cast<double*>(base + sr.set->off_partials);
       sa.rnorm = reinterpret_cast<float*>(base + sr.set->off_rnorm);
       sa.mu = r.mu; sa.eps = ctx->opt.eps;
       sa.nesterov = ctx->opt.nesterov;
@@ -330,12 +330,19 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
                 const muon_shape_t* shapes, int32_t count, const ChunkRun& r, cudaStream_t st,
                 const HostPipe* pipe = nullptr, const int64_t* lds = nullptr, const muon_layout* flat = nullptr) {
   int status;
-  Plan* plan = get_plan(ctx, shapes, count, &status);
+  std::vector<uint8_t> odd;                            // strided views whose pitch rules out the 8-element kernels
+  if (lds) {
+    odd.resize(size_t(count), 0);
+    bool any = false;
+    for (int32_t i = 0; i < count; ++i)
+      if (lds[i] % 8) odd[size_t(i)] = 1, any = true;
+    if (!any) odd.clear();
+  }
+  Plan* plan = get_plan(ctx, shapes, count, &status, odd.empty() ? nullptr : odd.data());
   if (!plan) return status;
   if (plan->live == 0) return MUON_OK;
   if (!ctx->ws || ctx->ws_bytes < plan->ws_bytes) return MUON_ERR_WORKSPACE_TOO_SMALL;
   std::vector<MatDesc> descs(size_t(plan->live));
-  bool pitch8 = true;                                  // every row pitch a multiple of 8 elements
   for (const Chunk& ch : plan->chunks) {
     for (int32_t j = 0; j < ch.count; ++j) {
       const int32_t i = ch.mats[size_t(j)];
@@ -351,7 +358,6 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
       d.cols = shapes[i].cols;
       d.ld = lds ? lds[i] : int64_t(d.cols);
       if (d.ld < d.cols || d.ld > 0x7fffffffLL) return MUON_ERR_INVALID_ARG;
-      if (d.ld % 8) pitch8 = false;
       d.seg_begin = flat ? flat->rowseg_begin[size_t(i)] : 0;
       d.seg_count = flat ? flat->rowseg_count[size_t(i)] : 0;
       d.transposed = d.rows > d.cols ? 1 : 0;
@@ -374,7 +380,6 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
     sr.tables = grouped ? &(*plan->set_tables)[k] : nullptr;
     sr.d_descs = static_cast<const MatDesc*>(d_descs) + plan->sets[k].desc_begin;
     sr.d_segs = flat ? flat->d_rowsegs : nullptr;
-    sr.pitch8 = pitch8;
     sr.flat_vec = flat ? flat->flat_vec : 8;
     return sr;
   };
@@ -517,7 +522,8 @@ int muon_workspace_bytes(const muon_options_t* opt, const muon_shape_t* shapes, 
   Plan p;
   const int st = build_plan(*opt, shapes, count, &p);
   if (st != MUON_OK) return st;
-  *bytes = p.ws_bytes;
+  // strided views with an odd pitch form groups of their own; the slack covers the alignment of the extra pieces
+  *bytes = p.ws_bytes ? p.ws_bytes + 4096 * p.chunks.size() : 0;
   return MUON_OK;
 }
 
@@ -594,8 +600,18 @@ int muon_layout_create(muon_ctx_t* ctx, const muon_layout_desc_t* desc, muon_lay
       items.push_back(it);
     }
   }
+  // items in flat order: the work of one shard is then a contiguous range (the shard-local kernels use it)
+  std::stable_sort(items.begin(), items.end(), [](const CopyItem& a, const CopyItem& b) { return a.flat_offset < b.flat_offset; });
   muon_layout* L = new (std::nothrow) muon_layout();
   if (!L) return MUON_ERR_CUDA;
+  L->shard_item_begin.assign(size_t(desc->num_shards) + 1, int64_t(items.size()));
+  {
+    size_t k = 0;
+    for (int32_t r = 0; r <= desc->num_shards; ++r) {
+      while (k < items.size() && items[k].flat_offset < int64_t(r) * desc->shard_len) ++k;
+      L->shard_item_begin[size_t(r)] = int64_t(k);
+    }
+  }
   L->desc = *desc;
   L->shapes.assign(desc->shapes, desc->shapes + desc->num_matrices);
   L->desc.shapes = nullptr;
@@ -640,11 +656,24 @@ int muon_layout_create(muon_ctx_t* ctx, const muon_layout_desc_t* desc, muon_lay
       return MUON_ERR_CUDA;
     }
   }
+  if (desc->num_matrices > 0) {
+    std::vector<float> scales(size_t(desc->num_matrices));
+    for (int32_t i = 0; i < desc->num_matrices; ++i)
+      scales[size_t(i)] = float(0.2 * std::sqrt(double(std::max(desc->shapes[i].rows, desc->shapes[i].cols))));
+    if (cudaMalloc(&L->d_scales, scales.size() * sizeof(float)) != cudaSuccess ||
+        cudaMemcpy(L->d_scales, scales.data(), scales.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
+      if (L->d_scales) cudaFree(L->d_scales);
+      if (L->d_rowsegs) cudaFree(L->d_rowsegs);
+      delete L;
+      return MUON_ERR_CUDA;
+    }
+  }
   if (!items.empty()) {
     if (cudaMalloc(&L->d_items, items.size() * sizeof(CopyItem)) != cudaSuccess ||
         cudaMemcpy(L->d_items, items.data(), items.size() * sizeof(CopyItem), cudaMemcpyHostToDevice) != cudaSuccess) {
       if (L->d_items) cudaFree(L->d_items);
       if (L->d_rowsegs) cudaFree(L->d_rowsegs);
+      if (L->d_scales) cudaFree(L->d_scales);
       delete L;
       return MUON_ERR_CUDA;
     }
@@ -655,13 +684,15 @@ int muon_layout_create(muon_ctx_t* ctx, const muon_layout_desc_t* desc, muon_lay
 
 void muon_layout_destroy(muon_layout_t* L) {
   if (!L) return;
-  if (L->d_items || L->d_rowsegs) cudaDeviceSynchronize();
+  if (L->d_items || L->d_rowsegs || L->d_scales) cudaDeviceSynchronize();
   if (L->d_items) cudaFree(L->d_items);
   if (L->d_rowsegs) cudaFree(L->d_rowsegs);
+  if (L->d_scales) cudaFree(L->d_scales);
   delete L;
 }
 
-static int copy_common(muon_ctx_t* ctx, void* flat, const muon_layout_t* L, void* const* mats, bool scatter, void* stream) {
+static int copy_common(muon_ctx_t* ctx, void* flat, const muon_layout_t* L, void* const* mats, bool scatter, void* stream,
+                       bool subset = false) {
   if (!ctx || !L) return MUON_ERR_INVALID_ARG;
   if (L->num_items == 0) return MUON_OK;
   if (!flat || !mats || !aligned(flat, 16)) return MUON_ERR_INVALID_ARG;
@@ -669,7 +700,8 @@ static int copy_common(muon_ctx_t* ctx, void* flat, const muon_layout_t* L, void
   const size_t es = size_t(L->desc.elem_size);
   for (int32_t i = 0; i < L->desc.num_matrices; ++i) {
     const bool empty = L->shapes[size_t(i)].rows == 0 || L->shapes[size_t(i)].cols == 0;
-    if (!empty && (!mats[i] || !aligned(mats[i], es))) return MUON_ERR_INVALID_ARG;
+    if (!empty && !mats[i] && !subset) return MUON_ERR_INVALID_ARG;
+    if (mats[i] && !aligned(mats[i], es)) return MUON_ERR_INVALID_ARG;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   void* d_mats = nullptr;
@@ -691,6 +723,70 @@ int muon_materialize(muon_ctx_t* ctx, const void* flat_buf, const muon_layout_t*
 int muon_scatter(muon_ctx_t* ctx, void* flat_buf, const muon_layout_t* layout, const void* const* matrices,
                  void* stream) {
   return copy_common(ctx, flat_buf, layout, const_cast<void* const*>(matrices), true, stream);
+}
+
+int muon_materialize_owned(muon_ctx_t* ctx, const void* flat_buf, const muon_layout_t* layout, void* const* matrices,
+                           void* stream) {
+  return copy_common(ctx, const_cast<void*>(flat_buf), layout, matrices, false, stream, true);
+}
+
+int muon_scatter_owned(muon_ctx_t* ctx, void* flat_buf, const muon_layout_t* layout, const void* const* matrices,
+                       void* stream) {
+  return copy_common(ctx, flat_buf, layout, const_cast<void* const*>(matrices), true, stream, true);
+}
+
+int muon_owner_plan(const muon_shape_t* shapes, int32_t count, int32_t ranks, int64_t batch_elems, int32_t* owner_of,
+                    int32_t* batch_of, int32_t* num_batches) {
+  return owner_plan_host(shapes, count, ranks, batch_elems, owner_of, batch_of, num_batches);
+}
+
+static int shard_common(muon_ctx_t* ctx, const muon_layout_t* L, int32_t shard) {
+  if (!ctx || !L || shard < 0 || shard >= L->desc.num_shards) return MUON_ERR_INVALID_ARG;
+  if (!DeviceGuardCheck::ok(ctx) || L->device != ctx->device) return MUON_ERR_CUDA;
+  return MUON_OK;
+}
+
+int muon_shard_momentum(muon_ctx_t* ctx, const muon_layout_t* layout, int32_t shard, const void* local_grads,
+                        void* local_momenta, void* local_staged, float mu, void* stream) {
+  const int rc = shard_common(ctx, layout, shard);
+  if (rc != MUON_OK) return rc;
+  if (!std::isfinite(mu)) return MUON_ERR_INVALID_ARG;
+  const int64_t b = layout->shard_item_begin[size_t(shard)], e = layout->shard_item_begin[size_t(shard) + 1];
+  if (e == b) return MUON_OK;
+  if (!local_grads || !local_momenta || !local_staged) return MUON_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Span sp(ctx, MUON_PHASE_MOMENTUM, st);
+  const int n = launch_shard_momentum(layout->d_items + b, e - b, int64_t(shard) * layout->desc.shard_len, local_grads, local_momenta,
+                                      local_staged, mu, ctx->opt.nesterov, ctx->opt.grad_dtype, ctx->opt.ns_precision, st);
+  if (n < 0) return n;
+  ctx->launches += n;
+  sp.end(n);
+  return MUON_OK;
+}
+
+int muon_shard_apply(muon_ctx_t* ctx, const muon_layout_t* layout, int32_t shard, void* local_params,
+                     const void* const* updates, float lr, float wd, void* stream) {
+  const int rc = shard_common(ctx, layout, shard);
+  if (rc != MUON_OK) return rc;
+  if (!std::isfinite(lr) || !std::isfinite(wd)) return MUON_ERR_INVALID_ARG;
+  const int64_t b = layout->shard_item_begin[size_t(shard)], e = layout->shard_item_begin[size_t(shard) + 1];
+  if (e == b) return MUON_OK;
+  if (!local_params || !updates) return MUON_ERR_INVALID_ARG;
+  const size_t es = elem_bytes_of_ns(ctx->opt.ns_precision);
+  for (int32_t i = 0; i < layout->desc.num_matrices; ++i)
+    if (updates[i] && !aligned(updates[i], es)) return MUON_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  void* d_updates = nullptr;
+  const int urc = upload(ctx, updates, size_t(layout->desc.num_matrices) * sizeof(void*), st, &d_updates);
+  if (urc != MUON_OK) return urc;
+  Span sp(ctx, MUON_PHASE_UPDATE, st);
+  const int n = launch_shard_apply(layout->d_items + b, e - b, int64_t(shard) * layout->desc.shard_len, local_params,
+                                   static_cast<const void* const*>(d_updates), layout->d_scales, lr, 1.0f - lr * wd,
+                                   ctx->opt.ns_precision, st);
+  if (n < 0) return n;
+  ctx->launches += n;
+  sp.end(n);
+  return MUON_OK;
 }
 
 static int check_common(muon_ctx_t* ctx, const muon_shape_t* shapes, int32_t count, int32_t ns_steps, const float* coeffs) {
@@ -1068,7 +1164,6 @@ extern "C" int muon_orthogonalize_static(const void* in, void* out, int32_t rows
   sr.tables = grouped ? &img.tables : nullptr;
   sr.d_descs = d_desc;
   sr.d_segs = nullptr;
-  sr.pitch8 = cols % 8 == 0;
   sr.flat_vec = 8;
   return run_set(&ctx, sr, r, st);
 }

@@ -2,7 +2,7 @@
 //   stage : M <- mu*M + G, u = G + mu*M (Nesterov), U = cast(u) written into the NS workspace in
 //           wide orientation (transposed through shared memory when rows > cols: the
 //           transpose-first rule of Section 6.6), plus per-tile sums of U^2
-//   norm  : r = 1 / (sqrt(sum U^2) + eps) per matrix, fixed-order reduction (Eq. 1, second line)
+//   norm  : r = 1 / (sqrt(sum U^2) + eps) per matrix, fixed-order reduction in double (Eq. 1, second line)
 //   apply : W <- W (1 - lr*wd) - lr * 0.2 sqrt(max(m,n)) * O, O read back through the transpose
 // All three are HBM-bound.  Reductions use a fixed shuffle/shared-memory tree and per-tile
 // partial sums, never floating-point atomics, so results are bit-identical run to run.
@@ -84,13 +84,16 @@ struct RowCursor {
   }
 };
 
-__device__ __forceinline__ float block_sum_256(float v, float* red) {
+// Sums of squares are carried in double from the first addition on: a square of a bf16 or fp32 value is exact in
+// double, and the accumulated rounding (about 1e-16 relative) is far below the final rounding of the reciprocal
+// norm to fp32 -- so the norm a matrix gets does not depend on which kernel variant (or tiling) summed it.
+__device__ __forceinline__ double block_sum_256(double v, double* red) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   const int w = threadIdx.x >> 5;
   if ((threadIdx.x & 31) == 0) red[w] = v;
   __syncthreads();
-  float t = 0.f;
+  double t = 0.0;
   if (threadIdx.x == 0) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) t += red[i];
@@ -120,7 +123,7 @@ __device__ __forceinline__ BlockPos locate_block(const Args& a) {
 template <typename GT, typename XT, bool MOM, bool FLAT>
 __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
   __shared__ XT tile[T][PADT];
-  __shared__ float red[8];
+  __shared__ double red[8];
   const BlockPos bp = locate_block(a);
   const ElemChunk ch = a.ch[bp.ci];
   const int t = bp.tile, ldx = ch.ldx;
@@ -133,7 +136,7 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   // 16-byte (fp32) / 8-byte (bf16) accesses need columns, pitch and, in flat-shard mode, every segment offset in fours
   const bool vec = ((d.cols | int(d.ld)) & 3) == 0 && (!FLAT || a.flat_vec >= 4);
-  float sum = 0.f;
+  double sum = 0.0;
   __shared__ RowSeg seg_cache[FLAT ? kSegCache : 1];
   RowCursor<FLAT> cur;
   cur.prepare(d, a.segs, seg_cache);
@@ -170,8 +173,8 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         if (MOM) {
-          m[i] = a.mu * m[i] + g[i];
-          u[i] = a.nesterov ? g[i] + a.mu * m[i] : m[i];
+          m[i] = __fmaf_rn(a.mu, m[i], g[i]);             // explicit roundings: every route to M' and u computes the same bits
+          u[i] = a.nesterov ? __fmaf_rn(a.mu, m[i], g[i]) : m[i];
         } else {
           u[i] = g[i];
         }
@@ -187,7 +190,7 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         xv[i] = XConv<XT>::from(u[i]);
-        const float q = XConv<XT>::to(xv[i]);
+        const double q = double(XConv<XT>::to(xv[i]));
         if (i < nv) sum += q * q;
       }
       if (!d.transposed) {
@@ -226,7 +229,7 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
       }
     }
   }
-  const float tot = block_sum_256(sum, red);
+  const double tot = block_sum_256(sum, red);
   if (threadIdx.x == 0) a.partials[ch.part_off + int64_t(bp.mat_local) * ch.tiles + t] = tot;
 }
 
@@ -240,9 +243,9 @@ __global__ void __launch_bounds__(256) norm_kernel(StageArgs a) {
   }
   const ElemChunk ch = a.ch[ci];
   const int mat_local = int(blockIdx.x) - first;
-  const float* p = a.partials + ch.part_off + int64_t(mat_local) * ch.tiles;
+  const double* p = a.partials + ch.part_off + int64_t(mat_local) * ch.tiles;
   double acc = 0.0;
-  for (int i = threadIdx.x; i < ch.tiles; i += 256) acc += double(p[i]);
+  for (int i = threadIdx.x; i < ch.tiles; i += 256) acc += p[i];
   red[threadIdx.x] = acc;
   __syncthreads();
   for (int o = 128; o > 0; o >>= 1) {
@@ -412,13 +415,13 @@ __host__ __device__ inline int wide_tiles(int rows, int cols) { return ((rows + 
 template <typename GT, bool MOM, bool FLAT>
 __global__ void __launch_bounds__(256, 6) stage_wide_kernel(StageArgs a) {
   __shared__ __align__(16) unsigned char tsm[WC * 128];
-  __shared__ float red[8];
+  __shared__ double red[8];
   const BlockPos bp = locate_block(a);
   const ElemChunk ch = a.ch[bp.ci];
   const int t = bp.tile, ldx = ch.ldx;
   const MatDesc d = a.descs[ch.desc_begin + bp.mat_local];
   const int tiles_c = (d.cols + WC - 1) / WC;
-  float sum = 0.f;
+  double sum = 0.0;
   if (t < wide_tiles(d.rows, d.cols)) {                      // block-uniform: the grid is sized for the larger orientation
     const int r0 = (t / tiles_c) * WR, c0 = (t % tiles_c) * WC;
     const GT* __restrict__ G = static_cast<const GT*>(d.g);
@@ -456,8 +459,8 @@ __global__ void __launch_bounds__(256, 6) stage_wide_kernel(StageArgs a) {
             m[0] = m0.x; m[1] = m0.y; m[2] = m0.z; m[3] = m0.w; m[4] = m1.x; m[5] = m1.y; m[6] = m1.z; m[7] = m1.w;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-              m[i] = a.mu * m[i] + g[i];
-              g[i] = a.nesterov ? g[i] + a.mu * m[i] : m[i];      // g now holds u
+              m[i] = __fmaf_rn(a.mu, m[i], g[i]);                 // explicit roundings, as in every other route to M' and u
+              g[i] = a.nesterov ? __fmaf_rn(a.mu, m[i], g[i]) : m[i];   // g now holds u
             }
             __stcs(reinterpret_cast<float4*>(M + off), make_float4(m[0], m[1], m[2], m[3]));
             __stcs(reinterpret_cast<float4*>(M + off) + 1, make_float4(m[4], m[5], m[6], m[7]));
@@ -467,7 +470,7 @@ __global__ void __launch_bounds__(256, 6) stage_wide_kernel(StageArgs a) {
           for (int i = 0; i < 4; ++i) {
             const __nv_bfloat162 b = __floats2bfloat162_rn(g[2 * i], g[2 * i + 1]);
             pk[i] = *reinterpret_cast<const uint32_t*>(&b);
-            const float q0 = __uint_as_float(pk[i] << 16), q1 = __uint_as_float(pk[i] & 0xffff0000u);
+            const double q0 = double(__uint_as_float(pk[i] << 16)), q1 = double(__uint_as_float(pk[i] & 0xffff0000u));
             sum += q0 * q0;
             sum += q1 * q1;
           }
@@ -494,7 +497,7 @@ __global__ void __launch_bounds__(256, 6) stage_wide_kernel(StageArgs a) {
       }
     }
   }
-  const float tot = block_sum_256(sum, red);
+  const double tot = block_sum_256(sum, red);
   if (threadIdx.x == 0) a.partials[ch.part_off + int64_t(bp.mat_local) * ch.tiles + t] = tot;
 }
 

@@ -44,6 +44,7 @@ struct Chunk {
   int32_t tiles_per_mat = 0;     // elementwise 64x64 tiles per matrix
   int32_t desc_begin = 0;        // index of the first MatDesc of this chunk in the uploaded table
   int32_t set = 0;               // launch set this chunk belongs to
+  bool pitch8 = true;            // every matrix of the chunk has a row pitch that is a multiple of 8 elements
   size_t off_x[2] = {0, 0}, off_a = 0, off_b = 0;   // byte offsets of the chunk's buffers in the workspace
   int64_t part_off = 0;          // float index of the chunk's tile partial sums inside the set's partial-sum area
   std::vector<int32_t> mats;     // caller indices, in caller order
@@ -72,7 +73,8 @@ struct Plan {
 };
 
 size_t elem_bytes_of_ns(int ns_precision);
-int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t count, Plan* plan);
+int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t count, Plan* plan,
+               const uint8_t* odd_pitch = nullptr);
 // Lays the chunks of one launch set out in a workspace (fills Chunk::off_*, part_off and the set's offsets).
 void layout_set(const muon_options_t& opt, std::vector<Chunk>* chunks, LaunchSet* set);
 // Tile list of a symmetric product over nb x nb blocks of 128: every unordered pair of blocks exactly once.
@@ -81,6 +83,8 @@ struct TilePatHost {
 };
 std::vector<TilePatHost> symmetric_tile_pattern(int nb);
 int validate_layout_host(const muon_layout_desc_t* d);
+int owner_plan_host(const muon_shape_t* shapes, int32_t count, int32_t ranks, int64_t batch_elems, int32_t* owner_of,
+                    int32_t* batch_of, int32_t* num_batches);
 
 // Copy work item of the gather/scatter kernel.
 struct alignas(16) CopyItem {
@@ -109,8 +113,10 @@ struct PhaseSpan {
 struct muon_layout {
   muon_layout_desc_t desc;            // shapes/segments pointers are nulled after create
   std::vector<muon_shape_t> shapes;
-  muon::CopyItem* d_items = nullptr;
+  muon::CopyItem* d_items = nullptr;                 // sorted by flat offset: the items of a shard are contiguous
   int64_t num_items = 0;
+  std::vector<int64_t> shard_item_begin;              // num_shards + 1 entries into d_items
+  float* d_scales = nullptr;                          // per matrix: 0.2 * sqrt(max(rows, cols))
   int device = 0;
   std::vector<std::vector<muon_segment_t>> segs_of;   // host copy of the segment table, grouped by matrix
   bool row_aligned = false;                           // every segment holds whole rows: the flat buffers can be addressed in place
@@ -147,6 +153,11 @@ namespace muon {
 int launch_copy(const CopyItem* items, int64_t num_items, void* flat, void* const* d_mats, int elem_size,
                 bool scatter, cudaStream_t st);
 
+int launch_shard_momentum(const CopyItem* items, int64_t num_items, int64_t shard_base, const void* g, void* m, void* staged,
+                          float mu, int nesterov, int grad_dtype, int ns_precision, cudaStream_t st);
+int launch_shard_apply(const CopyItem* items, int64_t num_items, int64_t shard_base, void* w, const void* const* d_updates,
+                       const float* d_scales, float lr, float decay, int ns_precision, cudaStream_t st);
+
 // One shape group inside an elementwise launch.
 struct ElemChunk {
   int32_t block_begin;   // first block of this chunk in the launch
@@ -163,7 +174,7 @@ struct StageArgs {
   const RowSeg* segs;     // device row-segment table (flat-shard mode), else null
   const MatDesc* descs;   // device, first record of the launch set
   char* ws;               // device, workspace base
-  float* partials;        // device, the set's partial sums
+  double* partials;       // device, the set's tile sums of squares
   float* rnorm;           // device, one per matrix of the set
   float mu, eps;
   int32_t nesterov, grad_dtype, ns_precision;

@@ -19,18 +19,22 @@ size_t elem_bytes_of_ns(int ns_precision) { return ns_precision == MUON_NS_FP32 
 // then packed into launch sets of at most chunk_elems elements in total (first fit, largest chunk
 // first): the chunks of a set are resident in the workspace together and share every launch, so a
 // set -- not a chunk -- is the unit the cap bounds.
-int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t count, Plan* plan) {
+// `odd_pitch` (may be null) marks strided views whose row pitch is not a multiple of 8 elements: they form groups
+// of their own, so that the elementwise kernels chosen for a matrix -- and with them the order in which its norm is
+// summed -- never depend on what else is in the call.
+int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t count, Plan* plan, const uint8_t* odd_pitch) {
   plan->chunks.clear();
   plan->sets.clear();
   plan->ws_bytes = 0;
   plan->live = 0;
-  std::map<std::pair<int32_t, int32_t>, std::vector<int32_t>> groups;
-  std::vector<std::pair<int32_t, int32_t>> order;
+  typedef std::pair<std::pair<int32_t, int32_t>, int32_t> GroupKey;      // ((s, l), odd pitch)
+  std::map<GroupKey, std::vector<int32_t>> groups;
+  std::vector<GroupKey> order;
   for (int32_t i = 0; i < count; ++i) {
     const int32_t r = shapes[i].rows, c = shapes[i].cols;
     if (r < 0 || c < 0) return MUON_ERR_INVALID_ARG;
     if (r == 0 || c == 0) continue;
-    const std::pair<int32_t, int32_t> key(std::min(r, c), std::max(r, c));
+    const GroupKey key(std::make_pair(std::min(r, c), std::max(r, c)), (odd_pitch && odd_pitch[i]) ? 1 : 0);
     auto it = groups.find(key);
     if (it == groups.end()) {
       order.push_back(key);
@@ -43,7 +47,7 @@ int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t co
   std::vector<Chunk> chunks;
   for (const auto& key : order) {
     const std::vector<int32_t>& idx = groups[key];
-    const int64_t per = int64_t(key.first) * key.second;
+    const int64_t per = int64_t(key.first.first) * key.first.second;
     // as few chunks as the cap allows, of (nearly) equal size: a short last chunk would run its fifteen
     // products on a mostly idle device
     const int64_t max_per_chunk = std::max<int64_t>(1, cap / per);
@@ -52,8 +56,9 @@ int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t co
     size_t b = 0;
     for (int64_t ci = 0; ci < num_chunks; ++ci) {
       Chunk ch;
-      ch.s = key.first;
-      ch.l = key.second;
+      ch.s = key.first.first;
+      ch.l = key.first.second;
+      ch.pitch8 = key.second == 0;
       ch.ldx = int32_t(up(size_t(ch.l), 8));
       ch.lda = int32_t(up(size_t(ch.s), 8));
       const size_t e = b + base + (size_t(ci) < rem ? 1 : 0);
@@ -106,7 +111,7 @@ int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t co
 }
 
 // Workspace of a launch set: per chunk X0, X1 [K, s, ldx] and A, B [K, s, lda] in the NS element type
-// (every piece 256-byte aligned), then the set's tile partial sums and one reciprocal norm per matrix.
+// (every piece 256-byte aligned), then the set's tile sums of squares (double) and one reciprocal norm per matrix.
 void layout_set(const muon_options_t& opt, std::vector<Chunk>* chunks, LaunchSet* set) {
   const size_t eb = elem_bytes_of_ns(opt.ns_precision);
   size_t off = 0;
@@ -126,7 +131,7 @@ void layout_set(const muon_options_t& opt, std::vector<Chunk>* chunks, LaunchSet
     parts += int64_t(c.count) * c.tiles_per_mat;
   }
   set->off_partials = off;
-  off += up(size_t(parts) * sizeof(float), 256);
+  off += up(size_t(parts) * sizeof(double), 256);
   set->off_rnorm = off;
   off += up(size_t(set->count) * sizeof(float), 256);
   set->bytes = off;
@@ -154,6 +159,52 @@ std::vector<TilePatHost> symmetric_tile_pattern(int nb) {
     tiles.push_back(TilePatHost{uint16_t(L), none, uint16_t(L), none});
   }
   return tiles;
+}
+
+// Compute-owner assignment and batching of the owner-sharded step (Section 6.4 step 2; Section 6.7 and
+// Algorithm 2).  Matrices are packed into batches in descending size (large matrices first, so that their result
+// broadcasts have the longest window to hide in); a batch is closed when the next matrix would take it past
+// batch_elems elements.  Inside a batch every matrix gets exactly one owner by greedy balancing of the
+// Newton-Schulz work (longest processing time first: matrices in descending cost, each to the rank with the
+// least work so far, lowest rank on ties), which keeps a batch's makespan within 4/3 - 1/(3 ranks) of optimal.
+// The cost of a matrix is what the engine really computes per iteration: 3 s^2 l + s^3 multiply-adds.
+int owner_plan_host(const muon_shape_t* shapes, int32_t count, int32_t ranks, int64_t batch_elems, int32_t* owner_of,
+                    int32_t* batch_of, int32_t* num_batches) {
+  if (count < 0 || ranks < 1 || (count > 0 && (!shapes || !owner_of || !batch_of)) || !num_batches) return MUON_ERR_INVALID_ARG;
+  std::vector<int32_t> live;
+  for (int32_t i = 0; i < count; ++i) {
+    if (shapes[i].rows < 0 || shapes[i].cols < 0) return MUON_ERR_INVALID_ARG;
+    owner_of[i] = batch_of[i] = -1;
+    if (shapes[i].rows > 0 && shapes[i].cols > 0) live.push_back(i);
+  }
+  auto elems = [&](int32_t i) { return int64_t(shapes[i].rows) * shapes[i].cols; };
+  auto cost = [&](int32_t i) {
+    const double s = std::min(shapes[i].rows, shapes[i].cols), l = std::max(shapes[i].rows, shapes[i].cols);
+    return 3.0 * s * s * l + s * s * s;
+  };
+  std::stable_sort(live.begin(), live.end(), [&](int32_t a, int32_t b) { return elems(a) > elems(b); });
+  int32_t nb = 0;
+  size_t pos = 0;
+  while (pos < live.size()) {
+    size_t end = pos;
+    int64_t filled = 0;
+    while (end < live.size() && (end == pos || batch_elems <= 0 || filled + elems(live[end]) <= batch_elems)) filled += elems(live[end++]);
+    std::vector<int32_t> batch(live.begin() + long(pos), live.begin() + long(end));
+    std::stable_sort(batch.begin(), batch.end(), [&](int32_t a, int32_t b) { return cost(a) > cost(b); });
+    std::vector<double> load(static_cast<size_t>(ranks), 0.0);
+    for (int32_t i : batch) {
+      size_t best = 0;
+      for (size_t r = 1; r < load.size(); ++r)
+        if (load[r] < load[best]) best = r;
+      load[best] += cost(i);
+      owner_of[i] = int32_t(best);
+      batch_of[i] = nb;
+    }
+    ++nb;
+    pos = end;
+  }
+  *num_batches = nb;
+  return MUON_OK;
 }
 
 int validate_layout_host(const muon_layout_desc_t* d) {

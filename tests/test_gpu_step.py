@@ -172,6 +172,14 @@ def test_batched_equals_alone_and_rerun_bit_exact(engine):
     for i, m in enumerate(mats):
         alone, _ = _ortho(mb, ctx, [m])
         assert np.array_equal(alone[0], together[i]), i
+    # a matrix whose row pitch rules out the 16-byte kernels must not change how its neighbours are summed
+    mixed_shapes = [(256, 256), (37, 53), (384, 640)]
+    mixed = [mats[0], wl.grad_np("batch", 0, 7, (37, 53)), wl.grad_np("batch", 0, 8, (384, 640))]
+    mixed_out, _ = _ortho(mb, ctx, mixed)
+    assert np.array_equal(mixed_out[0], together[0])
+    for i in (1, 2):
+        alone, _ = _ortho(mb, ctx, [mixed[i]])
+        assert np.array_equal(alone[0], mixed_out[i]), mixed_shapes[i]
     # a small chunk cap changes the batching but not the numbers
     ctx2 = _ctx(mb, "bf16", engine, chunk_elems=70000)
     capped, _ = _ortho(mb, ctx2, mats)
