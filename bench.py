@@ -349,6 +349,64 @@ def side_config(mb, name, cfg, shapes, dev, path, steps, peaks, local, layout_ki
     return rec
 
 
+def run_owner(args, world, rank, local):
+    """--parallelism owner: ONE optimizer step of the whole matrix set spread over the ranks (the owner-sharded
+    step of Section 6.4 / Algorithm 2): every rank holds one row shard of every parameter, momentum and gradient,
+    the staged shards are all-gathered per batch, each matrix is orthogonalised by its compute owner only, updates
+    are broadcast and every rank applies its slice.  Total work is fixed as N grows (strong scaling)."""
+    from paper_2609_21594_b200 import binding as mb
+    from paper_2609_21594_b200 import owner_sharded as osd
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the Muon path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    shapes = wl.shapes_llama8b(args.layers) if args.config == "llama8b" else wl.CONFIGS[args.config]()
+    ctx = mb.Context()
+    comm = osd.TorchComm() if world > 1 else osd.SingleComm()
+    st = osd.OwnerShardedStep(shapes, osd.CudaOps(ctx, device=dev), comm, batch_elems=args.batch_elems)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(wl.stream_seed(args.config, 0, rank, "owner"))
+    for b in range(len(st.batches)):
+        st.params[b].normal_(0.0, 0.02, generator=gen)
+        st.momenta[b].zero_()
+        st.grads[b].copy_(torch.randn(st.grads[b].shape, generator=gen, device=dev, dtype=torch.float32).mul_(1e-3))
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        st.step(LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.muon_launch_count()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier(world)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(args.steps):
+        st.step(LR, MU, WD, wl.NS_STEPS, wl.QUINTIC)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier(world)
+    clocks = sampler.stop() if rank == 0 else {}
+    ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
+    launches = ctx.muon_launch_count() - launches0
+    if ctx.muon_synchronize_and_check() != 0:
+        raise SystemExit("a bounded device-side wait expired during the timed region")
+    if rank != 0:
+        return
+    owned = [s for s, o in zip(shapes, st.owner_of) if o == rank]
+    line = {
+        "metric": METRIC, "value": 1e3 / ms, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{args.config}: {len(shapes)} matrices row-sharded over {world} rank(s), bf16 N(0, 1e-3) grads, fp32 params and momenta",
+                   "parallelism": f"owner-sharded x{world}", "batches": len(st.batches), "matrices_owned_by_rank0": len(owned),
+                   "ns_steps": wl.NS_STEPS, "coeffs": list(wl.QUINTIC), "lr": LR, "mu": MU, "wd": WD, "l2": "inputs_exceed_l2"},
+        "e2e": None, "gpu_launches": int(launches), "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def run_ours(args, world, rank, local):
     from paper_2609_21594_b200 import binding as mb   # fails loudly when the CUDA library is missing
 
@@ -498,6 +556,10 @@ def main():
                          "copy_only: gather and scatter alone")
     ap.add_argument("--layout", choices=["per_param", "flat_concat"], default="per_param",
                     help="flat-shard layout generator: per-parameter row split, or flat concatenation cut into equal parts")
+    ap.add_argument("--parallelism", choices=["replicas", "owner"], default="replicas",
+                    help="replicas: every rank runs the whole step on its own copy (the benchmark); owner: one step of the "
+                         "whole set spread over the ranks, each matrix orthogonalised by its compute owner")
+    ap.add_argument("--batch-elems", type=int, default=1 << 31, help="with --parallelism owner: elements per gather batch")
     ap.add_argument("--e2e-steps", type=int, default=8)
     ap.add_argument("--no-side-configs", dest="side_configs", action="store_false",
                     help="skip the records of the other configurations (1B, MoE, tiny, sharded-state flow)")
@@ -510,7 +572,10 @@ def main():
         return
     world, rank, local = dist_setup(args.gpus)
     try:
-        run_ours(args, world, rank, local)
+        if args.parallelism == "owner":
+            run_owner(args, world, rank, local)
+        else:
+            run_ours(args, world, rank, local)
     finally:
         if world > 1:
             import torch.distributed as dist

@@ -178,6 +178,7 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
   if (sr.tables) {
     auto launch = [&](const tc::TcTable& tab, float alpha, float beta, int gamma_mode) {
       tc::TcLaunch L;
+      L.persist = nullptr;
       for (int i = 0; i < tab.nprob; ++i) {
         L.maps[i] = tab.maps[i];
         L.info[i] = tab.info[i];
@@ -190,6 +191,32 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
       L.status = ctx->d_status;
       return launch_tc_grouped(ctx->device, L, st);
     };
+    // Small sets: the whole iteration in ONE cooperative launch, products separated by grid barriers instead of
+    // launch boundaries ("per-matrix NS launches starve the device for small matrices", Section 6.6 -- so do
+    // per-product launches when a product is a handful of tiles).
+    if (sr.tables->persist && r.ns_steps <= tc::kMaxPersistSteps && ctx->persist_pairs != 0) {
+      if (ctx->persist_pairs < 0) ctx->persist_pairs = std::max(0, tc_pair_max_resident(ctx->device));
+      const int pairs = std::min(ctx->persist_pairs, sr.tables->max_tiles);
+      if (pairs > 0 && sr.tables->max_tiles <= 2 * ctx->persist_pairs) {
+        tc::TcLaunch L;
+        std::memset(static_cast<void*>(&L), 0, sizeof(L));
+        L.coef_a = L.coef_b = -1;
+        L.status = ctx->d_status;
+        L.persist = sr.tables->persist;
+        L.ns_steps = r.ns_steps;
+        L.barrier = reinterpret_cast<uint32_t*>(ctx->d_status + 16);
+        L.barrier_base = ctx->barrier_count;
+        for (int k = 0; k < r.ns_steps; ++k)
+          for (int j = 0; j < 3; ++j) L.coef[k][j] = r.coeffs[(ctx->opt.coeffs_per_step ? 3 * k : 0) + j];
+        n = launch_tc_persistent(ctx->device, L, pairs, st);
+        if (n > 0) {
+          ctx->barrier_count += uint32_t(3 * r.ns_steps - 1) * uint32_t(2 * pairs);
+          *launches += n;
+          return MUON_OK;
+        }
+        ctx->persist_pairs = 0;      // a cooperative launch is not possible here: one launch per product from now on
+      }
+    }
     for (int k = 0; k < r.ns_steps; ++k) {
       const float* co = r.coeffs + (ctx->opt.coeffs_per_step ? 3 * k : 0);
       const int cur = k & 1;
@@ -931,6 +958,7 @@ int muon_ns_product(muon_ctx_t* ctx, const void* p, const void* q, const void* d
     rc = commit_slot(slot, img.data(), img.size(), st);
     if (rc != MUON_OK) return rc;
     tc::TcLaunch L;
+    L.persist = nullptr;
     L.maps[0] = tab.maps[0];
     L.info[0] = tab.info[0];
     L.nprob = 1;
@@ -1149,7 +1177,7 @@ extern "C" int muon_orthogonalize_static(const void* in, void* out, int32_t rows
   SetImage img;
   const bool grouped = grouped_engine(&ctx);
   if (grouped) {
-    rc = build_set_image(encode, ctx.ws, chunks, set, sb + kStaticTablesOff, &img, nullptr);
+    rc = build_set_image(encode, ctx.ws, chunks, set, sb + kStaticTablesOff, &img, nullptr, false);
     if (rc != MUON_OK) return rc;
     if (img.bytes.size() > kStaticHeader - kStaticTablesOff) return MUON_ERR_TOO_LARGE;
     img.bytes.resize((img.bytes.size() + 15) / 16 * 16, 0);

@@ -141,6 +141,8 @@ struct muon_ctx {
   int64_t phase_launches[MUON_NUM_PHASES] = {0, 0, 0, 0, 0};
   int64_t launches = 0;
   int64_t tmap_encodes = 0;                        // tensor maps encoded so far (plan binding and the per-launch engines)
+  uint32_t barrier_count = 0;                      // arrivals the grid-barrier counter (d_status[16]) has seen so far
+  int persist_pairs = -1;                          // CTA pairs a whole-iteration launch may use (-1: not asked yet, 0: off)
   void* tmap_encode = nullptr;                     // cuTensorMapEncodeTiled, resolved at run time
   cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;   // copy streams of the host-buffer path (created on first use)
   std::vector<cudaEvent_t> sync_events;            // untimed events that order the copy streams against the caller's stream

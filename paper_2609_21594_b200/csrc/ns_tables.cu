@@ -11,6 +11,7 @@
 namespace muon {
 
 using tc::TcMaps;
+using tc::TcPersist;
 using tc::TcProbInfo;
 using tc::TcTable;
 using tc::TilePat;
@@ -52,7 +53,7 @@ size_t add_pattern(ImageBuilder* ib, int nb, int32_t* count) {
 }  // namespace
 
 int build_set_image(void* encode_fn, const void* ws, const std::vector<Chunk>& chunks, const LaunchSet& set,
-                    const void* dev_base, SetImage* out, int64_t* encodes) {
+                    const void* dev_base, SetImage* out, int64_t* encodes, bool with_persist) {
   if (!encode_fn) return MUON_ERR_CUDA;
   ImageBuilder ib;
   ib.dev_base = static_cast<const char*>(dev_base);
@@ -163,6 +164,24 @@ int build_set_image(void* encode_fn, const void* ws, const std::vector<Chunk>& c
       tab.info[j] = p;
     }
     tab.total_tiles = tile_begin;
+  }
+  if (with_persist) {  // the five tables once more, in device memory, for the whole-iteration launch
+    const size_t off = ib.reserve(sizeof(TcPersist), 128);
+    TcPersist* pp = new TcPersist();
+    std::memset(static_cast<void*>(pp), 0, sizeof(TcPersist));
+    const TcTable* tabs[5] = {&T.g1[0], &T.g1[1], &T.g2, &T.g3[0], &T.g3[1]};
+    pp->nprob = n;
+    for (int kind = 0; kind < 5; ++kind) {
+      for (int j = 0; j < n; ++j) {
+        pp->maps[kind][j] = tabs[kind]->maps[j];
+        pp->info[kind][j] = tabs[kind]->info[j];
+      }
+      pp->total_tiles[kind] = tabs[kind]->total_tiles;
+      T.max_tiles = std::max(T.max_tiles, tabs[kind]->total_tiles);
+    }
+    std::memcpy(ib.bytes.data() + off, pp, sizeof(TcPersist));
+    delete pp;
+    T.persist = static_cast<const TcPersist*>(ib.dev(off));
   }
   out->bytes = std::move(ib.bytes);
   out->tables = T;

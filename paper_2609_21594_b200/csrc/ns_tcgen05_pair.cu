@@ -103,11 +103,42 @@ struct Tile {
   int cc, cd;    // column blocks (cd = -1: the tile is 128 columns wide)
 };
 
-__device__ __forceinline__ Tile decode_tile(int t, const TcLaunch& L) {
+// What one product of the launch looks like to the kernel: its problem list and its epilogue scalars.
+struct PhaseView {
+  const TcMaps* maps;
+  const TcProbInfo* info;
+  int nprob, total_tiles;
+  float alpha, beta;
+  int gamma_mode;
+};
+
+// Product `ph` of the launch.  A one-product launch carries its tables by value; a whole-iteration launch reads
+// them from device memory and derives the scalars of step k = ph / 3 from the coefficient rows:
+// A = gamma X X^T (gamma = r^2 at k = 0), B = b A + c A A^T, X' = gamma (a X + B X) (gamma = r at k = 0).
+__device__ __forceinline__ PhaseView phase_view(const TcLaunch& L, int ph) {
+  PhaseView v;
+  if (!L.persist) {
+    v.maps = L.maps; v.info = L.info; v.nprob = L.nprob; v.total_tiles = L.total_tiles;
+    v.alpha = L.alpha; v.beta = L.beta; v.gamma_mode = L.gamma_mode;
+    return v;
+  }
+  const int k = ph / 3, j = ph - 3 * k, cur = k & 1;
+  const int kind = j == 0 ? cur : (j == 1 ? 2 : 3 + cur);
+  v.maps = L.persist->maps[kind];
+  v.info = L.persist->info[kind];
+  v.nprob = L.persist->nprob;
+  v.total_tiles = L.persist->total_tiles[kind];
+  v.alpha = j == 1 ? L.coef[k][2] : 1.f;
+  v.beta = j == 0 ? 0.f : (j == 1 ? L.coef[k][1] : L.coef[k][0]);
+  v.gamma_mode = k == 0 ? (j == 0 ? 2 : (j == 2 ? 1 : 0)) : 0;
+  return v;
+}
+
+__device__ __forceinline__ Tile decode_tile(int t, const PhaseView& V) {
   int pi = 0;
-  for (int i = 1; i < L.nprob; ++i)
-    if (t >= L.info[i].tile_begin) pi = i;
-  const TcProbInfo& p = L.info[pi];
+  for (int i = 1; i < V.nprob; ++i)
+    if (t >= V.info[i].tile_begin) pi = i;
+  const TcProbInfo& p = V.info[pi];
   Tile r;
   r.prob = pi;
   const int u = t - p.tile_begin;
@@ -130,11 +161,11 @@ __device__ __forceinline__ Tile decode_tile(int t, const TcLaunch& L) {
   return r;
 }
 
-__device__ __forceinline__ EpiTile make_epi(const Tile& tl, int rank, const TcLaunch& L) {
+__device__ __forceinline__ EpiTile make_epi(const Tile& tl, int rank, const PhaseView& V, const TcLaunch& L) {
   EpiTile e;
-  const TcProbInfo& p = L.info[tl.prob];
-  e.map_d = &L.maps[tl.prob].d;
-  e.map_c = &L.maps[tl.prob].c;
+  const TcProbInfo& p = V.info[tl.prob];
+  e.map_d = &V.maps[tl.prob].d;
+  e.map_c = &V.maps[tl.prob].c;
   e.d = p.d;
   e.c = p.c;
   e.stride_c = p.stride_c;
@@ -149,11 +180,11 @@ __device__ __forceinline__ EpiTile make_epi(const Tile& tl, int rank, const TcLa
   e.mirror0 = sym && tl.cc != e.rblk && !(in_cols && (tl.cc == tl.ra || tl.cc == tl.rb));
   e.mirror1 = sym && tl.cd != e.rblk && !(in_cols && (tl.cd == tl.ra || tl.cd == tl.rb));
   e.valid = e.rblk >= 0;
-  e.alpha = L.alpha; e.beta = L.beta; e.gamma = 1.f;
+  e.alpha = V.alpha; e.beta = V.beta; e.gamma = 1.f;
   if (e.valid) {
-    if (L.gamma_mode) {
+    if (V.gamma_mode) {
       const float r = p.rnorm[tl.mat];
-      e.gamma = L.gamma_mode == 1 ? r : r * r;
+      e.gamma = V.gamma_mode == 1 ? r : r * r;
     }
     if (p.coef) {
       const float* co = p.coef + size_t(tl.mat) * L.coef_stride;
@@ -162,6 +193,31 @@ __device__ __forceinline__ EpiTile make_epi(const Tile& tl, int rank, const TcLa
     }
   }
   return e;
+}
+
+// Grid-wide barrier of the whole-iteration launch (all CTAs are resident: cooperative launch).  Arrival: one
+// thread per CTA, after its bulk stores have completed, publishes them and adds 1.  Wait: poll (bounded) until
+// every CTA has arrived for product `ph - 1`, then order the bulk loads that follow behind the acquire.
+__device__ __forceinline__ void grid_arrive(uint32_t* counter) {
+  asm volatile("fence.proxy.async;" ::: "memory");
+  __threadfence();
+  atomicAdd(counter, 1u);
+}
+__device__ __forceinline__ bool grid_wait(const TcLaunch& L, int ph, volatile int* abort_flag) {
+  const uint32_t target = L.barrier_base + uint32_t(ph) * gridDim.x;
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  while (true) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(L.barrier) : "memory");
+    if (int32_t(v - target) >= 0) break;
+    if ((++spins & 63u) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > WAIT_CYCLES) return false;
+    }
+  }
+  asm volatile("fence.proxy.async;" ::: "memory");
+  return true;
 }
 
 // ---- main-loop bodies, specialised at compile time on how the two operands are read (K-major as stored, or
@@ -271,7 +327,7 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
   const uint32_t rank = cluster_rank();
   const bool leader_cta = rank == 0;
   const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-  const int total_tiles = L.total_tiles;
+  const int nphase = L.persist ? 3 * L.ns_steps : 1;      // products this launch walks through
   const uint32_t peer_abort = map_to_cta(base + BAR_OFF + 200, rank ^ 1u);
   auto give_up = [&](int code) {                 // tell both CTAs of the pair, then the host
     *abort_flag = 1;
@@ -311,30 +367,34 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
     if (lane == 0) {
       LoopCtx lc{base, bars, abort_flag, 0u, 0u, 0u, map_to_cta(full_bar(0), 0)};
       bool ok = true;
-      for (int t = pair_id; t < total_tiles && ok; t += num_pairs) {
-        const Tile tl = decode_tile(t, L);
-        const TcProbInfo& p = L.info[tl.prob];
-        const TcMaps* mp = &L.maps[tl.prob];
-        const bool nn = p.nn != 0;
-        const bool narrow = tl.cd < 0;
-        const int num_kb = (p.kdim + BK - 1) / BK;
-        // this CTA's 128 rows of P (a missing row block reads beyond the matrix: zero fill)
-        const int rblk = rank ? tl.rb : tl.ra;
-        const int prow = rblk >= 0 ? rblk * BM : p.rblocks * BM;
-        // this CTA's half of the N columns: a whole column block of a 256-wide tile, half a block of a 128-wide one
-        const int qcol = narrow ? tl.cc * 128 + int(rank) * 64 : (rank ? tl.cd : tl.cc) * 128;
-        LoadArgs la;
-        la.mp = mp; la.mat = tl.mat; la.prow = prow; la.qcol = qcol;
-        la.stage_tx = narrow ? 2 * (A_BYTES + B_BYTES / 2) : 2 * STAGE_BYTES;
-        la.leader_cta = leader_cta; la.narrow = narrow;
-        // half-stored symmetric operands: k-blocks left of the tile's own block pair are read transposed
-        int p_flip_kb = p.p_half ? (tl.ra >> 1) * 4 : 0;            // k-blocks [0, p_flip_kb) of P come MN-major
-        int q_flip_kb = nn ? num_kb : (p.q_half ? (tl.cc >> 1) * 4 : 0);
-        p_flip_kb = p_flip_kb < num_kb ? p_flip_kb : num_kb;
-        q_flip_kb = q_flip_kb < num_kb ? q_flip_kb : num_kb;
+      for (int ph = 0; ph < nphase && ok; ++ph) {
+        const PhaseView V = phase_view(L, ph);
+        if (ph > 0 && !grid_wait(L, ph, abort_flag)) { ok = false; break; }   // operands written by the product before
+        for (int t = pair_id; t < V.total_tiles && ok; t += num_pairs) {
+          const Tile tl = decode_tile(t, V);
+          const TcProbInfo& p = V.info[tl.prob];
+          const TcMaps* mp = &V.maps[tl.prob];
+          const bool nn = p.nn != 0;
+          const bool narrow = tl.cd < 0;
+          const int num_kb = (p.kdim + BK - 1) / BK;
+          // this CTA's 128 rows of P (a missing row block reads beyond the matrix: zero fill)
+          const int rblk = rank ? tl.rb : tl.ra;
+          const int prow = rblk >= 0 ? rblk * BM : p.rblocks * BM;
+          // this CTA's half of the N columns: a whole column block of a 256-wide tile, half a block of a 128-wide one
+          const int qcol = narrow ? tl.cc * 128 + int(rank) * 64 : (rank ? tl.cd : tl.cc) * 128;
+          LoadArgs la;
+          la.mp = mp; la.mat = tl.mat; la.prow = prow; la.qcol = qcol;
+          la.stage_tx = narrow ? 2 * (A_BYTES + B_BYTES / 2) : 2 * STAGE_BYTES;
+          la.leader_cta = leader_cta; la.narrow = narrow;
+          // half-stored symmetric operands: k-blocks left of the tile's own block pair are read transposed
+          int p_flip_kb = p.p_half ? (tl.ra >> 1) * 4 : 0;            // k-blocks [0, p_flip_kb) of P come MN-major
+          int q_flip_kb = nn ? num_kb : (p.q_half ? (tl.cc >> 1) * 4 : 0);
+          p_flip_kb = p_flip_kb < num_kb ? p_flip_kb : num_kb;
+          q_flip_kb = q_flip_kb < num_kb ? q_flip_kb : num_kb;
 #define MUON_PRODUCE(AM, BM_, B0, B1) produce_range<AM, BM_>(lc, la, B0, B1)
-        MUON_FOR_K_PIECES(MUON_PRODUCE)
+          MUON_FOR_K_PIECES(MUON_PRODUCE)
 #undef MUON_PRODUCE
+        }
       }
       if (!ok) give_up(11);
       if (leader_cta) {   // every armed stage (both CTAs' bytes) has landed before shared memory is released
@@ -355,24 +415,27 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
         LoopCtx lc{base, bars, abort_flag, 0u, 0u, 0u, 0u};
         uint32_t tile_it = 0;
         bool ok = true;
-        for (int t = pair_id; t < total_tiles && ok; t += num_pairs, ++tile_it) {
-          const Tile tl = decode_tile(t, L);
-          const TcProbInfo& p = L.info[tl.prob];
-          const bool nn = p.nn != 0;
-          const int num_kb = (p.kdim + BK - 1) / BK;
-          const uint32_t idesc_base = make_idesc(false, 2 * BM, tl.cd >= 0 ? 256 : 128);
-          int p_flip_kb = p.p_half ? (tl.ra >> 1) * 4 : 0;
-          int q_flip_kb = nn ? num_kb : (p.q_half ? (tl.cc >> 1) * 4 : 0);
-          p_flip_kb = p_flip_kb < num_kb ? p_flip_kb : num_kb;
-          q_flip_kb = q_flip_kb < num_kb ? q_flip_kb : num_kb;
-          const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-          if (!mbar_wait(tempty_bar(int(acc)), aph ^ 1u, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t d_tmem = tmem_base + acc * 256u;
+        for (int ph = 0; ph < nphase && ok; ++ph) {       // no barrier here: the issuer only consumes what the producers loaded
+          const PhaseView V = phase_view(L, ph);
+          for (int t = pair_id; t < V.total_tiles && ok; t += num_pairs, ++tile_it) {
+            const Tile tl = decode_tile(t, V);
+            const TcProbInfo& p = V.info[tl.prob];
+            const bool nn = p.nn != 0;
+            const int num_kb = (p.kdim + BK - 1) / BK;
+            const uint32_t idesc_base = make_idesc(false, 2 * BM, tl.cd >= 0 ? 256 : 128);
+            int p_flip_kb = p.p_half ? (tl.ra >> 1) * 4 : 0;
+            int q_flip_kb = nn ? num_kb : (p.q_half ? (tl.cc >> 1) * 4 : 0);
+            p_flip_kb = p_flip_kb < num_kb ? p_flip_kb : num_kb;
+            q_flip_kb = q_flip_kb < num_kb ? q_flip_kb : num_kb;
+            const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+            if (!mbar_wait(tempty_bar(int(acc)), aph ^ 1u, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + acc * 256u;
 #define MUON_ISSUE(AM, BM_, B0, B1) issue_range<AM, BM_>(lc, d_tmem, idesc_base, B0, B1)
-          MUON_FOR_K_PIECES(MUON_ISSUE)
+            MUON_FOR_K_PIECES(MUON_ISSUE)
 #undef MUON_ISSUE
-          if (ok) tc_commit_pair(tfull_bar(int(acc)));
+            if (ok) tc_commit_pair(tfull_bar(int(acc)));
+          }
         }
         if (!ok) give_up(13);
         tc_commit_pair(drain_bar);       // arrives in both CTAs once every MMA issued above has finished
@@ -385,31 +448,50 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
     EpilogueState est;
     uint32_t tile_it = 0;
     bool ok = true;
-    bool have = pair_id < total_tiles;
-    Tile tl;
-    if (have) tl = decode_tile(pair_id, L);
-    for (int t = pair_id; have && ok; t += num_pairs, ++tile_it) {
-      const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-      const uint32_t taddr = tmem_base + acc * 256u + (uint32_t(quad * 32) << 16);
-      const EpiTile cur = make_epi(tl, int(rank), L);
-      EpiTile nxt;
-      nxt.valid = false;
-      nxt.d = nullptr;
-      have = t + num_pairs < total_tiles;
-      if (have) {
-        tl = decode_tile(t + num_pairs, L);
-        nxt = make_epi(tl, int(rank), L);
+    for (int ph = 0; ph < nphase && ok; ++ph) {
+      const PhaseView V = phase_view(L, ph);
+      if (ph > 0) {                                 // D chunks and result tiles of this product touch what the last one wrote
+        bool go = true;
+        if (lane == 0) go = grid_wait(L, ph, abort_flag);
+        if (!__shfl_sync(0xffffffffu, go ? 1 : 0, 0)) { ok = false; break; }
       }
-      if (cur.valid) {
-        ok = epilogue_tile(cur, nxt, taddr, epi_base, dfull_bar(0), egroup_bar, tfull_bar(int(acc)), aph, abort_flag, est, quad,
-                           lane);
-      } else {                                     // no rows for this CTA: hand the accumulator straight back
-        ok = mbar_wait(tfull_bar(int(acc)), aph, abort_flag);
+      bool have = pair_id < V.total_tiles;
+      Tile tl;
+      if (have) tl = decode_tile(pair_id, V);
+      for (int t = pair_id; have && ok; t += num_pairs, ++tile_it) {
+        const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+        const uint32_t taddr = tmem_base + acc * 256u + (uint32_t(quad * 32) << 16);
+        const EpiTile cur = make_epi(tl, int(rank), V, L);
+        EpiTile nxt;
+        nxt.valid = false;
+        nxt.d = nullptr;
+        have = t + num_pairs < V.total_tiles;       // the prefetch of D never crosses a product boundary
+        if (have) {
+          tl = decode_tile(t + num_pairs, V);
+          nxt = make_epi(tl, int(rank), V, L);
+        }
+        if (cur.valid) {
+          ok = epilogue_tile(cur, nxt, taddr, epi_base, dfull_bar(0), egroup_bar, tfull_bar(int(acc)), aph, abort_flag, est, quad,
+                             lane);
+        } else {                                    // no rows for this CTA: hand the accumulator straight back
+          ok = mbar_wait(tfull_bar(int(acc)), aph, abort_flag);
+        }
+        if (!ok) break;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(int(acc)), 0));   // the leader CTA counts both epilogues
       }
-      if (!ok) break;
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(int(acc)), 0));   // the leader CTA counts both epilogues
+      if (ok && L.persist && ph + 1 < nphase) {     // this CTA's part of the product is in memory: tell the grid
+        // the four warps meet first, so that every store of the product has been issued by the leader thread
+        __syncwarp();
+        if (lane == 0) mbar_arrive(egroup_bar);
+        ok = mbar_wait(egroup_bar, est.eph, abort_flag);
+        est.eph ^= 1u;
+        if (ok && quad == 2 && lane == 0) {
+          tma_wait_all();
+          grid_arrive(L.barrier);
+        }
+      }
     }
     if (quad == 2 && lane == 0) {
       tma_wait_all();                               // every store has landed before the CTA retires
@@ -454,6 +536,47 @@ int launch_tc_grouped(int device, const tc::TcLaunch& L, cudaStream_t st) {
   const unsigned grid = unsigned(2 * (L.total_tiles < pairs ? L.total_tiles : pairs));
   ns_product_pair_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(L);
   return cudaGetLastError() == cudaSuccess ? 1 : MUON_ERR_CUDA;
+}
+
+int tc_pair_max_resident(int device) {
+  if (tc_pair_grid_setup(device) < 0) return 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2, 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int clusters = 0;
+  if (cudaOccupancyMaxActiveClusters(&clusters, ns_product_pair_kernel, &cfg) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return clusters;
+}
+
+int launch_tc_persistent(int device, const tc::TcLaunch& L, int pairs, cudaStream_t st) {
+  if (!L.persist || pairs < 1) return MUON_ERR_INVALID_ARG;
+  if (tc_pair_grid_setup(device) < 0) return MUON_ERR_CUDA;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(2 * pairs), 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;      // every CTA resident at once: the grid barrier relies on it
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, ns_product_pair_kernel, L) != cudaSuccess) {
+    cudaGetLastError();
+    return MUON_ERR_UNSUPPORTED;
+  }
+  return 1;
 }
 
 }  // namespace muon

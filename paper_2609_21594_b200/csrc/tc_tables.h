@@ -48,6 +48,17 @@ struct TcProbInfo {
 };
 constexpr int kMaxProblems = kMaxElemChunks;
 
+// The five product tables of a launch set in device memory, for the launch that runs a whole Newton-Schulz
+// iteration by itself: [0], [1]: A = X X^T reading X iterate 0 / 1; [2]: B = bA + cA A^T; [3], [4]: X' = aX + B X
+// reading iterate 0 / 1 and writing the other.
+struct alignas(128) TcPersist {
+  TcMaps maps[5][kMaxProblems];
+  TcProbInfo info[5][kMaxProblems];
+  int32_t nprob;
+  int32_t total_tiles[5];
+};
+constexpr int kMaxPersistSteps = 16;
+
 // By-value arguments of one grouped launch.
 struct TcLaunch {
   TcMaps maps[kMaxProblems];
@@ -58,6 +69,13 @@ struct TcLaunch {
   int32_t coef_a, coef_b;    // index into a matrix's coefficient row that replaces alpha / beta (-1: keep the scalar)
   int32_t coef_stride;
   int32_t* status;
+  // Whole-iteration mode (persist != null): the launch walks 3 * ns_steps products, a grid-wide barrier between
+  // consecutive ones, and takes tables from device memory instead of maps / info above.
+  const TcPersist* persist;
+  int32_t ns_steps;
+  uint32_t barrier_base;     // value of *barrier when the launch starts
+  uint32_t* barrier;         // device counter: every CTA adds 1 per finished product
+  float coef[kMaxPersistSteps][3];   // (a_k, b_k, c_k)
 };
 
 // Host view of one product launch of a launch set: the device maps plus the by-value problem records.
@@ -93,10 +111,17 @@ struct SetTables {
   tc::TcTable g1[2];   // A = X X^T, reading X iterate 0 / 1
   tc::TcTable g2;      // B = bA + c A A^T
   tc::TcTable g3[2];   // X' = aX + B X, reading iterate 0 / 1 and writing the other
+  const tc::TcPersist* persist = nullptr;   // the same five tables in device memory (null: not built)
+  int32_t max_tiles = 0;                    // largest tile count of a product
 };
 
-// Launches the paired engine: tensor maps in device memory, everything else by value.
+// Launches the paired engine on one product (tables by value).
 int launch_tc_grouped(int device, const tc::TcLaunch& L, cudaStream_t st);
+// Launches the paired engine on a whole Newton-Schulz iteration (L.persist set): a cooperative launch of `pairs`
+// CTA pairs that must all be resident.  Returns 1, or < 0 when such a launch is not possible here.
+int launch_tc_persistent(int device, const tc::TcLaunch& L, int pairs, cudaStream_t st);
+// How many CTA pairs of the paired kernel can be resident at once on this device (0 when unknown).
+int tc_pair_max_resident(int device);
 // Number of SMs of the device (> 0), after making the paired kernel launchable there; < 0 on error.
 int tc_pair_grid_setup(int device);
 
@@ -113,7 +138,7 @@ struct SetImage {
   SetTables tables;       // device addresses inside refer to dev_base + offset
 };
 int build_set_image(void* encode_fn, const void* ws, const std::vector<Chunk>& chunks, const LaunchSet& set,
-                    const void* dev_base, SetImage* out, int64_t* encodes);
+                    const void* dev_base, SetImage* out, int64_t* encodes, bool with_persist = true);
 
 // Single stand-alone product (muon_ns_product): device image (maps and tile list) plus the by-value table.
 int build_product_image(void* encode_fn, const GemmArgs& g, const void* dev_base, std::vector<char>* bytes, tc::TcTable* table,

@@ -468,37 +468,50 @@ def test_ns_ragged_multi_tile_shapes(engine):
 
 def test_one_launch_per_product_for_all_shape_groups_and_no_encoding_in_steady_state():
     """The tensor engine runs each Newton-Schulz product as one kernel over every shape group that is resident
-    together: the d=256 layer (two core shapes) takes 3 * 5 product launches, not 30, and after the first step on
-    a workspace no tensor map is encoded again."""
+    together (3 * 5 product launches for the 1B-class layer with four core shapes, not 60), a set of a few tiles per
+    product runs the whole iteration in ONE launch, and after the first step on a workspace no tensor map is
+    encoded again."""
     from paper_2609_21594_b200 import binding as mb
 
-    ctx = _ctx(mb, "bf16", "tensor")
-    shapes = wl.shapes_tiny()
-    ctx.ensure_workspace(shapes)
-    ins = [bf16_input(wl.grad_np("grouped", 0, i, s))[0] for i, s in enumerate(shapes)]
-    outs = [torch.empty_like(t) for t in ins]
-    ctx.muon_orthogonalize_batched(ins, outs, shapes, 5, QUINTIC)          # binds the plan: encodes once
-    torch.cuda.synchronize()
-    enc0 = ctx.muon_tensor_map_encodes()
-    assert enc0 > 0
-    ctx.muon_profile_enable(True)
-    ctx.muon_profile_reset()
-    n0 = ctx.muon_launch_count()
-    for _ in range(3):
+    def run(shapes, name):
+        ctx = _ctx(mb, "bf16", "tensor")
+        ctx.ensure_workspace(shapes)
+        ins = [bf16_input(wl.grad_np(name, 0, i, s))[0] for i, s in enumerate(shapes)]
+        outs = [torch.empty_like(t) for t in ins]
+        ctx.muon_orthogonalize_batched(ins, outs, shapes, 5, QUINTIC)          # binds the plan: encodes once
+        torch.cuda.synchronize()
+        first = [o.clone() for o in outs]
+        enc0 = ctx.muon_tensor_map_encodes()
+        assert enc0 > 0
+        ctx.muon_profile_enable(True)
+        ctx.muon_profile_reset()
+        n0 = ctx.muon_launch_count()
+        for _ in range(3):
+            ctx.muon_orthogonalize_batched(ins, outs, shapes, 5, QUINTIC)
+        torch.cuda.synchronize()
+        ph = ctx.muon_profile_read()
+        ctx.muon_profile_enable(False)
+        assert ctx.muon_tensor_map_encodes() == enc0                           # steady state: nothing encoded
+        assert all(torch.equal(a, b) for a, b in zip(first, outs))
+        launches = (ph["ns"][1] // 3, (ctx.muon_launch_count() - n0) // 3)
+        # a new workspace address re-binds once
+        ctx.muon_set_workspace(torch.empty(mb.muon_workspace_bytes(ctx.opt, shapes) + 4096, dtype=torch.uint8, device="cuda"))
         ctx.muon_orthogonalize_batched(ins, outs, shapes, 5, QUINTIC)
-    torch.cuda.synchronize()
-    ph = ctx.muon_profile_read()
-    ctx.muon_profile_enable(False)
-    assert ph["ns"][1] == 3 * 15                                           # product launches: 15 per call
-    assert ctx.muon_launch_count() - n0 == 3 * (15 + 2 + 1)                # + stage, norm, apply (one wide launch each)
-    assert ctx.muon_tensor_map_encodes() == enc0                           # steady state: nothing encoded
-    # a new workspace address re-binds once
-    ctx.muon_set_workspace(torch.empty(mb.muon_workspace_bytes(ctx.opt, shapes) + 4096, dtype=torch.uint8, device="cuda"))
-    ctx.muon_orthogonalize_batched(ins, outs, shapes, 5, QUINTIC)
-    torch.cuda.synchronize()
-    assert ctx.muon_tensor_map_encodes() == 2 * enc0
-    assert ctx.muon_last_device_status() == 0
-    ctx.close()
+        torch.cuda.synchronize()
+        assert ctx.muon_tensor_map_encodes() == 2 * enc0
+        assert all(torch.equal(a, b) for a, b in zip(first, outs))
+        assert ctx.muon_last_device_status() == 0
+        ctx.close()
+        return launches, [host_f64(o) for o in outs], ins
+
+    # d=256 layer, two core shapes, a handful of tiles per product: one launch for the whole iteration
+    (ns, total), outs, ins = run(wl.shapes_tiny(), "grouped")
+    assert ns == 1 and total == 1 + 2 + 1                                      # + stage, norm, apply
+    ref = orc.newton_schulz(host_f64(ins[4]), 5, QUINTIC, 1e-7, "bf16")
+    assert rel(outs[4], ref) <= TOL_BF16
+    # one layer of the 1B-class stack: four core shapes in one launch set, too many tiles for the single launch
+    (ns, total), _, _ = run(wl.shapes_1b(1), "grouped1b")
+    assert ns == 15 and total == 15 + 2 + 1
 
 
 def test_many_small_heterogeneous_matrices():
