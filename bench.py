@@ -232,7 +232,9 @@ class Workload:
         self.n_elem = sum(m * n for m, n in shapes)
         row_scaled = cfg == "llama8b"
         gen = wl.layout_per_param if layout_kind == "per_param" else wl.layout_flat_concat
-        self.layout = gen(shapes, NUM_SHARDS)
+        # 32 equal layers in 8 shards would put every cut of the flat concatenation on a layer boundary: 7 shards there,
+        # so that the cuts fall inside matrices (mid-row)
+        self.layout = gen(shapes, NUM_SHARDS if layout_kind == "per_param" else NUM_SHARDS - 1)
         self.ctx = mb.Context()
         self.L = mb.Layout(self.ctx, self.layout, 2)
         self.ctx.ensure_workspace(shapes)
@@ -492,7 +494,7 @@ def run_ours(args, world, rank, local):
         side["llama8b_flat_state"] = side_config(mb, "llama8b, sharded-state flow (muon_step_flat)", "llama8b", shapes, dev,
                                                  "flat_state", 5, peaks, local)
         side["llama8b_layout_flat_concat_copy_only"] = side_config(
-            mb, "llama8b, gather + scatter only, flat-concatenation layout (cuts fall inside matrices)", "llama8b", shapes, dev,
+            mb, "llama8b, gather + scatter only, flat concatenation cut into 7 shards (cuts fall inside matrices, mid-row)", "llama8b", shapes, dev,
             "copy_only", 5, peaks, local, layout_kind="flat_concat")
         side["1b"] = side_config(mb, "1B-class stack, 112 matrices", "1b", wl.shapes_1b(), dev, "materialize", 10, peaks, local)
         side["moe"] = side_config(mb, "MoE stress, 784 matrices", "moe", wl.shapes_moe(), dev, "materialize", 5, peaks, local)

@@ -107,6 +107,10 @@ typedef struct {
   int32_t engine;          /* MUON_ENGINE_TENSOR (default) | MUON_ENGINE_TENSOR_1CTA | MUON_ENGINE_CUDA_CORE (bf16  */
                            /* products on CUDA cores; slow cross-check); fp32 NS always runs on CUDA cores          */
   int64_t chunk_elems;     /* batching cap in elements per batched NS invocation; default 1<<29 (Section 6.6) */
+  int32_t coeffs_per_matrix; /* 1: `coeffs` holds one row per matrix of the call, [count][3] or [count][3*ns_steps]:   */
+                           /* matrices of one call may iterate with different polynomials (a per-parameter-group  */
+                           /* choice in the pluggable design of Section 6.2); they still share their launches       */
+  int32_t reserved;        /* must be 0 */
 } muon_options_t;
 
 /* Fills *opt with the defaults: bf16 grads, bf16 NS, Nesterov, constant coefficients, eps 1e-7, cap 2^29. */
@@ -235,7 +239,8 @@ int muon_shard_apply(muon_ctx_t* ctx, const muon_layout_t* layout, int32_t shard
  *   params, momenta : host arrays [count] of device pointers to fp32 matrices (in/out)
  *   grads           : host array  [count] of device pointers, element type opt.grad_dtype
  *   shapes          : host, [count]; a matrix with rows==0 or cols==0 is skipped
- *   coeffs          : host, 3 floats (or 3*ns_steps when opt.coeffs_per_step)
+ *   coeffs          : host, 3 floats (or 3*ns_steps when opt.coeffs_per_step); with opt.coeffs_per_matrix one such
+ *                     row per matrix, row i for matrix i of this call
  * All matrix pointers must be 16-byte aligned.  Matrices are batched by core shape; the
  * results do not depend on how they are batched (bit-identical run to run). */
 int muon_step_batched(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
@@ -256,10 +261,19 @@ int muon_step_batched_out(muon_ctx_t* ctx, void* const* params, const void* cons
  * params[i], grads[i], momenta[i] and, when given, updates[i] point at element (0,0) of view i inside
  * tensors that share the physical layout; all use views[i].ld as row stride (ld >= cols).  Pointers must
  * be 16-byte aligned; the vectorised path also needs ld to be a multiple of 4 elements (other strides
- * run element-wise).  Elements outside the views are never touched.  Views of one call must not overlap. */
+ * run element-wise).  Elements outside the views are never touched.  Two views of one call that share an element of
+ * params, momenta or updates are rejected with MUON_ERR_INVALID_ARG before anything is launched (the check is
+ * muon_views_overlap applied to each of the three pointer arrays). */
 int muon_step_batched_views(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
                             void* const* updates, const muon_view_t* views, int32_t count, float lr, float mu,
                             float wd, int32_t ns_steps, const float* coeffs, void* stream);
+
+/* Host arithmetic only (needs no device): *overlap = 1 when two of the strided views -- view i has element (0,0)
+ * at address bases[i], rows x cols elements of elem_size bytes, ld elements between rows -- share a byte, else 0.
+ * Views with rows == 0, cols == 0 or a NULL base are ignored.  This is the check muon_step_batched_views applies to
+ * what it writes, so that the logical matrices of one physical parameter (row blocks of a fused QKV, interleaved
+ * gate/up rows, [E,M,N] planes: the model adapter of Section 6.6) can be validated once when a model is set up. */
+int muon_views_overlap(const void* const* bases, const muon_view_t* views, int32_t count, int32_t elem_size, int32_t* overlap);
 
 /* muon_step_flat: the sharded-state flow of Section 6.4 (steps 1 and 4) on one device -- parameters, momenta and
  * gradients STAY in flat shard buffers that share one layout (in the paper the momentum is never

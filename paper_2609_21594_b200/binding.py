@@ -10,6 +10,8 @@ import ctypes as C
 import os
 from typing import List, Optional, Sequence, Tuple
 
+import numpy as np
+
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmuon_b200.so")
 
@@ -52,7 +54,7 @@ class LayoutDesc(C.Structure):
 class Options(C.Structure):
     _fields_ = [("grad_dtype", C.c_int32), ("ns_precision", C.c_int32), ("nesterov", C.c_int32),
                 ("coeffs_per_step", C.c_int32), ("eps", C.c_float), ("engine", C.c_int32),
-                ("chunk_elems", C.c_int64)]
+                ("chunk_elems", C.c_int64), ("coeffs_per_matrix", C.c_int32), ("reserved", C.c_int32)]
 
 
 _vp = C.c_void_p
@@ -80,6 +82,7 @@ _sig = {
                                     C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
     "muon_step_batched_out": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(Shape),
                                         C.c_int32, C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
+    "muon_views_overlap": (C.c_int, [C.POINTER(_vp), C.POINTER(View), C.c_int32, C.c_int32, C.POINTER(C.c_int32)]),
     "muon_step_batched_views": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(View),
                                           C.c_int32, C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
     "muon_step_flat": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, C.c_float, C.c_float, C.c_float, C.c_int32, C.POINTER(C.c_float), _vp]),
@@ -157,6 +160,16 @@ def muon_workspace_bytes(opt: Options, shapes) -> int:
     out = C.c_size_t(0)
     _check(lib.muon_workspace_bytes(C.byref(opt), _shapes(shapes), len(shapes), C.byref(out)), "muon_workspace_bytes")
     return int(out.value)
+
+
+def muon_views_overlap(bases, views, elem_size: int) -> bool:
+    """bases: addresses (ints) of element (0,0) of each view; views: list of (rows, cols, ld).  Host arithmetic only."""
+    va = (View * max(1, len(views)))()
+    for i, (r, c, ld) in enumerate(views):
+        va[i].rows, va[i].cols, va[i].ld = int(r), int(c), int(ld)
+    out = C.c_int32(0)
+    _check(lib.muon_views_overlap(_ptrs(bases), va, len(views), int(elem_size), C.byref(out)), "muon_views_overlap")
+    return bool(out.value)
 
 
 def muon_plan_describe(opt: Options, shapes) -> Tuple[int, List[int]]:
@@ -241,6 +254,14 @@ def views_of_cols(tensor, col_counts):
     return out
 
 
+def views_of_interleaved_rows(tensor, ways: int):
+    """`ways` logical matrices stored row-interleaved in one 2-D tensor (gate and up projections kept as rows
+    g0, u0, g1, u1, ...): logical matrix w owns physical rows w, w + ways, ...; its row stride is ways * ld."""
+    assert tensor.dim() == 2 and tensor.stride(1) == 1 and tensor.shape[0] % ways == 0
+    ld = tensor.stride(0)
+    return [(w * ld, (tensor.shape[0] // ways, tensor.shape[1], ways * ld)) for w in range(ways)]
+
+
 def views_of_planes(tensor):
     """The E matrix planes of an [E, M, N] tensor: E independent M x N matrices, never one E x MN matrix."""
     assert tensor.dim() == 3 and tensor.stride(2) == 1
@@ -270,6 +291,12 @@ class Layout:
             self.close()
         except Exception:
             pass
+
+
+def _coeffs(coeffs):
+    """Host coefficient table: one row, or one row per matrix (2-D input), flattened row-major."""
+    flat = np.asarray(coeffs, dtype=np.float32).reshape(-1)
+    return (C.c_float * flat.size)(*flat.tolist())
 
 
 class Context:
@@ -337,12 +364,12 @@ class Context:
 
     # -- compute
     def muon_step_batched(self, params, grads, momenta, shapes, lr, mu, wd, ns_steps, coeffs, stream=None) -> None:
-        co = (C.c_float * len(coeffs))(*[float(c) for c in coeffs])
+        co = _coeffs(coeffs)
         _check(lib.muon_step_batched(self.handle, _ptrs(params), _ptrs(grads), _ptrs(momenta), _shapes(shapes),
                                      len(shapes), lr, mu, wd, ns_steps, co, _stream(stream)), "muon_step_batched")
 
     def muon_step_batched_out(self, params, grads, momenta, updates, shapes, lr, mu, wd, ns_steps, coeffs, stream=None) -> None:
-        co = (C.c_float * len(coeffs))(*[float(c) for c in coeffs])
+        co = _coeffs(coeffs)
         _check(lib.muon_step_batched_out(self.handle, _ptrs(params), _ptrs(grads), _ptrs(momenta),
                                          None if updates is None else _ptrs(updates), _shapes(shapes), len(shapes),
                                          lr, mu, wd, ns_steps, co, _stream(stream)), "muon_step_batched_out")
@@ -350,7 +377,7 @@ class Context:
     def muon_step_batched_views(self, params, grads, momenta, updates, views, lr, mu, wd, ns_steps, coeffs, stream=None) -> None:
         """params/grads/momenta/updates: lists of device addresses (ints) of element (0,0) of each view;
         views: list of (rows, cols, ld)."""
-        co = (C.c_float * len(coeffs))(*[float(c) for c in coeffs])
+        co = _coeffs(coeffs)
         va = (View * max(1, len(views)))()
         for i, (r, c, ld) in enumerate(views):
             va[i].rows, va[i].cols, va[i].ld = int(r), int(c), int(ld)
@@ -360,7 +387,7 @@ class Context:
 
     def muon_step_flat(self, layout: Layout, flat_params, flat_grads, flat_momenta, flat_updates, lr, mu, wd, ns_steps, coeffs,
                        stream=None) -> None:
-        co = (C.c_float * len(coeffs))(*[float(c) for c in coeffs])
+        co = _coeffs(coeffs)
         _check(lib.muon_step_flat(self.handle, layout.handle, flat_params.data_ptr(), flat_grads.data_ptr(),
                                   flat_momenta.data_ptr(), None if flat_updates is None else flat_updates.data_ptr(),
                                   lr, mu, wd, ns_steps, co, _stream(stream)), "muon_step_flat")
@@ -368,13 +395,13 @@ class Context:
     def muon_step_flat_host(self, host_flat_grads, host_flat_updates, layout: Layout, params, grads, momenta,
                             updates, lr, mu, wd, ns_steps, coeffs, stream=None) -> None:
         """host_flat_*: CPU tensors (pinned for asynchronous copies)."""
-        co = (C.c_float * len(coeffs))(*[float(c) for c in coeffs])
+        co = _coeffs(coeffs)
         _check(lib.muon_step_flat_host(self.handle, host_flat_grads.data_ptr(), host_flat_updates.data_ptr(),
                                        layout.handle, _ptrs(params), _ptrs(grads), _ptrs(momenta),
                                        _ptrs(updates), lr, mu, wd, ns_steps, co, _stream(stream)), "muon_step_flat_host")
 
     def muon_orthogonalize_batched(self, inputs, outputs, shapes, ns_steps, coeffs, flags=0, stream=None) -> None:
-        co = (C.c_float * len(coeffs))(*[float(c) for c in coeffs])
+        co = _coeffs(coeffs)
         _check(lib.muon_orthogonalize_batched(self.handle, _ptrs(inputs), _ptrs(outputs), _shapes(shapes), len(shapes),
                                               ns_steps, co, flags, _stream(stream)), "muon_orthogonalize_batched")
 

@@ -28,6 +28,7 @@ bool valid_options(const muon_options_t& o) {
   if (o.engine != MUON_ENGINE_TENSOR && o.engine != MUON_ENGINE_CUDA_CORE && o.engine != MUON_ENGINE_TENSOR_1CTA) return false;
   if (o.nesterov != 0 && o.nesterov != 1) return false;
   if (o.coeffs_per_step != 0 && o.coeffs_per_step != 1) return false;
+  if (o.coeffs_per_matrix != 0 && o.coeffs_per_matrix != 1) return false;
   if (!(o.eps >= 0.f) || !std::isfinite(o.eps)) return false;
   if (o.chunk_elems < 0) return false;
   return true;
@@ -139,8 +140,10 @@ struct ChunkRun {
   int32_t normalize;
   float lr, mu, wd;
   int32_t ns_steps;
-  const float* coeffs;
+  const float* coeffs;  // host: one row of `nco` floats, or one row per matrix of the call (opt.coeffs_per_matrix)
 };
+
+int coeff_row_len(const muon_ctx* ctx, int ns_steps) { return ctx->opt.coeffs_per_step ? 3 * ns_steps : 3; }
 
 // Everything the kernels of one launch set need besides the plan.
 struct SetRun {
@@ -150,6 +153,8 @@ struct SetRun {
   const MatDesc* d_descs;       // device, first record of the SET
   const RowSeg* d_segs;         // flat-shard mode, else null
   int32_t flat_vec;
+  const float* d_coef;          // device, per-matrix coefficient rows, first row of the SET (null: one row for all)
+  int32_t coef_stride;
 };
 
 int fill_elem_chunks(const SetRun& sr, bool want_wide, int x_index, ElemChunk* out) {
@@ -176,7 +181,7 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
   const float* rnorm = reinterpret_cast<const float*>(base + sr.set->off_rnorm);
   int n;
   if (sr.tables) {
-    auto launch = [&](const tc::TcTable& tab, float alpha, float beta, int gamma_mode) {
+    auto launch = [&](const tc::TcTable& tab, float alpha, float beta, int gamma_mode, int coef_a, int coef_b, int coef_off) {
       tc::TcLaunch L;
       L.persist = nullptr;
       for (int i = 0; i < tab.nprob; ++i) {
@@ -186,8 +191,10 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
       L.nprob = tab.nprob;
       L.total_tiles = tab.total_tiles;
       L.alpha = alpha; L.beta = beta; L.gamma_mode = gamma_mode;
-      L.coef_a = L.coef_b = -1;
-      L.coef_stride = 0;
+      L.coef_table = sr.d_coef;
+      L.coef_a = coef_a; L.coef_b = coef_b; L.coef_off = coef_off;
+      L.coef_stride = sr.coef_stride;
+      L.coef_per_step = ctx->opt.coeffs_per_step;
       L.status = ctx->d_status;
       return launch_tc_grouped(ctx->device, L, st);
     };
@@ -201,6 +208,9 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
         tc::TcLaunch L;
         std::memset(static_cast<void*>(&L), 0, sizeof(L));
         L.coef_a = L.coef_b = -1;
+        L.coef_table = sr.d_coef;
+        L.coef_stride = sr.coef_stride;
+        L.coef_per_step = ctx->opt.coeffs_per_step;
         L.status = ctx->d_status;
         L.persist = sr.tables->persist;
         L.ns_steps = r.ns_steps;
@@ -218,13 +228,14 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
       }
     }
     for (int k = 0; k < r.ns_steps; ++k) {
-      const float* co = r.coeffs + (ctx->opt.coeffs_per_step ? 3 * k : 0);
+      const int off = ctx->opt.coeffs_per_step ? 3 * k : 0;
+      const float* co = r.coeffs + off;      // with per-matrix rows these scalars are replaced row by row on the device
       const int cur = k & 1;
-      if ((n = launch(sr.tables->g1[cur], 1.f, 0.f, k == 0 ? 2 : 0)) < 0) return n;     // A = gamma X X^T
+      if ((n = launch(sr.tables->g1[cur], 1.f, 0.f, k == 0 ? 2 : 0, -1, -1, off)) < 0) return n;     // A = gamma X X^T
       *launches += n;
-      if ((n = launch(sr.tables->g2, co[2], co[1], 0)) < 0) return n;                   // B = b A + c A A^T (A symmetric)
+      if ((n = launch(sr.tables->g2, co[2], co[1], 0, 2, 1, off)) < 0) return n;                   // B = b A + c A A^T (A symmetric)
       *launches += n;
-      if ((n = launch(sr.tables->g3[cur], 1.f, co[0], k == 0 ? 1 : 0)) < 0) return n;   // X' = gamma (a X + B X)
+      if ((n = launch(sr.tables->g3[cur], 1.f, co[0], k == 0 ? 1 : 0, -1, 0, off)) < 0) return n;   // X' = gamma (a X + B X)
       *launches += n;
     }
     return MUON_OK;
@@ -237,10 +248,14 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
     const float* rn = rnorm + (ch.desc_begin - sr.set->desc_begin);
     const int64_t sx = int64_t(ch.s) * ch.ldx, sa_ = int64_t(ch.s) * ch.lda;
     for (int k = 0; k < r.ns_steps; ++k) {
-      const float* co = r.coeffs + (ctx->opt.coeffs_per_step ? 3 * k : 0);
+      const int off = ctx->opt.coeffs_per_step ? 3 * k : 0;
+      const float* co = r.coeffs + off;
       void* cur = xs[k & 1];
       void* nxt = xs[(k & 1) ^ 1];
       GemmArgs g{};
+      g.coef = sr.d_coef ? sr.d_coef + size_t(ch.desc_begin - sr.set->desc_begin) * size_t(sr.coef_stride) + off : nullptr;
+      g.coef_stride = sr.coef_stride;
+      g.coef_a = g.coef_b = -1;
       g.p = cur; g.q = cur; g.d = nullptr; g.c = A;
       g.m = ch.s; g.n = ch.s; g.kdim = ch.l;
       g.ldp = ch.ldx; g.ldq = ch.ldx; g.ldc = ch.lda;
@@ -253,6 +268,7 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
       g.kdim = ch.s; g.ldp = ch.lda; g.ldq = ch.lda;
       g.stride_p = sa_; g.stride_q = sa_;
       g.gamma_mode = 0; g.alpha = co[2]; g.beta = co[1];
+      g.coef_a = 2; g.coef_b = 1;
       if ((n = run_gemm(ctx, g, st)) < 0) return n;
       *launches += n;
       g.p = B; g.q = cur; g.d = cur; g.c = nxt;
@@ -260,6 +276,7 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
       g.ldp = ch.lda; g.ldq = ch.ldx; g.ldc = ch.ldx;
       g.stride_p = sa_; g.stride_q = sx; g.stride_c = sx;
       g.gamma_mode = (k == 0) ? 1 : 0; g.alpha = 1.f; g.beta = co[0]; g.nn = 1; g.symmetric = 0;
+      g.coef_a = -1; g.coef_b = 0;
       if ((n = run_gemm(ctx, g, st)) < 0) return n;
       *launches += n;
     }
@@ -400,8 +417,23 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
   void* d_descs = nullptr;
   status = upload(ctx, descs.data(), descs.size() * sizeof(MatDesc), st, &d_descs);
   if (status != MUON_OK) return status;
+  const float* d_coef = nullptr;
+  const int nco = coeff_row_len(ctx, r.ns_steps);
+  if (ctx->opt.coeffs_per_matrix) {                    // rows travel in the order of the matrix records
+    std::vector<float> rows(size_t(plan->live) * size_t(nco));
+    for (const Chunk& ch : plan->chunks)
+      for (int32_t j = 0; j < ch.count; ++j)
+        std::memcpy(&rows[size_t(ch.desc_begin + j) * size_t(nco)], r.coeffs + size_t(ch.mats[size_t(j)]) * size_t(nco),
+                    size_t(nco) * sizeof(float));
+    void* d = nullptr;
+    status = upload(ctx, rows.data(), rows.size() * sizeof(float), st, &d);
+    if (status != MUON_OK) return status;
+    d_coef = static_cast<const float*>(d);
+  }
   auto set_run = [&](size_t k) {
     SetRun sr;
+    sr.d_coef = d_coef ? d_coef + size_t(plan->sets[k].desc_begin) * size_t(nco) : nullptr;
+    sr.coef_stride = nco;
     sr.chunks = &plan->chunks;
     sr.set = &plan->sets[k];
     sr.tables = grouped ? &(*plan->set_tables)[k] : nullptr;
@@ -485,6 +517,8 @@ int muon_default_options(muon_options_t* opt) {
   opt->ns_precision = MUON_NS_BF16;
   opt->nesterov = 1;
   opt->coeffs_per_step = 0;
+  opt->coeffs_per_matrix = 0;
+  opt->reserved = 0;
   opt->eps = 1e-7f;
   opt->engine = MUON_ENGINE_TENSOR;
   opt->chunk_elems = int64_t(1) << 29;
@@ -820,8 +854,8 @@ static int check_common(muon_ctx_t* ctx, const muon_shape_t* shapes, int32_t cou
   if (!ctx || count < 0) return MUON_ERR_INVALID_ARG;
   if (count > 0 && !shapes) return MUON_ERR_INVALID_ARG;
   if (ns_steps < 1 || ns_steps > 64 || !coeffs) return MUON_ERR_INVALID_ARG;
-  const int nco = ctx->opt.coeffs_per_step ? 3 * ns_steps : 3;
-  for (int i = 0; i < nco; ++i)
+  const int64_t nco = int64_t(ctx->opt.coeffs_per_step ? 3 * ns_steps : 3) * (ctx->opt.coeffs_per_matrix ? count : 1);
+  for (int64_t i = 0; i < nco; ++i)
     if (!std::isfinite(coeffs[i])) return MUON_ERR_INVALID_ARG;
   if (!DeviceGuardCheck::ok(ctx)) return MUON_ERR_CUDA;
   return MUON_OK;
@@ -837,6 +871,15 @@ int muon_step_batched_out(muon_ctx_t* ctx, void* const* params, const void* cons
   if (!std::isfinite(lr) || !std::isfinite(mu) || !std::isfinite(wd)) return MUON_ERR_INVALID_ARG;
   ChunkRun r{1, 1, lr, mu, wd, ns_steps, coeffs};
   return run_batched(ctx, params, grads, momenta, updates, shapes, count, r, static_cast<cudaStream_t>(stream));
+}
+
+int muon_views_overlap(const void* const* bases, const muon_view_t* views, int32_t count, int32_t elem_size, int32_t* overlap) {
+  if (count < 0 || (count > 0 && (!bases || !views)) || elem_size <= 0 || !overlap) return MUON_ERR_INVALID_ARG;
+  for (int32_t i = 0; i < count; ++i)
+    if (views[i].rows < 0 || views[i].cols < 0 || (views[i].rows > 0 && views[i].cols > 0 && views[i].ld < views[i].cols))
+      return MUON_ERR_INVALID_ARG;
+  *overlap = views_overlap_host(bases, views, count, elem_size);
+  return MUON_OK;
 }
 
 int muon_step_batched_views(muon_ctx_t* ctx, void* const* params, const void* const* grads, void* const* momenta,
@@ -855,6 +898,12 @@ int muon_step_batched_views(muon_ctx_t* ctx, void* const* params, const void* co
   if (count == 0) return MUON_OK;
   if (!params || !grads || !momenta) return MUON_ERR_INVALID_ARG;
   if (!std::isfinite(lr) || !std::isfinite(mu) || !std::isfinite(wd)) return MUON_ERR_INVALID_ARG;
+  for (int32_t i = 0; i < count; ++i)
+    if (views[i].rows > 0 && views[i].cols > 0 && views[i].ld < views[i].cols) return MUON_ERR_INVALID_ARG;
+  // everything the call writes must be written once: two views that share an element would race
+  if (views_overlap_host(params, views, count, 4) || views_overlap_host(momenta, views, count, 4) ||
+      (updates && views_overlap_host(updates, views, count, ctx->opt.ns_precision == MUON_NS_BF16 ? 2 : 4)))
+    return MUON_ERR_INVALID_ARG;
   ChunkRun r{1, 1, lr, mu, wd, ns_steps, coeffs};
   return run_batched(ctx, params, grads, momenta, updates, shapes.data(), count, r, static_cast<cudaStream_t>(stream), nullptr,
                      lds.data());
@@ -964,8 +1013,9 @@ int muon_ns_product(muon_ctx_t* ctx, const void* p, const void* q, const void* d
     L.nprob = 1;
     L.total_tiles = tab.total_tiles;
     L.alpha = g.alpha; L.beta = g.beta; L.gamma_mode = g.gamma_mode;
+    L.coef_table = nullptr;
     L.coef_a = L.coef_b = -1;
-    L.coef_stride = 0;
+    L.coef_off = L.coef_stride = L.coef_per_step = 0;
     L.status = ctx->d_status;
     Span sp(ctx, MUON_PHASE_NS, st);
     nl = launch_tc_grouped(ctx->device, L, st);
@@ -1193,5 +1243,7 @@ extern "C" int muon_orthogonalize_static(const void* in, void* out, int32_t rows
   sr.d_descs = d_desc;
   sr.d_segs = nullptr;
   sr.flat_vec = 8;
+  sr.d_coef = nullptr;
+  sr.coef_stride = 0;
   return run_set(&ctx, sr, r, st);
 }

@@ -83,6 +83,8 @@ struct TilePatHost {
 };
 std::vector<TilePatHost> symmetric_tile_pattern(int nb);
 int validate_layout_host(const muon_layout_desc_t* d);
+// 1 when two of the strided views (element (0,0) at bases[i]) share an element, else 0.
+int views_overlap_host(const void* const* bases, const muon_view_t* views, int32_t count, int32_t elem_size);
 int owner_plan_host(const muon_shape_t* shapes, int32_t count, int32_t ranks, int64_t batch_elems, int32_t* owner_of,
                     int32_t* batch_of, int32_t* num_batches);
 
@@ -220,6 +222,10 @@ struct GemmArgs {
   float alpha, beta;
   int32_t nn;
   int32_t symmetric;   // op is P P^T with symmetric result (kernels may exploit it)
+  // per-matrix coefficients: matrix k takes alpha = coef[k * coef_stride + coef_a] (beta likewise with coef_b) when
+  // coef is set and the index is >= 0
+  const float* coef;   // device or null
+  int32_t coef_a, coef_b, coef_stride;
 };
 int launch_gemm_simt(const GemmArgs& a, int ns_precision, cudaStream_t st);
 int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st);   // tcgen05 engine, single-CTA kernel (bf16 only)

@@ -83,6 +83,12 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs a, int tiles_m,
     const float r = a.rnorm[mat];
     gamma = a.gamma_mode == 1 ? r : r * r;
   }
+  float alpha = a.alpha, beta = a.beta;
+  if (a.coef) {
+    const float* co = a.coef + size_t(mat) * size_t(a.coef_stride);
+    if (a.coef_a >= 0) alpha = co[a.coef_a];
+    if (a.coef_b >= 0) beta = co[a.coef_b];
+  }
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int r = m0 + ty * 4 + i;
@@ -92,8 +98,8 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs a, int tiles_m,
       const int c = n0 + tx * 4 + j;
       if (c >= a.n) continue;
       const size_t off = size_t(r) * a.ldc + c;
-      float v = a.alpha * acc[i][j];
-      if (D) v += a.beta * ldf<T>(D + off);
+      float v = alpha * acc[i][j];
+      if (D) v += beta * ldf<T>(D + off);
       C[off] = cvt<T>(gamma * v);
     }
   }

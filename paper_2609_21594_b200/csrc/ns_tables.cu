@@ -114,7 +114,7 @@ int build_set_image(void* encode_fn, const void* ws, const std::vector<Chunk>& c
       TcProbInfo p;
       std::memset(&p, 0, sizeof(p));
       p.rnorm = rnorm_base + (c.desc_begin - set.desc_begin);
-      p.coef = nullptr;
+      p.mat_begin = c.desc_begin - set.desc_begin;
       p.batch = c.count;
       const auto& pat = patterns[(c.s + 127) / 128];
       if (kind < 2) {            // A = gamma X X^T
@@ -213,7 +213,7 @@ int build_product_image(void* encode_fn, const GemmArgs& g, const void* dev_base
   p.d = static_cast<const __nv_bfloat16*>(g.d);
   p.c = static_cast<__nv_bfloat16*>(g.c);
   p.rnorm = g.rnorm;
-  p.coef = nullptr;
+  p.mat_begin = 0;
   p.stride_c = g.stride_c;
   p.m = g.m; p.n = g.n; p.kdim = g.kdim; p.ldc = g.ldc;
   p.batch = g.batch;

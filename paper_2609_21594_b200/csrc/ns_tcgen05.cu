@@ -203,6 +203,11 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
       e.cblk1 = tl.n0 + 128 < a.n ? tl.n0 / 128 + 1 : -1;
       e.mirror0 = e.mirror1 = a.symmetric && tl.n0 >= tl.m0 + BM;       // tile lies strictly above the diagonal
       e.alpha = a.alpha; e.beta = a.beta; e.gamma = 1.f;
+      if (a.coef) {
+        const float* co = a.coef + size_t(tl.mat) * size_t(a.coef_stride);
+        if (a.coef_a >= 0) e.alpha = co[a.coef_a];
+        if (a.coef_b >= 0) e.beta = co[a.coef_b];
+      }
       if (a.gamma_mode) {
         const float r = a.rnorm[tl.mat];
         e.gamma = a.gamma_mode == 1 ? r : r * r;
@@ -327,6 +332,7 @@ int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st) {
   t.rnorm = a.rnorm;
   t.gamma_mode = a.gamma_mode;
   t.alpha = a.alpha; t.beta = a.beta;
+  t.coef = a.coef; t.coef_a = a.coef_a; t.coef_b = a.coef_b; t.coef_stride = a.coef_stride;
   t.status = ctx->d_status;
   const int64_t tiles = int64_t(t.tiles_per_mat) * t.batch;
   const unsigned grid = unsigned(tiles < g_num_sms[ctx->device] ? tiles : g_num_sms[ctx->device]);

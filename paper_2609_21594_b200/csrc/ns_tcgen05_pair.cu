@@ -110,6 +110,7 @@ struct PhaseView {
   int nprob, total_tiles;
   float alpha, beta;
   int gamma_mode;
+  int coef_a, coef_b, coef_off;   // per-matrix coefficient rows: see TcLaunch
 };
 
 // Product `ph` of the launch.  A one-product launch carries its tables by value; a whole-iteration launch reads
@@ -120,6 +121,7 @@ __device__ __forceinline__ PhaseView phase_view(const TcLaunch& L, int ph) {
   if (!L.persist) {
     v.maps = L.maps; v.info = L.info; v.nprob = L.nprob; v.total_tiles = L.total_tiles;
     v.alpha = L.alpha; v.beta = L.beta; v.gamma_mode = L.gamma_mode;
+    v.coef_a = L.coef_a; v.coef_b = L.coef_b; v.coef_off = L.coef_off;
     return v;
   }
   const int k = ph / 3, j = ph - 3 * k, cur = k & 1;
@@ -131,6 +133,9 @@ __device__ __forceinline__ PhaseView phase_view(const TcLaunch& L, int ph) {
   v.alpha = j == 1 ? L.coef[k][2] : 1.f;
   v.beta = j == 0 ? 0.f : (j == 1 ? L.coef[k][1] : L.coef[k][0]);
   v.gamma_mode = k == 0 ? (j == 0 ? 2 : (j == 2 ? 1 : 0)) : 0;
+  v.coef_a = j == 1 ? 2 : -1;
+  v.coef_b = j == 0 ? -1 : (j == 1 ? 1 : 0);
+  v.coef_off = L.coef_per_step ? 3 * k : 0;
   return v;
 }
 
@@ -186,10 +191,10 @@ __device__ __forceinline__ EpiTile make_epi(const Tile& tl, int rank, const Phas
       const float r = p.rnorm[tl.mat];
       e.gamma = V.gamma_mode == 1 ? r : r * r;
     }
-    if (p.coef) {
-      const float* co = p.coef + size_t(tl.mat) * L.coef_stride;
-      if (L.coef_a >= 0) e.alpha = co[L.coef_a];
-      if (L.coef_b >= 0) e.beta = co[L.coef_b];
+    if (L.coef_table) {
+      const float* co = L.coef_table + size_t(p.mat_begin + tl.mat) * size_t(L.coef_stride) + V.coef_off;
+      if (V.coef_a >= 0) e.alpha = __ldg(co + V.coef_a);
+      if (V.coef_b >= 0) e.beta = __ldg(co + V.coef_b);
     }
   }
   return e;
@@ -247,7 +252,9 @@ struct LoadArgs {
   bool leader_cta, narrow;
 };
 
-template <bool A_MN, bool B_MN>
+// ALIAS: a diagonal tile of a symmetric product (column blocks == row blocks): each CTA's half of Q is its own P tile,
+// so Q is not loaded at all and the MMA reads both operands from the P buffer.
+template <bool A_MN, bool B_MN, bool ALIAS>
 __device__ __forceinline__ bool produce_range(LoopCtx& c, const LoadArgs& a, int kb_begin, int kb_end) {
   for (int kb = kb_begin; kb < kb_end; ++kb, c.advance()) {
     const int s = int(c.s);
@@ -262,6 +269,7 @@ __device__ __forceinline__ bool produce_range(LoopCtx& c, const LoadArgs& a, int
       tma_load_3d_pair(sa, &a.mp->ph, fb, a.prow, k0, a.mat);
       tma_load_3d_pair(sa + 64 * BK * 2, &a.mp->ph, fb, a.prow + 64, k0, a.mat);
     }
+    if (ALIAS) continue;
     if (!B_MN) {                                   // 128 rows of Q, or the 64 a 128-wide tile needs
       tma_load_3d_pair(sb, a.narrow ? &a.mp->qh : &a.mp->q, fb, k0, a.qcol, a.mat);
     } else {                                       // 64 k-rows x 64 columns, twice for a 256-wide tile
@@ -275,7 +283,8 @@ __device__ __forceinline__ bool produce_range(LoopCtx& c, const LoadArgs& a, int
 // A shared-memory descriptor is a constant high part (layout, strides) plus the start address in 16-byte units.
 // K-major: 16 k = 32 bytes along a 128-byte row; MN-major: 16 k-rows of 128 bytes each.
 template <bool A_MN, bool B_MN>
-__device__ __forceinline__ bool issue_range(LoopCtx& c, uint32_t d_tmem, uint32_t idesc_base, int kb_begin, int kb_end) {
+__device__ __forceinline__ bool issue_range(LoopCtx& c, uint32_t d_tmem, uint32_t idesc_base, uint32_t b_off, int kb_begin,
+                                            int kb_end) {
   constexpr uint32_t idesc_major = (A_MN ? 1u << 15 : 0u) | (B_MN ? 1u << 16 : 0u);
   constexpr uint64_t a_hi = A_MN ? DESC_HI_MN : DESC_HI_K, b_hi = B_MN ? DESC_HI_MN : DESC_HI_K;
   constexpr uint32_t a_step = A_MN ? (UK * 128) >> 4 : (UK * 2) >> 4, b_step = B_MN ? (UK * 128) >> 4 : (UK * 2) >> 4;
@@ -284,7 +293,7 @@ __device__ __forceinline__ bool issue_range(LoopCtx& c, uint32_t d_tmem, uint32_
     const int s = int(c.s);
     if (!mbar_wait(full_bar_of(c, s), c.ph, c.abort_flag)) return false;
     tc_fence_after();
-    const uint32_t a0 = (c.base + uint32_t(s) * STAGE_BYTES) >> 4, b0 = a0 + (A_BYTES >> 4);
+    const uint32_t a0 = (c.base + uint32_t(s) * STAGE_BYTES) >> 4, b0 = a0 + b_off;
 #pragma unroll
     for (int k = 0; k < BK / UK; ++k)
       tc_mma_pair(d_tmem, a_hi | uint64_t(a0 + uint32_t(k) * a_step), b_hi | uint64_t(b0 + uint32_t(k) * b_step), idesc,
@@ -384,14 +393,16 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
           const int qcol = narrow ? tl.cc * 128 + int(rank) * 64 : (rank ? tl.cd : tl.cc) * 128;
           LoadArgs la;
           la.mp = mp; la.mat = tl.mat; la.prow = prow; la.qcol = qcol;
-          la.stage_tx = narrow ? 2 * (A_BYTES + B_BYTES / 2) : 2 * STAGE_BYTES;
+          const bool alias = p.symmetric != 0 && !nn && !narrow && tl.cc == tl.ra && tl.cd == tl.rb;
+          la.stage_tx = alias ? 2 * A_BYTES : (narrow ? 2 * (A_BYTES + B_BYTES / 2) : 2 * STAGE_BYTES);
           la.leader_cta = leader_cta; la.narrow = narrow;
           // half-stored symmetric operands: k-blocks left of the tile's own block pair are read transposed
           int p_flip_kb = p.p_half ? (tl.ra >> 1) * 4 : 0;            // k-blocks [0, p_flip_kb) of P come MN-major
           int q_flip_kb = nn ? num_kb : (p.q_half ? (tl.cc >> 1) * 4 : 0);
           p_flip_kb = p_flip_kb < num_kb ? p_flip_kb : num_kb;
           q_flip_kb = q_flip_kb < num_kb ? q_flip_kb : num_kb;
-#define MUON_PRODUCE(AM, BM_, B0, B1) produce_range<AM, BM_>(lc, la, B0, B1)
+#define MUON_PRODUCE(AM, BM_, B0, B1) \
+  (alias ? produce_range<AM, BM_, true>(lc, la, B0, B1) : produce_range<AM, BM_, false>(lc, la, B0, B1))
           MUON_FOR_K_PIECES(MUON_PRODUCE)
 #undef MUON_PRODUCE
         }
@@ -427,11 +438,14 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
             int q_flip_kb = nn ? num_kb : (p.q_half ? (tl.cc >> 1) * 4 : 0);
             p_flip_kb = p_flip_kb < num_kb ? p_flip_kb : num_kb;
             q_flip_kb = q_flip_kb < num_kb ? q_flip_kb : num_kb;
+            // diagonal tile of a symmetric product: Q was not loaded, both operands come from the P buffer
+            const bool alias = p.symmetric != 0 && !nn && tl.cd >= 0 && tl.cc == tl.ra && tl.cd == tl.rb;
+            const uint32_t b_off = alias ? 0u : uint32_t(A_BYTES >> 4);
             const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
             if (!mbar_wait(tempty_bar(int(acc)), aph ^ 1u, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + acc * 256u;
-#define MUON_ISSUE(AM, BM_, B0, B1) issue_range<AM, BM_>(lc, d_tmem, idesc_base, B0, B1)
+#define MUON_ISSUE(AM, BM_, B0, B1) issue_range<AM, BM_>(lc, d_tmem, idesc_base, b_off, B0, B1)
             MUON_FOR_K_PIECES(MUON_ISSUE)
 #undef MUON_ISSUE
             if (ok) tc_commit_pair(tfull_bar(int(acc)));

@@ -260,4 +260,46 @@ int validate_layout_host(const muon_layout_desc_t* d) {
   return MUON_OK;
 }
 
+// Do two strided views written by one call share an element?  View i covers, for every row r < rows, the bytes
+// [base_i + r * ld * es, + cols * es).  Candidates are found by sweeping the views' bounding intervals in address order;
+// a candidate pair is settled row by row (the rows of one view against the at most two rows of the other it can meet).
+int views_overlap_host(const void* const* bases, const muon_view_t* views, int32_t count, int32_t elem_size) {
+  struct Box {
+    uintptr_t lo, hi;   // bounding interval [lo, hi)
+    int32_t i;
+  };
+  std::vector<Box> boxes;
+  boxes.reserve(size_t(count));
+  const uintptr_t es = uintptr_t(elem_size);
+  for (int32_t i = 0; i < count; ++i) {
+    const muon_view_t& v = views[i];
+    if (v.rows <= 0 || v.cols <= 0 || !bases[i]) continue;
+    const uintptr_t lo = reinterpret_cast<uintptr_t>(bases[i]);
+    boxes.push_back({lo, lo + (uintptr_t(v.rows - 1) * uintptr_t(v.ld) + uintptr_t(v.cols)) * es, i});
+  }
+  std::sort(boxes.begin(), boxes.end(), [](const Box& a, const Box& b) { return a.lo < b.lo || (a.lo == b.lo && a.i < b.i); });
+  auto rows_meet = [&](const Box& a, const Box& b) {
+    const muon_view_t& va = views[a.i];
+    const muon_view_t& vb = views[b.i];
+    const uintptr_t pa = uintptr_t(va.ld) * es, pb = uintptr_t(vb.ld) * es;
+    const uintptr_t wa = uintptr_t(va.cols) * es, wb = uintptr_t(vb.cols) * es;
+    for (int32_t r = 0; r < va.rows; ++r) {
+      const uintptr_t lo = a.lo + uintptr_t(r) * pa, hi = lo + wa;
+      if (hi <= b.lo || lo >= b.hi) continue;
+      // rows of b that may meet [lo, hi): the one that starts last at or before lo, and every row starting inside
+      int64_t j0 = lo > b.lo ? int64_t((lo - b.lo) / pb) : 0;
+      for (int64_t j = j0; j < vb.rows; ++j) {
+        const uintptr_t blo = b.lo + uintptr_t(j) * pb;
+        if (blo >= hi) break;
+        if (blo + wb > lo) return true;
+      }
+    }
+    return false;
+  };
+  for (size_t x = 0; x < boxes.size(); ++x)
+    for (size_t y = x + 1; y < boxes.size() && boxes[y].lo < boxes[x].hi; ++y)
+      if (rows_meet(boxes[x], boxes[y])) return 1;
+  return 0;
+}
+
 }  // namespace muon

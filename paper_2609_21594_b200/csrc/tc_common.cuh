@@ -20,6 +20,8 @@ struct TcArgs {
   const float* rnorm;
   int32_t gamma_mode;
   float alpha, beta;
+  const float* coef;        // per-matrix coefficient rows (null: alpha, beta above for every matrix)
+  int32_t coef_a, coef_b, coef_stride;
   int32_t* status;
 };
 

@@ -32,7 +32,7 @@ struct TcProbInfo {
   const __nv_bfloat16* d;    // aux matrix (may be null)
   __nv_bfloat16* c;
   const float* rnorm;        // per matrix (gamma modes 1, 2)
-  const float* coef;         // per matrix coefficient rows [batch][coef_stride] or null
+  int64_t mat_begin;         // index of the problem's first matrix inside the launch set (row of per-matrix tables)
   const TilePat* pattern;    // explicit tile list per matrix (symmetric products); null: dense 2 x 2 block grid
   int64_t stride_c;
   int32_t m, n, kdim, ldc;
@@ -66,8 +66,11 @@ struct TcLaunch {
   int32_t nprob, total_tiles;
   float alpha, beta;
   int32_t gamma_mode;        // 0: 1, 1: r, 2: r*r
-  int32_t coef_a, coef_b;    // index into a matrix's coefficient row that replaces alpha / beta (-1: keep the scalar)
-  int32_t coef_stride;
+  // Per-matrix coefficients: row (mat_begin + matrix) of coef_table, coef_stride floats per row, replaces the scalars:
+  // alpha = row[coef_off + coef_a], beta = row[coef_off + coef_b] (an index < 0 keeps the scalar).  A whole-iteration
+  // launch derives the indices from the product it is in (coef_off = 3 * step when coef_per_step).
+  const float* coef_table;   // device, first row of the launch set; null: scalars only
+  int32_t coef_a, coef_b, coef_off, coef_stride, coef_per_step;
   int32_t* status;
   // Whole-iteration mode (persist != null): the launch walks 3 * ns_steps products, a grid-wide barrier between
   // consecutive ones, and takes tables from device memory instead of maps / info above.

@@ -103,3 +103,35 @@ def test_llama3_8b_set_in_8_flat_shards():
     # the last matrix (down, 4096 x 14336)
     sample = [0, 2, 7 * 1 + 4, len(shapes) - 1]
     _run_config("llama8b", shapes, True, sample, wl.layout_per_param)
+
+
+def test_llama3_8b_flat_concat_round_trip_bit_exact():
+    """The layout generator whose shard cuts fall inside matrices (the flat concatenation cut at aligned points), at the
+    benchmark's full size: scatter then gather must reproduce every matrix bit for bit, every segment must sit where the
+    table says, and the padding of the flat buffer must never be written."""
+    from paper_2609_21594_b200 import binding as mb
+
+    dev = torch.device("cuda", 0)
+    shapes = wl.shapes_llama8b()
+    # 32 equal layers over 8 shards would put every cut on a layer boundary; 7 shards cut inside matrices, mid-row
+    layout = wl.layout_flat_concat(shapes, 7)
+    inside = [sg for sg in layout.segments if sg.elem_begin != 0]
+    assert len(inside) >= 6 and any(sg.elem_begin % shapes[sg.matrix][1] for sg in inside)
+    ctx = mb.Context()
+    L = mb.Layout(ctx, layout, 2)
+    src = [wl.device_draw("llama8b_fc", 0, i, "grad", s, dev, std=1e-3, dtype=torch.bfloat16) for i, s in enumerate(shapes)]
+    flat = torch.full((layout.flat_len,), 0x7B7B, dtype=torch.int16, device=dev).view(torch.bfloat16)
+    ctx.muon_scatter(flat, L, src)
+    back = [torch.full(s, float("nan"), dtype=torch.bfloat16, device=dev) for s in shapes]
+    ctx.muon_materialize(flat, L, back)
+    torch.cuda.synchronize()
+    pad_mask = torch.ones(layout.flat_len, dtype=torch.bool, device=dev)
+    for sg in layout.segments:
+        pad_mask[sg.flat_offset:sg.flat_offset + sg.elem_count] = False
+        a = src[sg.matrix].view(-1)[sg.elem_begin:sg.elem_begin + sg.elem_count].view(torch.int16)
+        assert torch.equal(a, flat[sg.flat_offset:sg.flat_offset + sg.elem_count].view(torch.int16)), sg
+    assert bool((flat.view(torch.int16)[pad_mask] == 0x7B7B).all())
+    for i in range(len(shapes)):
+        assert torch.equal(back[i].view(torch.int16), src[i].view(torch.int16)), i
+    L.close()
+    ctx.close()

@@ -424,6 +424,73 @@ def test_per_step_coefficient_sets_on_the_bf16_engines(engine):
     ctx.close()
 
 
+@pytest.mark.parametrize("engine,precision", [("tensor", "bf16"), ("tensor_1cta", "bf16"), ("cuda_core", "bf16"), ("tensor", "fp32")])
+@pytest.mark.parametrize("per_step", [0, 1])
+def test_per_matrix_coefficient_rows(engine, precision, per_step):
+    """coeffs_per_matrix: every matrix of one call iterates with its own polynomial while sharing the launches of its
+    shape group.  Two coefficient sets are mixed inside one shape group and across groups; each result must match the
+    oracle run with that matrix's row and must be far from the oracle run with the other row."""
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = _ctx(mb, precision, engine, coeffs_per_step=per_step, coeffs_per_matrix=1)
+    set_a = [3.4445, -4.7750, 2.0315]
+    set_b = [1.5, -0.5, 0.0]
+    if per_step:
+        row_a = [4.0, -6.0, 2.5, 3.8, -5.5, 2.2, 3.4445, -4.7750, 2.0315, 2.9, -3.6, 1.6, 2.3, -2.0, 0.7]
+        row_b = [1.5, -0.5, 0.0, 2.0, -1.5, 0.5, 1.5, -0.5, 0.0, 3.0, -3.2, 1.2, 1.5, -0.5, 0.0]
+    else:
+        row_a, row_b = set_a, set_b
+    shapes = [(256, 384), (384, 256), (256, 384), (130, 200), (256, 384), (130, 200)]
+    pick = [0, 1, 1, 0, 0, 1]
+    rows = [row_a if p == 0 else row_b for p in pick]
+    mats = [wl.grad_np("permat", 0, i, s) for i, s in enumerate(shapes)]
+    outs, vals = _ortho(mb, ctx, mats, steps=5, coeffs=rows)
+    mode, tol = ("bf16", TOL_BF16) if precision == "bf16" else ("fp64", TOL_FP32)
+    for i, (o, v) in enumerate(zip(outs, vals)):
+        assert rel(o, orc.newton_schulz(v, 5, rows[i], 1e-7, mode)) <= tol, i
+        other = row_b if pick[i] == 0 else row_a
+        assert rel(o, orc.newton_schulz(v, 5, other, 1e-7, mode)) > 5e-2, i
+    ctx.close()
+
+
+def test_per_matrix_coefficient_rows_one_launch_per_product():
+    """The same on a set large enough for one launch per product (not the whole-iteration launch), through the full step:
+    alternating rows inside one shape group; bit-identical to running each coefficient class in a call of its own."""
+    from paper_2609_21594_b200 import binding as mb
+
+    shapes = [(512, 1024)] * 20 + [(1024, 512)] * 4
+    rows = [[3.4445, -4.7750, 2.0315] if i % 3 else [3.0, -3.2, 1.2] for i in range(len(shapes))]
+    ctx = _ctx(mb, "bf16", "tensor", "bf16", coeffs_per_matrix=1)
+    ctx.ensure_workspace(shapes)
+    gen = torch.Generator(device="cuda").manual_seed(77)
+    Wn = [torch.randn(s, device="cuda", generator=gen) * 0.02 for s in shapes]
+    Gn = [(torch.randn(s, device="cuda", generator=gen) * 1e-3).to(torch.bfloat16) for s in shapes]
+    W, M = [w.clone() for w in Wn], [torch.zeros_like(w) for w in Wn]
+    O = [torch.empty(s, dtype=torch.bfloat16, device="cuda") for s in shapes]
+    n0 = ctx.muon_launch_count()
+    ctx.muon_step_batched_out(W, Gn, M, O, shapes, 0.02, 0.95, 0.01, 5, rows)
+    torch.cuda.synchronize()
+    assert ctx.muon_launch_count() - n0 == 15 + 3          # 15 product launches, stage, norm, apply
+    assert ctx.muon_last_device_status() == 0
+    ctx.close()
+    ref = _ctx(mb, "bf16", "tensor", "bf16")
+    ref.ensure_workspace(shapes)
+    for cls in ([3.4445, -4.7750, 2.0315], [3.0, -3.2, 1.2]):
+        idx = [i for i in range(len(shapes)) if rows[i] == cls]
+        W2, M2 = [Wn[i].clone() for i in idx], [torch.zeros_like(Wn[i]) for i in idx]
+        O2 = [torch.empty(shapes[i], dtype=torch.bfloat16, device="cuda") for i in idx]
+        ref.muon_step_batched_out(W2, [Gn[i] for i in idx], M2, O2, [shapes[i] for i in idx], 0.02, 0.95, 0.01, 5, cls)
+        torch.cuda.synchronize()
+        for j, i in enumerate(idx):
+            assert torch.equal(O2[j].view(torch.int16), O[i].view(torch.int16)), i
+            assert torch.equal(W2[j], W[i]), i
+    # one sample against the oracle
+    for i in (0, 1):
+        v = Gn[i].to(torch.float64).cpu().numpy()
+        assert rel(host_f64(O[i]), orc.newton_schulz(v, 5, rows[i], 1e-7, "bf16")) <= TOL_BF16
+    ref.close()
+
+
 def test_plain_momentum_rule_and_eps_option():
     """nesterov = 0 (u = M') and a non-default epsilon are options of the context, not compile-time choices."""
     from paper_2609_21594_b200 import binding as mb

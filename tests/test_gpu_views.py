@@ -92,6 +92,41 @@ def test_ragged_sub_block_leaves_its_surroundings_alone():
     _check(mb, (100, 72), lambda t: [(3 * t.stride(0) + 8, (97, 53, t.stride(0)))], "ragged")
 
 
+def test_row_interleaved_gate_up():
+    """Gate and up projections stored as alternating rows of one [2m, n] tensor: two views with row stride 2n, the second
+    offset by n elements.  Also three-way interleaving with an odd row count per view."""
+    from paper_2609_21594_b200 import binding as mb
+
+    _check(mb, (512, 384), lambda t: mb.views_of_interleaved_rows(t, 2), "gate_up")          # wide logical matrices
+    _check(mb, (1536, 256), lambda t: mb.views_of_interleaved_rows(t, 2), "gate_up_tall")    # tall: transposed path
+    _check(mb, (3 * 131, 200), lambda t: mb.views_of_interleaved_rows(t, 3), "three_way")
+
+
+def test_overlapping_views_are_rejected_before_any_launch():
+    from paper_2609_21594_b200 import binding as mb
+
+    ctx = mb.Context()
+    W, G, M = _physical("overlap", (128, 256))
+    W0, M0 = W.clone(), M.clone()
+    ctx.ensure_workspace([(64, 256), (65, 256)])
+    es = W.element_size()
+    n0 = ctx.muon_launch_count()
+    # rows 0..63 and rows 63..127: one shared row
+    views = [(64, 256, 256), (65, 256, 256)]
+    with pytest.raises(mb.MuonError) as e:
+        ctx.muon_step_batched_views([W.data_ptr(), W.data_ptr() + 63 * 256 * es], [G.data_ptr(), G.data_ptr() + 63 * 256 * 2],
+                                    [M.data_ptr(), M.data_ptr() + 64 * 256 * es], None, views, LR, MU, WD, 5, QUINTIC)
+    assert e.value.code == mb.ERR_INVALID_ARG
+    # the same momentum twice
+    with pytest.raises(mb.MuonError) as e:
+        ctx.muon_step_batched_views([W.data_ptr(), W.data_ptr() + 64 * 256 * es], [G.data_ptr(), G.data_ptr() + 64 * 256 * 2],
+                                    [M.data_ptr(), M.data_ptr()], None, [(64, 256, 256)] * 2, LR, MU, WD, 5, QUINTIC)
+    assert e.value.code == mb.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert ctx.muon_launch_count() == n0 and torch.equal(W, W0) and torch.equal(M, M0)
+    ctx.close()
+
+
 def test_views_reject_bad_strides():
     from paper_2609_21594_b200 import binding as mb
 

@@ -102,3 +102,60 @@ def test_workspace_is_the_largest_launch_set():
     x = (4 * 256 * 256 + 2 * 256 * 1024) * 2
     a = (4 * 256 * 256 + 2 * 256 * 256) * 2
     assert 2 * x + 2 * a <= need <= 2 * x + 2 * a + 16384
+
+
+# ----------------------------------------------------------------------------- strided views: overlap check
+def _brute_overlap(bases, views, es):
+    seen = set()
+    for b, (r, c, ld) in zip(bases, views):
+        if not b or r == 0 or c == 0:
+            continue
+        mine = set()
+        for i in range(r):
+            lo = b + i * ld * es
+            mine.update(range(lo, lo + c * es))
+        if seen & mine:
+            return True
+        seen |= mine
+    return False
+
+
+def test_views_overlap_known_cases():
+    base, es = 1 << 20, 4
+    # fused QKV: three row blocks of one [3*64, 96] tensor
+    qkv = [(64, 96, 96)] * 3
+    assert not mb.muon_views_overlap([base + k * 64 * 96 * es for k in range(3)], qkv, es)
+    assert mb.muon_views_overlap([base, base + 63 * 96 * es, base + 128 * 96 * es], qkv, es)        # second starts one row early
+    # gate/up stored row-interleaved in one [2*m, n] tensor: row stride 2n, second view offset by n
+    m, n = 40, 24
+    assert not mb.muon_views_overlap([base, base + n * es], [(m, n, 2 * n)] * 2, es)
+    assert mb.muon_views_overlap([base, base + (n - 1) * es], [(m, n, 2 * n)] * 2, es)               # offset one element short
+    # side-by-side column factors of one [m, 3n] tensor
+    assert not mb.muon_views_overlap([base + k * n * es for k in range(3)], [(m, n, 3 * n)] * 3, es)
+    assert mb.muon_views_overlap([base, base + n * es], [(m, n + 1, 3 * n), (m, n, 3 * n)], es)
+    # bounding intervals nest but no element is shared: a narrow view in the padding columns of a wide one
+    assert not mb.muon_views_overlap([base, base + 16 * es], [(10, 16, 32), (10, 8, 32)], es)
+    # identical views, empty views, null bases
+    assert mb.muon_views_overlap([base, base], [(3, 5, 5)] * 2, es)
+    assert not mb.muon_views_overlap([base, base], [(3, 5, 5), (0, 5, 5)], es)
+    assert not mb.muon_views_overlap([base, 0], [(3, 5, 5)] * 2, es)
+    with pytest.raises(mb.MuonError):
+        mb.muon_views_overlap([base], [(3, 5, 4)], es)                                                # ld < cols
+
+
+def test_views_overlap_against_brute_force():
+    rng = np.random.default_rng(5)
+    hits = 0
+    for case in range(300):
+        es = int(rng.choice([2, 4]))
+        k = int(rng.integers(2, 6))
+        views, bases = [], []
+        for _ in range(k):
+            r, c = int(rng.integers(0, 7)), int(rng.integers(0, 7))
+            ld = c + int(rng.integers(0, 9))
+            views.append((r, c, max(ld, 1)))
+            bases.append(4096 + es * int(rng.integers(0, 60)))
+        want = _brute_overlap(bases, views, es)
+        hits += want
+        assert mb.muon_views_overlap(bases, views, es) == want, (case, bases, views, es)
+    assert 30 < hits < 270          # the sample exercises both answers
