@@ -146,6 +146,15 @@ int muon_plan_describe(const muon_options_t* opt, const muon_shape_t* shapes, in
 int muon_plan_launch_sets(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count,
                           int32_t* num_sets, int32_t* set_of);
 
+/* Host-only description of what muon_step_flat_host runs: the launch sets of its plan -- the plan above with two
+ * small sets (about 2^24 elements each) split off the group with the smallest matrices -- and the order in which the
+ * pipeline runs them: one small set first and the other last, because the inbound copy before the first kernel and
+ * the outbound copy after the last one are the only copies nothing overlaps; in between, largest first (the
+ * descending-size order of Section 6.7).  set_of[i]: launch set of matrix i (-1 for empty matrices; may be NULL);
+ * order[k]: the set that runs k-th (may be NULL; at most order_capacity entries are written). */
+int muon_plan_pipeline(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count, int32_t* num_sets,
+                       int32_t* set_of, int32_t* order, int32_t order_capacity);
+
 /* Host-only: the tile list the tensor engine uses for a symmetric product (A = X X^T, A A^T) whose result has
  * `blocks` x `blocks` blocks of 128 rows/columns.  Tile i is tiles[4i..4i+3] = (ra, rb, cc, cd): row blocks ra
  * and rb (one per CTA of a pair; 0xFFFF = none) against column blocks cc and cd (0xFFFF = the tile is 128

@@ -66,6 +66,8 @@ _sig = {
     "muon_set_workspace": (C.c_int, [_vp, _vp, C.c_size_t]),
     "muon_plan_describe": (C.c_int, [C.POINTER(Options), C.POINTER(Shape), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
     "muon_plan_launch_sets": (C.c_int, [C.POINTER(Options), C.POINTER(Shape), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
+    "muon_plan_pipeline": (C.c_int, [C.POINTER(Options), C.POINTER(Shape), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32),
+                                     C.POINTER(C.c_int32), C.c_int32]),
     "muon_symmetric_tiles": (C.c_int, [C.c_int32, C.POINTER(C.c_uint16), C.c_int32, C.POINTER(C.c_int32)]),
     "muon_layout_validate": (C.c_int, [C.POINTER(LayoutDesc)]),
     "muon_layout_create": (C.c_int, [_vp, C.POINTER(LayoutDesc), C.POINTER(_vp)]),
@@ -160,6 +162,16 @@ def muon_workspace_bytes(opt: Options, shapes) -> int:
     out = C.c_size_t(0)
     _check(lib.muon_workspace_bytes(C.byref(opt), _shapes(shapes), len(shapes), C.byref(out)), "muon_workspace_bytes")
     return int(out.value)
+
+
+def muon_plan_pipeline(opt: Options, shapes) -> Tuple[List[int], List[int]]:
+    """(launch set of every matrix, order in which the host-buffer pipeline runs the sets)."""
+    n = C.c_int32(0)
+    set_of = (C.c_int32 * max(1, len(shapes)))()
+    cap = len(shapes) + 2
+    order = (C.c_int32 * cap)()
+    _check(lib.muon_plan_pipeline(C.byref(opt), _shapes(shapes), len(shapes), C.byref(n), set_of, order, cap), "muon_plan_pipeline")
+    return [int(set_of[i]) for i in range(len(shapes))], [int(order[k]) for k in range(int(n.value))]
 
 
 def muon_views_overlap(bases, views, elem_size: int) -> bool:

@@ -106,16 +106,18 @@ struct Span {
   }
 };
 
-Plan* get_plan(muon_ctx* ctx, const muon_shape_t* shapes, int32_t count, int* status, const uint8_t* odd_pitch = nullptr) {
+Plan* get_plan(muon_ctx* ctx, const muon_shape_t* shapes, int32_t count, int* status, const uint8_t* odd_pitch = nullptr,
+               int64_t edge_elems = 0) {
   std::string key(reinterpret_cast<const char*>(shapes), size_t(count) * sizeof(muon_shape_t));
   if (odd_pitch) key.append(reinterpret_cast<const char*>(odd_pitch), size_t(count));
+  if (edge_elems) key.append("/edge").append(std::to_string(edge_elems));
   auto it = ctx->plans.find(key);
   if (it != ctx->plans.end()) {
     *status = MUON_OK;
     return &it->second;
   }
   Plan p;
-  *status = build_plan(ctx->opt, shapes, count, &p, odd_pitch);
+  *status = build_plan(ctx->opt, shapes, count, &p, odd_pitch, edge_elems);
   if (*status != MUON_OK) return nullptr;
   if (ctx->plans.size() > 64) {
     for (auto& kv : ctx->plans) release_plan_tables(&kv.second);
@@ -351,6 +353,32 @@ int run_set(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStream_t st)
 // Host-buffer pipeline: per launch set, gradients arrive by DMA straight into the whole-matrix buffers (the
 // copy engine performs the gather) and updates leave the same way, on two copy streams that run ahead
 // of / behind the compute stream.
+constexpr int64_t kPipeEdgeElems = int64_t(1) << 24;
+
+// Order in which the host-buffer pipeline runs the launch sets: only the first set's inbound copy and the last
+// set's outbound copy are exposed, so the smallest set goes first and the second smallest last; the others keep the
+// plan's order (largest first, the descending-size order of Section 6.7).
+std::vector<size_t> pipeline_order(const Plan& plan) {
+  std::vector<size_t> order(plan.sets.size());
+  for (size_t c = 0; c < order.size(); ++c) order[c] = c;
+  auto elems = [&](size_t c) { return plan.sets[c].elems; };
+  if (plan.pipeline_ordered) return order;       // the plan was built with ramp sets at both ends, in running order
+  if (order.size() > 2) {
+    size_t small = 0;
+    for (size_t c = 1; c < order.size(); ++c)
+      if (elems(c) < elems(small)) small = c;
+    order.erase(order.begin() + long(small));
+    size_t second = 0;
+    for (size_t k = 1; k < order.size(); ++k)
+      if (elems(order[k]) < elems(order[second])) second = k;
+    const size_t last = order[second];
+    order.erase(order.begin() + long(second));
+    order.insert(order.begin(), small);
+    order.push_back(last);
+  }
+  return order;
+}
+
 struct HostPipe {
   const char* host_in;
   char* host_out;
@@ -382,7 +410,8 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
       if (lds[i] % 8) odd[size_t(i)] = 1, any = true;
     if (!any) odd.clear();
   }
-  Plan* plan = get_plan(ctx, shapes, count, &status, odd.empty() ? nullptr : odd.data());
+  // host-buffer pipeline: the first and the last batch are small (16 Mi elements), see build_plan
+  Plan* plan = get_plan(ctx, shapes, count, &status, odd.empty() ? nullptr : odd.data(), pipe ? kPipeEdgeElems : 0);
   if (!plan) return status;
   if (plan->live == 0) return MUON_OK;
   if (!ctx->ws || ctx->ws_bytes < plan->ws_bytes) return MUON_ERR_WORKSPACE_TOO_SMALL;
@@ -455,38 +484,28 @@ int run_batched(muon_ctx* ctx, void* const* w, const void* const* g, void* const
   if (!ev || cudaEventRecord(ev, st) != cudaSuccess) return MUON_ERR_CUDA;
   if (cudaStreamWaitEvent(ctx->h2d_stream, ev, 0) != cudaSuccess || cudaStreamWaitEvent(ctx->d2h_stream, ev, 0) != cudaSuccess)
     return MUON_ERR_CUDA;
-  // Order of the batches: only the first batch's inbound copy and the last batch's outbound copy are exposed,
-  // so the smallest batch goes first and the second smallest last; the others keep the plan's order
-  // (largest first, the descending-size order of Section 6.7).
-  std::vector<size_t> order(plan->sets.size());
-  for (size_t c = 0; c < order.size(); ++c) order[c] = c;
-  auto elems = [&](size_t c) { return plan->sets[c].elems; };
-  if (order.size() > 2) {
-    size_t small = 0;
-    for (size_t c = 1; c < order.size(); ++c)
-      if (elems(c) < elems(small)) small = c;
-    order.erase(order.begin() + long(small));
-    size_t second = 0;
-    for (size_t k = 1; k < order.size(); ++k)
-      if (elems(order[k]) < elems(order[second])) second = k;
-    const size_t last = order[second];
-    order.erase(order.begin() + long(second));
-    order.insert(order.begin(), small);
-    order.push_back(last);
-  }
+  const std::vector<size_t> order = pipeline_order(*plan);
   std::vector<cudaEvent_t> arrived(plan->sets.size());
-  for (size_t c : order) {                                       // all inbound copies are queued up front, in batch order
+  auto enqueue_inbound = [&](size_t c) {
     for (int32_t ci : plan->sets[c].chunks)
       for (int32_t i : plan->chunks[size_t(ci)].mats)
         for (const muon_segment_t& sg : pipe->layout->segs_of[size_t(i)])
           if (cudaMemcpyAsync(static_cast<char*>(const_cast<void*>(g[i])) + size_t(sg.elem_begin) * es,
                               pipe->host_in + size_t(sg.flat_offset) * es, size_t(sg.elem_count) * es, cudaMemcpyHostToDevice,
                               ctx->h2d_stream) != cudaSuccess)
-            return MUON_ERR_CUDA;
+            return false;
     arrived[c] = next_sync_event(ctx);
-    if (!arrived[c] || cudaEventRecord(arrived[c], ctx->h2d_stream) != cudaSuccess) return MUON_ERR_CUDA;
-  }
-  for (size_t c : order) {
+    return arrived[c] && cudaEventRecord(arrived[c], ctx->h2d_stream) == cudaSuccess;
+  };
+  // Inbound copies are queued a few sets ahead of the kernels that need them, not all up front: a stream takes
+  // only so many pending operations before the enqueueing call blocks, and a host thread stuck queueing the copies of
+  // late sets would launch the kernels of the early ones late.
+  constexpr size_t kInboundAhead = 3;
+  size_t queued = 0;
+  for (size_t pos = 0; pos < order.size(); ++pos) {
+    while (queued < order.size() && queued <= pos + kInboundAhead)
+      if (!enqueue_inbound(order[queued++])) return MUON_ERR_CUDA;
+    const size_t c = order[pos];
     if (cudaStreamWaitEvent(st, arrived[c], 0) != cudaSuccess) return MUON_ERR_CUDA;
     status = run_set(ctx, set_run(c), r, st);
     if (status != MUON_OK) return status;
@@ -616,6 +635,26 @@ int muon_plan_launch_sets(const muon_options_t* opt, const muon_shape_t* shapes,
     for (int32_t i = 0; i < count; ++i) set_of[i] = -1;
     for (const Chunk& c : p.chunks)
       for (int32_t i : c.mats) set_of[i] = c.set;
+  }
+  return MUON_OK;
+}
+
+int muon_plan_pipeline(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count, int32_t* num_sets, int32_t* set_of,
+                       int32_t* order, int32_t order_capacity) {
+  if (!opt || !num_sets || count < 0 || (count > 0 && !shapes) || order_capacity < 0) return MUON_ERR_INVALID_ARG;
+  if (!valid_options(*opt)) return MUON_ERR_INVALID_ARG;
+  Plan p;
+  const int st = build_plan(*opt, shapes, count, &p, nullptr, kPipeEdgeElems);
+  if (st != MUON_OK) return st;
+  *num_sets = int32_t(p.sets.size());
+  if (set_of) {
+    for (int32_t i = 0; i < count; ++i) set_of[i] = -1;
+    for (const Chunk& c : p.chunks)
+      for (int32_t i : c.mats) set_of[i] = c.set;
+  }
+  if (order) {
+    const std::vector<size_t> ord = pipeline_order(p);
+    for (size_t k = 0; k < ord.size() && k < size_t(order_capacity); ++k) order[k] = int32_t(ord[k]);
   }
   return MUON_OK;
 }

@@ -66,6 +66,7 @@ struct Plan {
   std::vector<LaunchSet> sets;
   size_t ws_bytes = 0;
   int32_t live = 0;      // matrices with rows > 0 and cols > 0
+  bool pipeline_ordered = false;   // the sets are listed in the order the host-buffer pipeline runs them (ramps at both ends)
   // tensor-core tables: built when the plan first runs on a workspace, rebuilt when the workspace moves
   void* d_tables = nullptr;
   const void* tables_ws = nullptr;
@@ -74,7 +75,7 @@ struct Plan {
 
 size_t elem_bytes_of_ns(int ns_precision);
 int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t count, Plan* plan,
-               const uint8_t* odd_pitch = nullptr);
+               const uint8_t* odd_pitch = nullptr, int64_t edge_elems = 0);
 // Lays the chunks of one launch set out in a workspace (fills Chunk::off_*, part_off and the set's offsets).
 void layout_set(const muon_options_t& opt, std::vector<Chunk>* chunks, LaunchSet* set);
 // Tile list of a symmetric product over nb x nb blocks of 128: every unordered pair of blocks exactly once.

@@ -1,5 +1,6 @@
 // Host-side planning: shape-fused batching (Section 6.6), workspace carving, layout validation.
 #include <algorithm>
+#include <cstdlib>
 #include <iterator>
 #include <map>
 #include <numeric>
@@ -22,83 +23,196 @@ size_t elem_bytes_of_ns(int ns_precision) { return ns_precision == MUON_NS_FP32 
 // `odd_pitch` (may be null) marks strided views whose row pitch is not a multiple of 8 elements: they form groups
 // of their own, so that the elementwise kernels chosen for a matrix -- and with them the order in which its norm is
 // summed -- never depend on what else is in the call.
-int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t count, Plan* plan, const uint8_t* odd_pitch) {
+// `edge_elems` > 0 (the host-buffer pipeline): the sets come out in the order the pipeline runs them, with a ramp at
+// either end.  Copies and kernels overlap only from the second set on, and a set's kernels cannot start before its own
+// inbound copy has finished, so a pipeline that opens with a full-size set waits for its whole copy, and one that closes
+// with a full-size set waits for that set's whole outbound copy.  The ramp sets start at about edge_elems elements and
+// grow as fast as the kernels of the sets before them can cover the next copy; the sets in the middle are the ordinary
+// ones, largest first (the descending-size order of Section 6.7).
+int build_plan(const muon_options_t& opt, const muon_shape_t* shapes, int32_t count, Plan* plan, const uint8_t* odd_pitch,
+               int64_t edge_elems) {
   plan->chunks.clear();
   plan->sets.clear();
   plan->ws_bytes = 0;
   plan->live = 0;
+  plan->pipeline_ordered = false;
   typedef std::pair<std::pair<int32_t, int32_t>, int32_t> GroupKey;      // ((s, l), odd pitch)
-  std::map<GroupKey, std::vector<int32_t>> groups;
-  std::vector<GroupKey> order;
-  for (int32_t i = 0; i < count; ++i) {
+  auto key_of = [&](int32_t i) {
     const int32_t r = shapes[i].rows, c = shapes[i].cols;
-    if (r < 0 || c < 0) return MUON_ERR_INVALID_ARG;
-    if (r == 0 || c == 0) continue;
-    const GroupKey key(std::make_pair(std::min(r, c), std::max(r, c)), (odd_pitch && odd_pitch[i]) ? 1 : 0);
-    auto it = groups.find(key);
-    if (it == groups.end()) {
-      order.push_back(key);
-      it = groups.emplace(key, std::vector<int32_t>()).first;
-    }
-    it->second.push_back(i);
-    plan->live++;
+    return GroupKey(std::make_pair(std::min(r, c), std::max(r, c)), (odd_pitch && odd_pitch[i]) ? 1 : 0);
+  };
+  auto elems_of_mat = [&](int32_t i) { return int64_t(shapes[i].rows) * shapes[i].cols; };
+  std::vector<int32_t> live;
+  int64_t total = 0;
+  for (int32_t i = 0; i < count; ++i) {
+    if (shapes[i].rows < 0 || shapes[i].cols < 0) return MUON_ERR_INVALID_ARG;
+    if (shapes[i].rows == 0 || shapes[i].cols == 0) continue;
+    live.push_back(i);
+    total += elems_of_mat(i);
   }
+  plan->live = int32_t(live.size());
   const int64_t cap = opt.chunk_elems > 0 ? opt.chunk_elems : (int64_t(1) << 29);
-  std::vector<Chunk> chunks;
-  for (const auto& key : order) {
-    const std::vector<int32_t>& idx = groups[key];
-    const int64_t per = int64_t(key.first.first) * key.first.second;
-    // as few chunks as the cap allows, of (nearly) equal size: a short last chunk would run its fifteen
-    // products on a mostly idle device
-    const int64_t max_per_chunk = std::max<int64_t>(1, cap / per);
-    const int64_t num_chunks = (int64_t(idx.size()) + max_per_chunk - 1) / max_per_chunk;
-    const size_t base = idx.size() / size_t(num_chunks), rem = idx.size() % size_t(num_chunks);
-    size_t b = 0;
-    for (int64_t ci = 0; ci < num_chunks; ++ci) {
-      Chunk ch;
-      ch.s = key.first.first;
-      ch.l = key.first.second;
-      ch.pitch8 = key.second == 0;
-      ch.ldx = int32_t(up(size_t(ch.l), 8));
-      ch.lda = int32_t(up(size_t(ch.s), 8));
-      const size_t e = b + base + (size_t(ci) < rem ? 1 : 0);
-      ch.mats.assign(idx.begin() + long(b), idx.begin() + long(e));
-      b = e;
-      ch.count = int32_t(ch.mats.size());
-      const int32_t ts = (ch.s + kElemTile - 1) / kElemTile, tl = (ch.l + kElemTile - 1) / kElemTile;
-      ch.tiles_per_mat = ts * tl;
-      chunks.push_back(std::move(ch));
-    }
-  }
-  // first-fit decreasing into launch sets (stable for equal sizes, so the result is a pure function of the shape list)
+
+  // a bin = the chunks of one launch set
+  std::vector<std::vector<Chunk>> bins;
+  auto make_chunk = [&](const GroupKey& key, std::vector<int32_t>::const_iterator b, std::vector<int32_t>::const_iterator e) {
+    Chunk ch;
+    ch.s = key.first.first;
+    ch.l = key.first.second;
+    ch.pitch8 = key.second == 0;
+    ch.ldx = int32_t(up(size_t(ch.l), 8));
+    ch.lda = int32_t(up(size_t(ch.s), 8));
+    ch.mats.assign(b, e);
+    ch.count = int32_t(ch.mats.size());
+    const int32_t ts = (ch.s + kElemTile - 1) / kElemTile, tl = (ch.l + kElemTile - 1) / kElemTile;
+    ch.tiles_per_mat = ts * tl;
+    return ch;
+  };
   auto elems_of = [](const Chunk& c) { return int64_t(c.count) * c.s * c.l; };
-  std::vector<size_t> by_size(chunks.size());
-  std::iota(by_size.begin(), by_size.end(), size_t(0));
-  std::stable_sort(by_size.begin(), by_size.end(), [&](size_t a, size_t b) { return elems_of(chunks[a]) > elems_of(chunks[b]); });
-  std::vector<std::vector<size_t>> bins;
-  std::vector<int64_t> fill;
-  for (size_t ci : by_size) {
-    const int64_t e = elems_of(chunks[ci]);
-    size_t k = 0;
-    while (k < bins.size() && (fill[k] + e > cap || bins[k].size() >= size_t(kMaxElemChunks))) ++k;
-    if (k == bins.size()) {
-      bins.emplace_back();
-      fill.push_back(0);
+
+  // ---- ramps (pipeline plans only, and only when the ramps leave at least half of the work to full-size sets)
+  std::vector<std::vector<int32_t>> ramp[2];       // [0]: opening sets, first to last; [1]: closing sets, last to first
+  if (edge_elems > 0 && total >= 16 * edge_elems) {
+    // Ramp sets are built from the matrices with the most Newton-Schulz work per element (their kernels hide the most
+    // copy time per byte copied); matrices with little work per element stay in the middle of the pipeline.  A set may
+    // hold edge_elems elements plus what the kernels of the sets before it can cover: kFlopsPerElem flops of kernel work
+    // per element copied (about 1.3 PFLOP/s of products against 25 G elements/s over the host link, with a margin).
+    constexpr double kFlopsPerElem = 65536.0;
+    auto flops_of_mat = [&](int32_t i) {                    // five steps of (3 s^2 l + s^3) multiply-adds
+      const double sm = double(std::min(shapes[i].rows, shapes[i].cols)), lg = double(std::max(shapes[i].rows, shapes[i].cols));
+      return 10.0 * sm * sm * (3.0 * lg + sm);
+    };
+    std::vector<int32_t> asc = live;
+    std::stable_sort(asc.begin(), asc.end(), [&](int32_t a, int32_t b) {
+      const double da = flops_of_mat(a) / double(elems_of_mat(a)), db = flops_of_mat(b) / double(elems_of_mat(b));
+      return da > db || (da == db && elems_of_mat(a) < elems_of_mat(b));
+    });
+    size_t cur = 0;
+    int64_t used = 0;
+    double work_before[2] = {0.0, 0.0};
+    bool open[2] = {true, true};
+    while (open[0] || open[1]) {
+      for (int side = 0; side < 2; ++side) {
+        if (!open[side]) continue;
+        const int64_t target = std::min(edge_elems + int64_t(work_before[side] / kFlopsPerElem), cap);
+        std::vector<int32_t> set;
+        std::vector<GroupKey> keys;
+        int64_t e = 0;
+        double w = 0.0;
+        size_t c = cur;
+        while (c < asc.size() && e < target) {
+          const int64_t m = elems_of_mat(asc[c]);
+          if (!set.empty() && e + m > std::max(target, edge_elems)) break;      // never overshoot the target by a matrix
+          const GroupKey k = key_of(asc[c]);
+          if (std::find(keys.begin(), keys.end(), k) == keys.end()) {
+            if (keys.size() == size_t(kMaxElemChunks)) break;
+            keys.push_back(k);
+          }
+          set.push_back(asc[c]);
+          e += m;
+          w += flops_of_mat(asc[c]);
+          ++c;
+        }
+        // the ramp ends where its sets reach half the cap, or where it would take more than a quarter of the work
+        if (set.empty() || used + e > total / 4 || target >= cap / 2) {
+          open[side] = false;
+          continue;
+        }
+        cur = c;
+        used += e;
+        work_before[side] += w;
+        ramp[side].push_back(std::move(set));
+      }
     }
-    bins[k].push_back(ci);
-    fill[k] += e;
+    std::vector<uint8_t> taken(size_t(count), 0);
+    for (int side = 0; side < 2; ++side)
+      for (const auto& set : ramp[side])
+        for (int32_t i : set) taken[size_t(i)] = 1;
+    live.erase(std::remove_if(live.begin(), live.end(), [&](int32_t i) { return taken[size_t(i)] != 0; }), live.end());
   }
+  auto bin_of_set = [&](std::vector<int32_t> set) {         // one launch set from an explicit list of matrices
+    std::sort(set.begin(), set.end());
+    std::vector<GroupKey> keys;
+    std::map<GroupKey, std::vector<int32_t>> by_key;
+    for (int32_t i : set) {
+      const GroupKey k = key_of(i);
+      if (by_key.find(k) == by_key.end()) keys.push_back(k);
+      by_key[k].push_back(i);
+    }
+    std::vector<Chunk> bin;
+    for (const GroupKey& k : keys) bin.push_back(make_chunk(k, by_key[k].begin(), by_key[k].end()));
+    std::stable_sort(bin.begin(), bin.end(), [&](const Chunk& a, const Chunk& b) { return elems_of(a) > elems_of(b); });
+    return bin;
+  };
+  for (auto& set : ramp[0]) bins.push_back(bin_of_set(std::move(set)));
+
+  // ---- the ordinary sets: shape groups, evenly cut at the cap, packed first fit (largest first)
+  {
+    std::map<GroupKey, std::vector<int32_t>> groups;
+    std::vector<GroupKey> order;
+    for (int32_t i : live) {
+      const GroupKey key = key_of(i);
+      auto it = groups.find(key);
+      if (it == groups.end()) {
+        order.push_back(key);
+        it = groups.emplace(key, std::vector<int32_t>()).first;
+      }
+      it->second.push_back(i);
+    }
+    std::vector<Chunk> chunks;
+    for (const auto& key : order) {
+      const std::vector<int32_t>& idx = groups[key];
+      const int64_t per = int64_t(key.first.first) * key.first.second;
+      // as few chunks as the cap allows, of (nearly) equal size: a short last chunk would run its fifteen
+      // products on a mostly idle device
+      const int64_t max_per_chunk = std::max<int64_t>(1, cap / per);
+      const int64_t num_chunks = (int64_t(idx.size()) + max_per_chunk - 1) / max_per_chunk;
+      const size_t base = idx.size() / size_t(num_chunks), rem = idx.size() % size_t(num_chunks);
+      size_t b = 0;
+      for (int64_t ci = 0; ci < num_chunks; ++ci) {
+        const size_t e = b + base + (size_t(ci) < rem ? 1 : 0);
+        chunks.push_back(make_chunk(key, idx.begin() + long(b), idx.begin() + long(e)));
+        b = e;
+      }
+    }
+    // first-fit decreasing (stable for equal sizes, so the result is a pure function of the shape list)
+    std::vector<size_t> by_size(chunks.size());
+    std::iota(by_size.begin(), by_size.end(), size_t(0));
+    std::stable_sort(by_size.begin(), by_size.end(), [&](size_t a, size_t b) { return elems_of(chunks[a]) > elems_of(chunks[b]); });
+    std::vector<std::vector<size_t>> packed;
+    std::vector<int64_t> fill;
+    for (size_t ci : by_size) {
+      const int64_t e = elems_of(chunks[ci]);
+      size_t k = 0;
+      while (k < packed.size() && (fill[k] + e > cap || packed[k].size() >= size_t(kMaxElemChunks))) ++k;
+      if (k == packed.size()) {
+        packed.emplace_back();
+        fill.push_back(0);
+      }
+      packed[k].push_back(ci);
+      fill[k] += e;
+    }
+    for (const auto& pk : packed) {
+      std::vector<Chunk> bin;
+      for (size_t ci : pk) bin.push_back(std::move(chunks[ci]));
+      bins.push_back(std::move(bin));
+    }
+  }
+  for (size_t k = ramp[1].size(); k-- > 0;) bins.push_back(bin_of_set(std::move(ramp[1][k])));
+  plan->pipeline_ordered = !ramp[0].empty() || !ramp[1].empty();
+
   // final order: set by set, descriptors contiguous inside a set
   int32_t desc_begin = 0;
   for (size_t k = 0; k < bins.size(); ++k) {
     LaunchSet set;
     set.desc_begin = desc_begin;
-    set.elems = fill[k];
-    for (size_t ci : bins[k]) {
-      Chunk ch = std::move(chunks[ci]);
+    set.elems = 0;
+    for (Chunk& src : bins[k]) {
+      Chunk ch = std::move(src);
       ch.set = int32_t(k);
       ch.desc_begin = desc_begin;
       desc_begin += ch.count;
+      set.elems += elems_of(ch);
       set.chunks.push_back(int32_t(plan->chunks.size()));
       plan->chunks.push_back(std::move(ch));
     }

@@ -135,3 +135,49 @@ def test_llama3_8b_flat_concat_round_trip_bit_exact():
         assert torch.equal(back[i].view(torch.int16), src[i].view(torch.int16)), i
     L.close()
     ctx.close()
+
+
+def test_host_buffer_pipeline_with_ramp_sets_matches_the_device_resident_step():
+    """muon_step_flat_host on a set large enough for its plan to ramp (8 layers of the 1B-class stack, 360 M elements:
+    small sets first and last, full-size sets in between).  Different batching,
+    same results: parameters, momenta, updates and the host-side flat update buffer are bit-identical to scatter-free
+    device-resident muon_step_batched_out on the same gradients."""
+    from paper_2609_21594_b200 import binding as mb
+
+    dev = torch.device("cuda", 0)
+    shapes = wl.shapes_1b(8)
+    opt = mb.muon_default_options()
+    set_of, order = mb.muon_plan_pipeline(opt, shapes)
+    assert len(order) >= mb.muon_plan_launch_sets(opt, shapes)[0] + 2         # the ramps are really there
+    ctx = mb.Context()
+    ctx.ensure_workspace(shapes)
+    layout = wl.layout_per_param(shapes, 8)
+    L = mb.Layout(ctx, layout, 2)
+    W0 = [wl.device_draw("pipe", 0, i, "param", s, dev, std=0.02, dtype=torch.float32) for i, s in enumerate(shapes)]
+    G = [wl.device_draw("pipe", 0, i, "grad", s, dev, std=1e-3, dtype=torch.bfloat16) for i, s in enumerate(shapes)]
+    M0 = [wl.device_draw("pipe", 1, i, "grad", s, dev, std=1e-3, dtype=torch.float32) for i, s in enumerate(shapes)]
+    flat = torch.zeros(layout.flat_len, dtype=torch.bfloat16, device=dev)
+    ctx.muon_scatter(flat, L, G)
+    host_in = torch.empty(layout.flat_len, dtype=torch.bfloat16).pin_memory()
+    host_in.copy_(flat)
+    host_out = torch.zeros(layout.flat_len, dtype=torch.bfloat16).pin_memory()
+    # device-resident reference
+    Wa, Ma = [w.clone() for w in W0], [m.clone() for m in M0]
+    Oa = [torch.empty(s, dtype=torch.bfloat16, device=dev) for s in shapes]
+    ctx.muon_step_batched_out(Wa, G, Ma, Oa, shapes, LR, MU, WD, wl.NS_STEPS, QUINTIC)
+    # host-buffer pipeline (gradients arrive by copy engine into Gb)
+    Wb, Mb = [w.clone() for w in W0], [m.clone() for m in M0]
+    Gb = [torch.zeros(s, dtype=torch.bfloat16, device=dev) for s in shapes]
+    Ob = [torch.zeros(s, dtype=torch.bfloat16, device=dev) for s in shapes]
+    ctx.muon_step_flat_host(host_in, host_out, L, Wb, Gb, Mb, Ob, LR, MU, WD, wl.NS_STEPS, QUINTIC)
+    torch.cuda.synchronize()
+    assert ctx.muon_last_device_status() == 0
+    for i in range(len(shapes)):
+        assert torch.equal(Gb[i].view(torch.int16), G[i].view(torch.int16)), i
+        assert torch.equal(Wb[i], Wa[i]) and torch.equal(Mb[i], Ma[i]), i
+        assert torch.equal(Ob[i].view(torch.int16), Oa[i].view(torch.int16)), i
+    flat_o = torch.zeros(layout.flat_len, dtype=torch.bfloat16, device=dev)
+    ctx.muon_scatter(flat_o, L, Oa)
+    assert torch.equal(host_out.view(torch.int16), flat_o.cpu().view(torch.int16))
+    L.close()
+    ctx.close()

@@ -159,3 +159,54 @@ def test_views_overlap_against_brute_force():
         hits += want
         assert mb.muon_views_overlap(bases, views, es) == want, (case, bases, views, es)
     assert 30 < hits < 270          # the sample exercises both answers
+
+
+# ----------------------------------------------------------------------------- host-buffer pipeline plan
+@pytest.mark.parametrize("name", ["llama8b", "moe", "1b", "tiny", "odd"])
+def test_pipeline_plan_ramps(name):
+    """What muon_step_flat_host runs: every matrix in exactly one set, every set within the cap and within 8 core
+    shapes, and -- when the work is large enough to ramp -- sets listed in running order that open and close with about
+    2^24 elements and grow no faster than the kernels of the sets before them can cover the next copy (65536 flops of
+    Newton-Schulz work per element copied), so that the copies no kernel overlaps stay short."""
+    shapes = {"llama8b": wl.shapes_llama8b, "moe": wl.shapes_moe, "1b": wl.shapes_1b, "tiny": wl.shapes_tiny,
+              "odd": wl.shapes_odd}[name]()
+    opt = mb.muon_default_options()
+    set_of, order = mb.muon_plan_pipeline(opt, shapes)
+    nsets = len(order)
+    assert sorted(order) == list(range(nsets))
+    assert all(0 <= s < nsets for s in set_of) and len(set_of) == len(shapes)
+    elems, work = [0] * nsets, [0.0] * nsets
+    kinds = [set() for _ in range(nsets)]
+    for (m, n), s in zip(shapes, set_of):
+        sm, lg = min(m, n), max(m, n)
+        elems[s] += m * n
+        work[s] += 10.0 * sm * sm * (3 * lg + sm)
+        kinds[s].add((sm, lg))
+    cap, edge = 1 << 29, 1 << 24
+    assert all(0 < e <= cap or len(k) == 1 for e, k in zip(elems, kinds))
+    assert all(len(k) <= 8 for k in kinds)
+    total = sum(elems)
+    if total < 16 * edge:                                   # too little work to ramp: the ordinary plan
+        assert (nsets, set_of) == mb.muon_plan_launch_sets(opt, shapes)
+        return
+    assert order == list(range(nsets))                      # listed in running order
+    biggest = max(m * n for m, n in shapes)
+    assert elems[0] <= max(edge, biggest) and elems[-1] <= max(edge, biggest)
+
+    def ramp_length(seq):
+        done, k = 0.0, 0
+        while k < len(seq) and elems[seq[k]] < cap // 2:
+            target = edge + done / 65536.0
+            if elems[seq[k]] > max(target, edge, min(m * n for m, n in shapes)):
+                break
+            done += work[seq[k]]
+            k += 1
+        return k
+
+    up, down = ramp_length(list(range(nsets))), ramp_length(list(range(nsets - 1, -1, -1)))
+    assert up >= 2 and down >= 2, (up, down, elems)
+    # the ramps are made of the matrices with the most work per element
+    dens = sorted({(10.0 * min(m, n) ** 2 * (3 * max(m, n) + min(m, n))) / (m * n) for m, n in shapes}, reverse=True)
+    assert work[0] / elems[0] == pytest.approx(dens[0])
+    # and leave most of the work to full-size sets
+    assert sum(e for e in elems if e >= cap // 4) >= total // 2
