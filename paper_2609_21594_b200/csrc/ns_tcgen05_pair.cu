@@ -470,20 +470,16 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
         if (!__shfl_sync(0xffffffffu, go ? 1 : 0, 0)) { ok = false; break; }
       }
       bool have = pair_id < V.total_tiles;
-      Tile tl;
-      if (have) tl = decode_tile(pair_id, V);
+      EpiTile cur, nxt;                             // each tile is decoded once: `nxt` becomes `cur`
+      if (have) nxt = make_epi(decode_tile(pair_id, V), int(rank), V, L);
       for (int t = pair_id; have && ok; t += num_pairs, ++tile_it) {
         const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
         const uint32_t taddr = tmem_base + acc * 256u + (uint32_t(quad * 32) << 16);
-        const EpiTile cur = make_epi(tl, int(rank), V, L);
-        EpiTile nxt;
+        cur = nxt;
         nxt.valid = false;
         nxt.d = nullptr;
         have = t + num_pairs < V.total_tiles;       // the prefetch of D never crosses a product boundary
-        if (have) {
-          tl = decode_tile(t + num_pairs, V);
-          nxt = make_epi(tl, int(rank), V, L);
-        }
+        if (have) nxt = make_epi(decode_tile(t + num_pairs, V), int(rank), V, L);
         if (cur.valid) {
           ok = epilogue_tile(cur, nxt, taddr, epi_base, dfull_bar(0), egroup_bar, tfull_bar(int(acc)), aph, abort_flag, est, quad,
                              lane);
