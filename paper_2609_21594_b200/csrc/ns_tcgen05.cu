@@ -223,8 +223,8 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
       nxt.valid = false;
       nxt.d = nullptr;
       if (t + int(gridDim.x) < total_tiles) nxt = epi_of(decode_tile(t + int(gridDim.x), a));
-      ok = epilogue_tile(cur, nxt, taddr, epi_base, dfull_bar(0), egroup_bar, tfull_bar(int(acc)), aph, abort_flag, est, quad,
-                         lane);
+      ok = epilogue_tile<1>(cur, nxt, taddr, epi_base, dfull_bar(0), egroup_bar, tfull_bar(int(acc)), aph, abort_flag, est, quad,
+                            lane, 0, quad == 2 && lane == 0);
       if (!ok) break;
       tc_fence_before();
       __syncwarp();

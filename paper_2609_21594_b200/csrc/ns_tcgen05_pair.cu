@@ -11,16 +11,18 @@
 // the tile spans column blocks cc and cd (N = 256) or cc alone (N = 128), and CTA r stages half of the
 // N columns of Q per 64-wide k-block.  The leader (r = 0) issues tcgen05.mma.cta_group::2 of shape
 // M256 x N x K16; each CTA keeps its 128 x N fp32 accumulator in its own TMEM (double-buffered) and runs
-// its own epilogue.  Symmetric products (P = Q, C = C^T) come with an explicit per-matrix tile list that
-// covers every unordered pair of blocks exactly once, so no block of the triangle is computed twice and a
-// ragged last block costs a 128-wide tile instead of a 256-wide one; off-diagonal blocks are mirrored.
+// its own epilogue with eight warps (two per TMEM lane quadrant, each converting half of every 64-column
+// chunk: the epilogue of a tile is a chain of latencies, and tiles with few k-blocks wait for it).
+// Symmetric products (P = Q, C = C^T) come with an explicit per-matrix tile list over the block triangle
+// (2 x 2 block tiles, a ragged last column block gets 128-wide tiles); a symmetric result is stored only
+// where tiles compute it and read transposed where a consumer needs the other half.
 //
 // Synchronisation (all waits bounded):
 //   full[s]    leader only.  The leader's producer arms it with the bytes of BOTH CTAs; both producers'
 //              TMA loads complete on it (cta_group::2 form, no multicast).
 //   empty[s]   in each CTA; the leader's tcgen05.commit arrives on both (commit multicast).
 //   tfull[a]   in each CTA; commit multicast after a tile's last k-block.
-//   tempty[a]  leader only, 8 arrivals: the four epilogue warps of each CTA (remote arrive).
+//   tempty[a]  leader only, 16 arrivals: the eight epilogue warps of each CTA (remote arrive).
 //   drain      in each CTA; the issuer's last commit, awaited before TMEM is freed.
 // A role that gives up sets the abort flag of BOTH CTAs (remote store), records a code in the status word
 // and leaves; everybody else notices the flag inside its own bounded wait.
@@ -43,7 +45,9 @@ constexpr int B_BYTES = 128 * BK * 2;         // 16 KiB: this CTA's half of the 
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BUFS * EPI_BYTES + 1024 + 256;
 constexpr int TMEM_COLS = 512;
-constexpr int NUM_THREADS = 192;
+constexpr int EPI_SPLIT = 2;                      // epilogue warps per TMEM lane quadrant
+constexpr int EPI_WARPS = 4 * EPI_SPLIT;
+constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;   // warp 0: TMA producer, warp 1: MMA issuer, then the epilogue warps
 // constant parts of the shared-memory matrix descriptors (see make_desc): K-major (LBO 16, SBO 1024) and
 // MN-major (LBO 8 KiB between 64-element chunks, SBO 1024), 128-byte swizzle
 constexpr uint64_t DESC_HI_K = (uint64_t(16 >> 4) << 16) | (uint64_t(1024 >> 4) << 32) | (uint64_t(1) << 46) | (uint64_t(2) << 61);
@@ -351,10 +355,10 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(tfull_bar(i), 1);
-      mbar_init(tempty_bar(i), 8);
+      mbar_init(tempty_bar(i), 2 * EPI_WARPS);     // every epilogue warp of both CTAs
     }
     for (int i = 0; i < EPI_BUFS; ++i) mbar_init(dfull_bar(i), 1);
-    mbar_init(egroup_bar, 4);
+    mbar_init(egroup_bar, EPI_WARPS);
     mbar_init(drain_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -459,6 +463,8 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
   } else {
     // ------------------------------------------------------------------ epilogue warps (per CTA: its 128 rows)
     const int quad = warp & 3;                     // TMEM lane quadrant this warp may read
+    const int part = (warp - 2) >> 2;              // which share of a chunk's columns this warp converts
+    const bool epi_leader = warp == 2 && lane == 0;
     EpilogueState est;
     uint32_t tile_it = 0;
     bool ok = true;
@@ -481,8 +487,8 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
         have = t + num_pairs < V.total_tiles;       // the prefetch of D never crosses a product boundary
         if (have) nxt = make_epi(decode_tile(t + num_pairs, V), int(rank), V, L);
         if (cur.valid) {
-          ok = epilogue_tile(cur, nxt, taddr, epi_base, dfull_bar(0), egroup_bar, tfull_bar(int(acc)), aph, abort_flag, est, quad,
-                             lane);
+          ok = epilogue_tile<EPI_SPLIT>(cur, nxt, taddr, epi_base, dfull_bar(0), egroup_bar, tfull_bar(int(acc)), aph, abort_flag,
+                                        est, quad, lane, part, epi_leader);
         } else {                                    // no rows for this CTA: hand the accumulator straight back
           ok = mbar_wait(tfull_bar(int(acc)), aph, abort_flag);
         }
@@ -497,13 +503,13 @@ ns_product_pair_kernel(const __grid_constant__ TcLaunch L) {
         if (lane == 0) mbar_arrive(egroup_bar);
         ok = mbar_wait(egroup_bar, est.eph, abort_flag);
         est.eph ^= 1u;
-        if (ok && quad == 2 && lane == 0) {
+        if (ok && epi_leader) {
           tma_wait_all();
           grid_arrive(L.barrier);
         }
       }
     }
-    if (quad == 2 && lane == 0) {
+    if (epi_leader) {
       tma_wait_all();                               // every store has landed before the CTA retires
       if (!ok)                                      // a prefetched D chunk may still be landing: give it (bounded) time
         for (int i = 0; i < 64; ++i) __nanosleep(1000);

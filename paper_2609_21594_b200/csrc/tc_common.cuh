@@ -181,10 +181,16 @@ __device__ __forceinline__ int epi_chunk_col(const EpiTile& t, int cb) {        
 // place (one bf16 rounding of gamma*(beta*D + alpha*acc)), TMA stores the chunk; an off-diagonal block of a
 // symmetric product is also written transposed with plain stores (64 contiguous bytes per warp instruction).
 // `next` is the tile this CTA processes afterwards (for the prefetch).  Returns false when a bounded wait expired.
+// SPLIT warps share a lane quadrant (they may all read its 32 TMEM lanes): warp `part` of them handles columns
+// [part * 64 / SPLIT, (part + 1) * 64 / SPLIT) of every chunk, so a chunk's conversion work is spread over 4 * SPLIT warps.
+// `leader`: the one thread of the group that issues TMA loads and stores.
+template <int SPLIT>
 __device__ __forceinline__ bool epilogue_tile(const EpiTile& cur, const EpiTile& next, uint32_t taddr, uint32_t epi_base,
                                               uint32_t dfull_bar0, uint32_t egroup_bar, uint32_t tfull_bar, uint32_t aph,
-                                              volatile int* abort_flag, EpilogueState& st, int quad, int lane) {
-  const bool leader = quad == 2 && lane == 0;        // warp 2 is the first epilogue warp
+                                              volatile int* abort_flag, EpilogueState& st, int quad, int lane, int part,
+                                              bool leader) {
+  static_assert(SPLIT == 1 || SPLIT == 2, "one or two warps per lane quadrant");
+  constexpr int WCOLS = EPI_COLS / SPLIT;            // columns of a chunk this warp converts
   const int lrow = quad * 32 + lane;
   auto group_sync = [&]() -> bool {                  // rendezvous of the four warps on an mbarrier: bounded like every wait
     __syncwarp();
@@ -243,14 +249,16 @@ __device__ __forceinline__ bool epilogue_tile(const EpiTile& cur, const EpiTile&
       if (!group_sync()) return false;                // the leader's wait_group above frees the buffer for everyone
     }
     st.d_in_flight = prefetch;
-    uint32_t v[64];
-    tc_ld32(taddr + uint32_t(cb * EPI_COLS), *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
-    tc_ld32(taddr + uint32_t(cb * EPI_COLS + 32), *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+    uint32_t v[WCOLS];
+#pragma unroll
+    for (int h = 0; h < WCOLS / 32; ++h)
+      tc_ld32(taddr + uint32_t(cb * EPI_COLS + part * WCOLS + h * 32), *reinterpret_cast<uint32_t(*)[32]>(&v[h * 32]));
     tc_wait_ld();
     const bool mirror = cb < 2 ? cur.mirror0 : cur.mirror1;
     const uint32_t srow = ebuf + uint32_t(lrow) * 128u;
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {                     // 16-byte piece q of the row sits at piece q ^ (row & 7)
+    for (int qq = 0; qq < WCOLS / 8; ++qq) {          // 16-byte piece q of the row sits at piece q ^ (row & 7)
+      const int q = part * (WCOLS / 8) + qq;
       const uint32_t addr = srow + (uint32_t(q ^ (lrow & 7)) << 4);
       uint32_t d0 = 0, d1 = 0, d2 = 0, d3 = 0;
       if (cur.d) asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3) : "r"(addr));
@@ -258,7 +266,7 @@ __device__ __forceinline__ bool epilogue_tile(const EpiTile& cur, const EpiTile&
       uint32_t oo[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        float x0 = alpha * __uint_as_float(v[q * 8 + 2 * e]), x1 = alpha * __uint_as_float(v[q * 8 + 2 * e + 1]);
+        float x0 = alpha * __uint_as_float(v[qq * 8 + 2 * e]), x1 = alpha * __uint_as_float(v[qq * 8 + 2 * e + 1]);
         if (cur.d) {
           const __nv_bfloat162 dp = *reinterpret_cast<const __nv_bfloat162*>(&dd[e]);
           x0 += beta * __low2float(dp);
