@@ -131,11 +131,14 @@ def newton_schulz(U: np.ndarray, steps: int, coeffs: Sequence[float], eps: float
     Transpose-first rule (Section 6.6): when rows > cols the iteration runs on U^T so the
     Gram factor A = X X^T is the small square; the result is transposed back.
 
+    The step of Eq. 1 is evaluated as the matrix polynomial it is: X_{k+1} = P_k X_k with
+    P_k = a_k I + b_k A + c_k A^2, A = X_k X_k^T (three produced matrices per step: A, P, X).
+
     Rounding schedule in "bf16" mode ("cast then fold"): U is taken as given (already
     bf16-valued); the normaliser r = 1/(||U||_F + eps) is not applied to U but folded
-    into the first step, A = r^2 (U U^T) and X_1 = r (a U + B U), which equals Eq. 1 on
-    X_0 = r U exactly in real arithmetic; each produced A, B, X is rounded once.
-    `trace`, if given, receives (A, B, X) after every step (in the working orientation).
+    into the first step, A = r^2 (U U^T) and X_1 = r (P U), which equals Eq. 1 on
+    X_0 = r U exactly in real arithmetic; each produced A, P, X is rounded once.
+    `trace`, if given, receives (A, P, X) after every step (in the working orientation).
     """
     U = np.asarray(U, dtype=np.float64)
     rows, cols = U.shape
@@ -146,18 +149,19 @@ def newton_schulz(U: np.ndarray, steps: int, coeffs: Sequence[float], eps: float
         X = _round(r * X, mode)
         return X.T.copy() if tall else X
     r = 1.0 / (np.sqrt(np.sum(X * X)) + eps)
+    eye = np.eye(X.shape[0])
     for k in range(steps):
         a, b, c = _coeff(coeffs, k)
         if k == 0:
             A = _round((r * r) * np.matmul(X, X.T), mode)
-            B = _round(b * A + c * np.matmul(A, A), mode)
-            X = _round(r * (a * X + np.matmul(B, X)), mode)
+            P = _round(a * eye + b * A + c * np.matmul(A, A), mode)
+            X = _round(r * np.matmul(P, X), mode)
         else:
             A = _round(np.matmul(X, X.T), mode)
-            B = _round(b * A + c * np.matmul(A, A), mode)
-            X = _round(a * X + np.matmul(B, X), mode)
+            P = _round(a * eye + b * A + c * np.matmul(A, A), mode)
+            X = _round(np.matmul(P, X), mode)
         if trace is not None:
-            trace.append((A.copy(), B.copy(), X.copy()))
+            trace.append((A.copy(), P.copy(), X.copy()))
     return X.T.copy() if tall else X
 
 
@@ -165,8 +169,8 @@ def ns_single_step(X: np.ndarray, a: float, b: float, c: float, mode: str = "fp6
     """One iteration of Eq. 1 on an already-normalised, wide-or-square X (teacher-forced checks)."""
     X = np.asarray(X, dtype=np.float64)
     A = _round(np.matmul(X, X.T), mode)
-    B = _round(b * A + c * np.matmul(A, A), mode)
-    return _round(a * X + np.matmul(B, X), mode)
+    P = _round(a * np.eye(X.shape[0]) + b * A + c * np.matmul(A, A), mode)
+    return _round(np.matmul(P, X), mode)
 
 
 # --------------------------------------------------------------------------- full step

@@ -368,12 +368,12 @@ def test_bf16_mode_rounding_points_on_scalars():
     x = u
     a, b, c = QUINTIC
     A = _bf(r * r * u * u)
-    B = _bf(b * A + c * A * A)
-    x = _bf(r * (a * u + B * u))
+    P = _bf(a + b * A + c * A * A)      # the polynomial a I + b A + c A^2 is one produced matrix, rounded once
+    x = _bf(r * (P * u))
     for _ in range(4):
         A = _bf(x * x)
-        B = _bf(b * A + c * A * A)
-        x = _bf(a * x + B * x)
+        P = _bf(a + b * A + c * A * A)
+        x = _bf(P * x)
     got = orc.newton_schulz(np.array([[u]]), 5, QUINTIC, eps, "bf16")
     assert got[0, 0] == x
     # and it is NOT what un-rounded arithmetic gives (the roundings are really applied)
@@ -388,12 +388,12 @@ def test_bf16_mode_diagonal_matrix_follows_scalar_schedule():
     xs = []
     for u in d:
         A = _bf(r * r * u * u)
-        B = _bf(b * A + c * A * A)
-        x = _bf(r * (a * u + B * u))
+        P = _bf(a + b * A + c * A * A)
+        x = _bf(r * (P * u))
         for _ in range(4):
             A = _bf(x * x)
-            B = _bf(b * A + c * A * A)
-            x = _bf(a * x + B * x)
+            P = _bf(a + b * A + c * A * A)
+            x = _bf(P * x)
         xs.append(x)
     got = orc.newton_schulz(np.diag(d), 5, QUINTIC, eps, "bf16")
     assert np.array_equal(got, np.diag(xs))
