@@ -183,7 +183,8 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
   const float* rnorm = reinterpret_cast<const float*>(base + sr.set->off_rnorm);
   int n;
   if (sr.tables) {
-    auto launch = [&](const tc::TcTable& tab, float alpha, float beta, int gamma_mode, int coef_a, int coef_b, int coef_off) {
+    auto launch = [&](const tc::TcTable& tab, float alpha, float beta, float diag, int gamma_mode, int coef_a, int coef_b, int coef_d,
+                      int coef_off) {
       tc::TcLaunch L;
       L.persist = nullptr;
       for (int i = 0; i < tab.nprob; ++i) {
@@ -192,9 +193,9 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
       }
       L.nprob = tab.nprob;
       L.total_tiles = tab.total_tiles;
-      L.alpha = alpha; L.beta = beta; L.gamma_mode = gamma_mode;
+      L.alpha = alpha; L.beta = beta; L.diag = diag; L.gamma_mode = gamma_mode;
       L.coef_table = sr.d_coef;
-      L.coef_a = coef_a; L.coef_b = coef_b; L.coef_off = coef_off;
+      L.coef_a = coef_a; L.coef_b = coef_b; L.coef_d = coef_d; L.coef_off = coef_off;
       L.coef_stride = sr.coef_stride;
       L.coef_per_step = ctx->opt.coeffs_per_step;
       L.status = ctx->d_status;
@@ -209,7 +210,7 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
       if (pairs > 0 && sr.tables->max_tiles <= 2 * ctx->persist_pairs) {
         tc::TcLaunch L;
         std::memset(static_cast<void*>(&L), 0, sizeof(L));
-        L.coef_a = L.coef_b = -1;
+        L.coef_a = L.coef_b = L.coef_d = -1;
         L.coef_table = sr.d_coef;
         L.coef_stride = sr.coef_stride;
         L.coef_per_step = ctx->opt.coeffs_per_step;
@@ -233,11 +234,11 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
       const int off = ctx->opt.coeffs_per_step ? 3 * k : 0;
       const float* co = r.coeffs + off;      // with per-matrix rows these scalars are replaced row by row on the device
       const int cur = k & 1;
-      if ((n = launch(sr.tables->g1[cur], 1.f, 0.f, k == 0 ? 2 : 0, -1, -1, off)) < 0) return n;     // A = gamma X X^T
+      if ((n = launch(sr.tables->g1[cur], 1.f, 0.f, 0.f, k == 0 ? 2 : 0, -1, -1, -1, off)) < 0) return n;   // A = gamma X X^T
       *launches += n;
-      if ((n = launch(sr.tables->g2, co[2], co[1], 0, 2, 1, off)) < 0) return n;                   // B = b A + c A A^T (A symmetric)
+      if ((n = launch(sr.tables->g2, co[2], co[1], co[0], 0, 2, 1, 0, off)) < 0) return n;                  // P = a I + b A + c A A^T
       *launches += n;
-      if ((n = launch(sr.tables->g3[cur], 1.f, co[0], k == 0 ? 1 : 0, -1, 0, off)) < 0) return n;   // X' = gamma (a X + B X)
+      if ((n = launch(sr.tables->g3[cur], 1.f, 0.f, 0.f, k == 0 ? 1 : 0, -1, -1, -1, off)) < 0) return n;   // X' = gamma P X
       *launches += n;
     }
     return MUON_OK;
@@ -257,7 +258,8 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
       GemmArgs g{};
       g.coef = sr.d_coef ? sr.d_coef + size_t(ch.desc_begin - sr.set->desc_begin) * size_t(sr.coef_stride) + off : nullptr;
       g.coef_stride = sr.coef_stride;
-      g.coef_a = g.coef_b = -1;
+      g.coef_a = g.coef_b = g.coef_d = -1;
+      g.diag = 0.f;
       g.p = cur; g.q = cur; g.d = nullptr; g.c = A;
       g.m = ch.s; g.n = ch.s; g.kdim = ch.l;
       g.ldp = ch.ldx; g.ldq = ch.ldx; g.ldc = ch.lda;
@@ -269,16 +271,16 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
       g.p = A; g.q = A; g.d = A; g.c = B;
       g.kdim = ch.s; g.ldp = ch.lda; g.ldq = ch.lda;
       g.stride_p = sa_; g.stride_q = sa_;
-      g.gamma_mode = 0; g.alpha = co[2]; g.beta = co[1];
-      g.coef_a = 2; g.coef_b = 1;
+      g.gamma_mode = 0; g.alpha = co[2]; g.beta = co[1]; g.diag = co[0];         // P = a I + b A + c A A^T
+      g.coef_a = 2; g.coef_b = 1; g.coef_d = 0;
       if ((n = run_gemm(ctx, g, st)) < 0) return n;
       *launches += n;
-      g.p = B; g.q = cur; g.d = cur; g.c = nxt;
+      g.p = B; g.q = cur; g.d = nullptr; g.c = nxt;                                  // X' = gamma P X
       g.m = ch.s; g.n = ch.l; g.kdim = ch.s;
       g.ldp = ch.lda; g.ldq = ch.ldx; g.ldc = ch.ldx;
       g.stride_p = sa_; g.stride_q = sx; g.stride_c = sx;
-      g.gamma_mode = (k == 0) ? 1 : 0; g.alpha = 1.f; g.beta = co[0]; g.nn = 1; g.symmetric = 0;
-      g.coef_a = -1; g.coef_b = 0;
+      g.gamma_mode = (k == 0) ? 1 : 0; g.alpha = 1.f; g.beta = 0.f; g.diag = 0.f; g.nn = 1; g.symmetric = 0;
+      g.coef_a = g.coef_b = g.coef_d = -1;
       if ((n = run_gemm(ctx, g, st)) < 0) return n;
       *launches += n;
     }
@@ -1053,7 +1055,8 @@ int muon_ns_product(muon_ctx_t* ctx, const void* p, const void* q, const void* d
     L.total_tiles = tab.total_tiles;
     L.alpha = g.alpha; L.beta = g.beta; L.gamma_mode = g.gamma_mode;
     L.coef_table = nullptr;
-    L.coef_a = L.coef_b = -1;
+    L.diag = 0.f;
+    L.coef_a = L.coef_b = L.coef_d = -1;
     L.coef_off = L.coef_stride = L.coef_per_step = 0;
     L.status = ctx->d_status;
     Span sp(ctx, MUON_PHASE_NS, st);

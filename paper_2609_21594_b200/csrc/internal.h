@@ -211,7 +211,7 @@ int launch_apply(const ApplyArgs& a, cudaStream_t st);
 // no staging buffer, no host-to-device copy that could outlive its source.
 int launch_poke(void* dst, const void* src, size_t bytes, cudaStream_t st);
 
-// C[k] = gamma_k * (beta * D[k] + alpha * op(P[k], Q[k])),  op = P Q^T (nn=0) or P Q (nn=1)
+// C[k] = gamma_k * (beta * D[k] + alpha * op(P[k], Q[k]) + diag * I),  op = P Q^T (nn=0) or P Q (nn=1)
 struct GemmArgs {
   const void* p; const void* q; const void* d; void* c;
   int32_t m, n, kdim;
@@ -221,12 +221,13 @@ struct GemmArgs {
   const float* rnorm;  // device, per matrix
   int32_t gamma_mode;  // 0: 1, 1: r, 2: r*r
   float alpha, beta;
+  float diag;          // added to the diagonal elements C[i][i] (square results)
   int32_t nn;
   int32_t symmetric;   // op is P P^T with symmetric result (kernels may exploit it)
-  // per-matrix coefficients: matrix k takes alpha = coef[k * coef_stride + coef_a] (beta likewise with coef_b) when
+  // per-matrix coefficients: matrix k takes alpha = coef[k * coef_stride + coef_a] (beta, diag likewise with coef_b, coef_d) when
   // coef is set and the index is >= 0
   const float* coef;   // device or null
-  int32_t coef_a, coef_b, coef_stride;
+  int32_t coef_a, coef_b, coef_d, coef_stride;   // coef_d: index that replaces diag
 };
 int launch_gemm_simt(const GemmArgs& a, int ns_precision, cudaStream_t st);
 int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st);   // tcgen05 engine, single-CTA kernel (bf16 only)

@@ -1,8 +1,8 @@
 // Plain CUDA-core batched product kernel for the Newton-Schulz iteration (Eq. 1).
 // It serves the fp32 precision mode (every product in true fp32: TF32 operands are not
 // accurate enough for a 1e-4 match to fp64) and shapes the tensor-core engine does not take.
-//   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k]^T)      (nn = 0:  A = X X^T,  B = bA + c A A^T)
-//   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k])        (nn = 1:  X' = aX + B X)
+//   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k]^T + diag * I)   (nn = 0:  A = X X^T,  P = aI + bA + c A A^T)
+//   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k])                (nn = 1:  X' = P X)
 #include "internal.h"
 
 namespace muon {
@@ -83,11 +83,12 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs a, int tiles_m,
     const float r = a.rnorm[mat];
     gamma = a.gamma_mode == 1 ? r : r * r;
   }
-  float alpha = a.alpha, beta = a.beta;
+  float alpha = a.alpha, beta = a.beta, diag = a.diag;
   if (a.coef) {
     const float* co = a.coef + size_t(mat) * size_t(a.coef_stride);
     if (a.coef_a >= 0) alpha = co[a.coef_a];
     if (a.coef_b >= 0) beta = co[a.coef_b];
+    if (a.coef_d >= 0) diag = co[a.coef_d];
   }
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -100,6 +101,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs a, int tiles_m,
       const size_t off = size_t(r) * a.ldc + c;
       float v = alpha * acc[i][j];
       if (D) v += beta * ldf<T>(D + off);
+      if (r == c) v += diag;
       C[off] = cvt<T>(gamma * v);
     }
   }

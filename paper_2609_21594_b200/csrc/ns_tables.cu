@@ -71,7 +71,7 @@ int build_set_image(void* encode_fn, const void* ws, const std::vector<Chunk>& c
     }
   }
   // tensor maps per chunk: X iterates as 128-row boxes (P, Q, D, C), as 64-row boxes (Q of a 128-wide tile) and as
-  // 64 x 64 boxes (the MN-major operand of X' = aX + B X); A as 128- and 64-row boxes, B as 128-row boxes
+  // 64 x 64 boxes (the MN-major operand of X' = P X); A as 128- and 64-row boxes, B as 128-row boxes
   struct Maps {
     CUtensorMap xr[2], xh[2], a, ah, b, bh;
   };
@@ -129,7 +129,7 @@ int build_set_image(void* encode_fn, const void* ws, const std::vector<Chunk>& c
         p.row_pairs = 0;
         p.pattern = static_cast<const TilePat*>(ib.dev(pat.first));
         p.tiles_per_mat = pat.second;
-      } else if (kind == 2) {    // B = beta A + alpha A A^T
+      } else if (kind == 2) {    // P = delta I + beta A + alpha A A^T
         m.p = m.q = m.d = mp.a;
         m.ph = m.qh = mp.ah;
         m.c = mp.b;
@@ -142,7 +142,7 @@ int build_set_image(void* encode_fn, const void* ws, const std::vector<Chunk>& c
         p.row_pairs = 0;
         p.pattern = static_cast<const TilePat*>(ib.dev(pat.first));
         p.tiles_per_mat = pat.second;
-      } else {                   // X' = gamma (beta X + B X)
+      } else {                   // X' = gamma P X
         const int cur = kind - 3;
         m.p = mp.b;
         m.ph = mp.bh;
@@ -150,7 +150,7 @@ int build_set_image(void* encode_fn, const void* ws, const std::vector<Chunk>& c
         m.q = m.qh = mp.xh[cur];                   // 64 x 64 boxes: same geometry as the 64-row boxes
         m.d = mp.xr[cur];
         m.c = mp.xr[cur ^ 1];
-        p.d = reinterpret_cast<const __nv_bfloat16*>(wsb + c.off_x[cur]);
+        p.d = nullptr;
         p.c = reinterpret_cast<__nv_bfloat16*>(const_cast<char*>(wsb + c.off_x[cur ^ 1]));
         p.m = c.s; p.n = c.l; p.kdim = c.s; p.ldc = c.ldx; p.stride_c = int64_t(c.s) * c.ldx;
         p.nn = 1;

@@ -2,8 +2,8 @@
 // operands and fp32 accumulation in tensor memory.  It serves matrices of at most 128 rows and is the
 // cross-check of the paired-CTA kernel, which runs everything else.
 //
-//   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k]^T)     nn = 0   (A = X X^T,  B = bA + cA A^T)
-//   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k])       nn = 1   (X' = aX + B X)
+//   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k]^T + diag * I)   nn = 0   (A = X X^T,  P = aI + bA + cA A^T)
+//   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k])                nn = 1   (X' = P X)
 //
 // One persistent CTA per SM, 192 threads, warp-specialised:
 //   warp 0      TMA producer: cp.async.bulk.tensor loads of 128B-swizzled operand tiles into a
@@ -202,11 +202,12 @@ ns_product_tc_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
       e.cblk0 = tl.n0 / 128;
       e.cblk1 = tl.n0 + 128 < a.n ? tl.n0 / 128 + 1 : -1;
       e.mirror0 = e.mirror1 = a.symmetric && tl.n0 >= tl.m0 + BM;       // tile lies strictly above the diagonal
-      e.alpha = a.alpha; e.beta = a.beta; e.gamma = 1.f;
+      e.alpha = a.alpha; e.beta = a.beta; e.diag = a.diag; e.gamma = 1.f;
       if (a.coef) {
         const float* co = a.coef + size_t(tl.mat) * size_t(a.coef_stride);
         if (a.coef_a >= 0) e.alpha = co[a.coef_a];
         if (a.coef_b >= 0) e.beta = co[a.coef_b];
+        if (a.coef_d >= 0) e.diag = co[a.coef_d];
       }
       if (a.gamma_mode) {
         const float r = a.rnorm[tl.mat];
@@ -331,8 +332,8 @@ int launch_gemm_tc(muon_ctx* ctx, const GemmArgs& a, cudaStream_t st) {
   }
   t.rnorm = a.rnorm;
   t.gamma_mode = a.gamma_mode;
-  t.alpha = a.alpha; t.beta = a.beta;
-  t.coef = a.coef; t.coef_a = a.coef_a; t.coef_b = a.coef_b; t.coef_stride = a.coef_stride;
+  t.alpha = a.alpha; t.beta = a.beta; t.diag = a.diag;
+  t.coef = a.coef; t.coef_a = a.coef_a; t.coef_b = a.coef_b; t.coef_d = a.coef_d; t.coef_stride = a.coef_stride;
   t.status = ctx->d_status;
   const int64_t tiles = int64_t(t.tiles_per_mat) * t.batch;
   const unsigned grid = unsigned(tiles < g_num_sms[ctx->device] ? tiles : g_num_sms[ctx->device]);

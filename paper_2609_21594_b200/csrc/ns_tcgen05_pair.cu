@@ -1,9 +1,9 @@
 // Paired-CTA tensor-core engine for the Newton-Schulz products (Eq. 1), grouped over heterogeneous
-// shapes: ONE launch computes the same product (A = X X^T, B = bA + cA A^T or X' = aX + B X) for every
+// shapes: ONE launch computes the same product (A = X X^T, P = aI + bA + cA A^T or X' = P X) for every
 // shape group that is resident in the workspace (the shape-fused batching of Section 6.6, taken one
 // step further: not one batched kernel per core shape but one per product for all core shapes).
 //
-//   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k]^T)   (nn = 0)      C[k] = ... P[k] Q[k]   (nn = 1)
+//   C[k] = gamma_k * (beta * D[k] + alpha * P[k] Q[k]^T + diag * I)   (nn = 0)      C[k] = ... P[k] Q[k]   (nn = 1)
 //
 // The launch reads a table of problems from global memory (tensor maps encoded once per plan, shapes,
 // tile counts) and walks one global tile list with persistent clusters of two CTAs.  A tile is given in
@@ -112,20 +112,20 @@ struct PhaseView {
   const TcMaps* maps;
   const TcProbInfo* info;
   int nprob, total_tiles;
-  float alpha, beta;
+  float alpha, beta, diag;
   int gamma_mode;
-  int coef_a, coef_b, coef_off;   // per-matrix coefficient rows: see TcLaunch
+  int coef_a, coef_b, coef_d, coef_off;   // per-matrix coefficient rows: see TcLaunch
 };
 
 // Product `ph` of the launch.  A one-product launch carries its tables by value; a whole-iteration launch reads
 // them from device memory and derives the scalars of step k = ph / 3 from the coefficient rows:
-// A = gamma X X^T (gamma = r^2 at k = 0), B = b A + c A A^T, X' = gamma (a X + B X) (gamma = r at k = 0).
+// A = gamma X X^T (gamma = r^2 at k = 0), P = a I + b A + c A A^T, X' = gamma P X (gamma = r at k = 0).
 __device__ __forceinline__ PhaseView phase_view(const TcLaunch& L, int ph) {
   PhaseView v;
   if (!L.persist) {
     v.maps = L.maps; v.info = L.info; v.nprob = L.nprob; v.total_tiles = L.total_tiles;
-    v.alpha = L.alpha; v.beta = L.beta; v.gamma_mode = L.gamma_mode;
-    v.coef_a = L.coef_a; v.coef_b = L.coef_b; v.coef_off = L.coef_off;
+    v.alpha = L.alpha; v.beta = L.beta; v.diag = L.diag; v.gamma_mode = L.gamma_mode;
+    v.coef_a = L.coef_a; v.coef_b = L.coef_b; v.coef_d = L.coef_d; v.coef_off = L.coef_off;
     return v;
   }
   const int k = ph / 3, j = ph - 3 * k, cur = k & 1;
@@ -135,10 +135,12 @@ __device__ __forceinline__ PhaseView phase_view(const TcLaunch& L, int ph) {
   v.nprob = L.persist->nprob;
   v.total_tiles = L.persist->total_tiles[kind];
   v.alpha = j == 1 ? L.coef[k][2] : 1.f;
-  v.beta = j == 0 ? 0.f : (j == 1 ? L.coef[k][1] : L.coef[k][0]);
+  v.beta = j == 1 ? L.coef[k][1] : 0.f;
+  v.diag = j == 1 ? L.coef[k][0] : 0.f;
   v.gamma_mode = k == 0 ? (j == 0 ? 2 : (j == 2 ? 1 : 0)) : 0;
   v.coef_a = j == 1 ? 2 : -1;
-  v.coef_b = j == 0 ? -1 : (j == 1 ? 1 : 0);
+  v.coef_b = j == 1 ? 1 : -1;
+  v.coef_d = j == 1 ? 0 : -1;
   v.coef_off = L.coef_per_step ? 3 * k : 0;
   return v;
 }
@@ -189,7 +191,7 @@ __device__ __forceinline__ EpiTile make_epi(const Tile& tl, int rank, const Phas
   e.mirror0 = sym && tl.cc != e.rblk && !(in_cols && (tl.cc == tl.ra || tl.cc == tl.rb));
   e.mirror1 = sym && tl.cd != e.rblk && !(in_cols && (tl.cd == tl.ra || tl.cd == tl.rb));
   e.valid = e.rblk >= 0;
-  e.alpha = V.alpha; e.beta = V.beta; e.gamma = 1.f;
+  e.alpha = V.alpha; e.beta = V.beta; e.diag = V.diag; e.gamma = 1.f;
   if (e.valid) {
     if (V.gamma_mode) {
       const float r = p.rnorm[tl.mat];
@@ -199,6 +201,7 @@ __device__ __forceinline__ EpiTile make_epi(const Tile& tl, int rank, const Phas
       const float* co = L.coef_table + size_t(p.mat_begin + tl.mat) * size_t(L.coef_stride) + V.coef_off;
       if (V.coef_a >= 0) e.alpha = __ldg(co + V.coef_a);
       if (V.coef_b >= 0) e.beta = __ldg(co + V.coef_b);
+      if (V.coef_d >= 0) e.diag = __ldg(co + V.coef_d);
     }
   }
   return e;

@@ -19,9 +19,9 @@ struct TcArgs {
   int32_t symmetric;        // C = C^T: compute tiles that touch the upper triangle, mirror the strictly upper ones
   const float* rnorm;
   int32_t gamma_mode;
-  float alpha, beta;
-  const float* coef;        // per-matrix coefficient rows (null: alpha, beta above for every matrix)
-  int32_t coef_a, coef_b, coef_stride;
+  float alpha, beta, diag;
+  const float* coef;        // per-matrix coefficient rows (null: alpha, beta, diag above for every matrix)
+  int32_t coef_a, coef_b, coef_d, coef_stride;
   int32_t* status;
 };
 
@@ -157,8 +157,12 @@ struct EpiTile {
   int32_t cblk0, cblk1;
   bool mirror0, mirror1;     // also write the 128 x 128 block transposed (symmetric products, off-diagonal blocks)
   float alpha, beta, gamma;
+  float diag;                // added to C[i][i] before gamma (0: nothing to add)
   bool valid;
 };
+
+struct DiagYes { static constexpr bool value = true; };
+struct DiagNo { static constexpr bool value = false; };
 
 // State the four epilogue warps carry from tile to tile.
 struct EpilogueState {
@@ -256,36 +260,48 @@ __device__ __forceinline__ bool epilogue_tile(const EpiTile& cur, const EpiTile&
     tc_wait_ld();
     const bool mirror = cb < 2 ? cur.mirror0 : cur.mirror1;
     const uint32_t srow = ebuf + uint32_t(lrow) * 128u;
+    // the chunk holds diagonal elements only when its column block is this CTA's row block
+    const bool diag_chunk = cur.diag != 0.f && (c0 >> 7) == cur.rblk;
+    auto convert = [&](auto with_diag) {
+      constexpr bool DIAG = decltype(with_diag)::value;
 #pragma unroll
-    for (int qq = 0; qq < WCOLS / 8; ++qq) {          // 16-byte piece q of the row sits at piece q ^ (row & 7)
-      const int q = part * (WCOLS / 8) + qq;
-      const uint32_t addr = srow + (uint32_t(q ^ (lrow & 7)) << 4);
-      uint32_t d0 = 0, d1 = 0, d2 = 0, d3 = 0;
-      if (cur.d) asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3) : "r"(addr));
-      const uint32_t dd[4] = {d0, d1, d2, d3};
-      uint32_t oo[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        float x0 = alpha * __uint_as_float(v[qq * 8 + 2 * e]), x1 = alpha * __uint_as_float(v[qq * 8 + 2 * e + 1]);
-        if (cur.d) {
-          const __nv_bfloat162 dp = *reinterpret_cast<const __nv_bfloat162*>(&dd[e]);
-          x0 += beta * __low2float(dp);
-          x1 += beta * __high2float(dp);
-        }
-        const __nv_bfloat162 o = __floats2bfloat162_rn(gamma * x0, gamma * x1);
-        oo[e] = *reinterpret_cast<const uint32_t*>(&o);
-      }
-      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(oo[0]), "r"(oo[1]), "r"(oo[2]), "r"(oo[3]) : "memory");
-      if (mirror && row_ok) {                         // C[c][row] = C[row][c]
+      for (int qq = 0; qq < WCOLS / 8; ++qq) {        // 16-byte piece q of the row sits at piece q ^ (row & 7)
+        const int q = part * (WCOLS / 8) + qq;
+        const uint32_t addr = srow + (uint32_t(q ^ (lrow & 7)) << 4);
+        uint32_t d0 = 0, d1 = 0, d2 = 0, d3 = 0;
+        if (cur.d) asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3) : "r"(addr));
+        const uint32_t dd[4] = {d0, d1, d2, d3};
+        uint32_t oo[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const int c = c0 + q * 8 + 2 * e;
-          const __nv_bfloat162 o = *reinterpret_cast<const __nv_bfloat162*>(&oo[e]);
-          if (c < cur.n) cmat[size_t(c) * cur.ldc + row] = __low2bfloat16(o);
-          if (c + 1 < cur.n) cmat[size_t(c + 1) * cur.ldc + row] = __high2bfloat16(o);
+          float x0 = alpha * __uint_as_float(v[qq * 8 + 2 * e]), x1 = alpha * __uint_as_float(v[qq * 8 + 2 * e + 1]);
+          if (cur.d) {
+            const __nv_bfloat162 dp = *reinterpret_cast<const __nv_bfloat162*>(&dd[e]);
+            x0 += beta * __low2float(dp);
+            x1 += beta * __high2float(dp);
+          }
+          if (DIAG) {
+            const int c = c0 + q * 8 + 2 * e;
+            if (c == row) x0 += cur.diag;
+            if (c + 1 == row) x1 += cur.diag;
+          }
+          const __nv_bfloat162 o = __floats2bfloat162_rn(gamma * x0, gamma * x1);
+          oo[e] = *reinterpret_cast<const uint32_t*>(&o);
+        }
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(oo[0]), "r"(oo[1]), "r"(oo[2]), "r"(oo[3]) : "memory");
+        if (mirror && row_ok) {                       // C[c][row] = C[row][c]
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int c = c0 + q * 8 + 2 * e;
+            const __nv_bfloat162 o = *reinterpret_cast<const __nv_bfloat162*>(&oo[e]);
+            if (c < cur.n) cmat[size_t(c) * cur.ldc + row] = __low2bfloat16(o);
+            if (c + 1 < cur.n) cmat[size_t(c + 1) * cur.ldc + row] = __high2bfloat16(o);
+          }
         }
       }
-    }
+    };
+    if (diag_chunk) convert(DiagYes());
+    else convert(DiagNo());
     fence_async_smem();                               // generic-proxy writes -> visible to the TMA store
     if (!group_sync()) return false;                  // everyone is done with the buffer (reads of D, writes of C)
     if (leader) {

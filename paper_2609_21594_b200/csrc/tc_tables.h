@@ -49,7 +49,7 @@ struct TcProbInfo {
 constexpr int kMaxProblems = kMaxElemChunks;
 
 // The five product tables of a launch set in device memory, for the launch that runs a whole Newton-Schulz
-// iteration by itself: [0], [1]: A = X X^T reading X iterate 0 / 1; [2]: B = bA + cA A^T; [3], [4]: X' = aX + B X
+// iteration by itself: [0], [1]: A = X X^T reading X iterate 0 / 1; [2]: P = aI + bA + cA A^T; [3], [4]: X' = P X
 // reading iterate 0 / 1 and writing the other.
 struct alignas(128) TcPersist {
   TcMaps maps[5][kMaxProblems];
@@ -65,12 +65,13 @@ struct TcLaunch {
   TcProbInfo info[kMaxProblems];
   int32_t nprob, total_tiles;
   float alpha, beta;
+  float diag;                // added to the diagonal of the result (the a_k I of P_k = a_k I + b_k A + c_k A^2)
   int32_t gamma_mode;        // 0: 1, 1: r, 2: r*r
   // Per-matrix coefficients: row (mat_begin + matrix) of coef_table, coef_stride floats per row, replaces the scalars:
-  // alpha = row[coef_off + coef_a], beta = row[coef_off + coef_b] (an index < 0 keeps the scalar).  A whole-iteration
+  // alpha = row[coef_off + coef_a], beta = row[coef_off + coef_b], diag = row[coef_off + coef_d] (an index < 0 keeps the scalar).  A whole-iteration
   // launch derives the indices from the product it is in (coef_off = 3 * step when coef_per_step).
   const float* coef_table;   // device, first row of the launch set; null: scalars only
-  int32_t coef_a, coef_b, coef_off, coef_stride, coef_per_step;
+  int32_t coef_a, coef_b, coef_d, coef_off, coef_stride, coef_per_step;
   int32_t* status;
   // Whole-iteration mode (persist != null): the launch walks 3 * ns_steps products, a grid-wide barrier between
   // consecutive ones, and takes tables from device memory instead of maps / info above.
@@ -112,8 +113,8 @@ inline bool encode_map(void* fn, CUtensorMap* map, const void* ptr, int cols, in
 // Tables of one launch set (tensor-core engine): for each product the problem list, longest k first.
 struct SetTables {
   tc::TcTable g1[2];   // A = X X^T, reading X iterate 0 / 1
-  tc::TcTable g2;      // B = bA + c A A^T
-  tc::TcTable g3[2];   // X' = aX + B X, reading iterate 0 / 1 and writing the other
+  tc::TcTable g2;      // P = aI + bA + c A A^T
+  tc::TcTable g3[2];   // X' = P X, reading iterate 0 / 1 and writing the other
   const tc::TcPersist* persist = nullptr;   // the same five tables in device memory (null: not built)
   int32_t max_tiles = 0;                    // largest tile count of a product
 };

@@ -411,11 +411,13 @@ def test_step_out_and_flat_host_path_match_the_plain_step():
 @pytest.mark.parametrize("engine", ENGINES)
 def test_per_step_coefficient_sets_on_the_bf16_engines(engine):
     """A different (a_k, b_k, c_k) at every step -- the form the paper's default (asymmetric, five-step) variant
-    takes (its values are not printed, so arbitrary per-step triples stand in)."""
+    takes (its values are not printed, so arbitrary per-step triples stand in; they are chosen so that the iteration stays
+    bounded on all three shapes -- an earlier set drove one singular value of the 130 x 200 case to 166 in float64, where
+    no rounding schedule can be compared with another)."""
     from paper_2609_21594_b200 import binding as mb
 
     ctx = _ctx(mb, "bf16", engine, coeffs_per_step=1)
-    co = [4.0, -6.0, 2.5, 3.8, -5.5, 2.2, 3.4445, -4.7750, 2.0315, 2.9, -3.6, 1.6, 2.3, -2.0, 0.7]
+    co = [3.2, -4.2, 1.7, 3.0, -3.6, 1.4, 3.4445, -4.7750, 2.0315, 2.6, -2.8, 1.0, 2.0, -1.5, 0.5]
     shapes = [(256, 384), (384, 256), (130, 200)]
     mats = [wl.grad_np("perstep16", 0, i, s) for i, s in enumerate(shapes)]
     outs, vals = _ortho(mb, ctx, mats, steps=5, coeffs=co)
@@ -436,7 +438,7 @@ def test_per_matrix_coefficient_rows(engine, precision, per_step):
     set_a = [3.4445, -4.7750, 2.0315]
     set_b = [1.5, -0.5, 0.0]
     if per_step:
-        row_a = [4.0, -6.0, 2.5, 3.8, -5.5, 2.2, 3.4445, -4.7750, 2.0315, 2.9, -3.6, 1.6, 2.3, -2.0, 0.7]
+        row_a = [3.2, -4.2, 1.7, 3.0, -3.6, 1.4, 3.4445, -4.7750, 2.0315, 2.6, -2.8, 1.0, 2.0, -1.5, 0.5]
         row_b = [1.5, -0.5, 0.0, 2.0, -1.5, 0.5, 1.5, -0.5, 0.0, 3.0, -3.2, 1.2, 1.5, -0.5, 0.0]
     else:
         row_a, row_b = set_a, set_b
