@@ -115,3 +115,30 @@ def test_flat_state_needs_whole_row_segments():
     assert e.value.code == mb.ERR_UNSUPPORTED and ctx.muon_launch_count() == before
     L.close()
     ctx.close()
+
+
+def test_head_interleaved_fused_qkv_as_a_layout():
+    """A permuting transform of the model adapter (Section 6.6), expressed as a layout: a grouped-query fused QKV projection
+    stored group by group -- [q heads of group 0 | k0 | v0 | q heads of group 1 | k1 | v1 | ...] along the rows of one
+    physical [G * 6 * 64, d] tensor.  The logical matrices Wq (all q heads), Wk and Wv are made of row runs that alternate
+    through the physical tensor, so no single strided view describes them; a segment table does.  The physical tensor IS
+    the flat buffer: parameters, momenta and gradients are updated in place, bit-identical to the ordinary step on
+    contiguous copies of the three logical matrices."""
+    from paper_2609_21594_b200 import binding as mb
+
+    groups, hd, d = 4, 64, 256
+    q_rows, kv_rows = 4 * hd, hd                       # per group: four query heads, one key head, one value head
+    per_group = q_rows + 2 * kv_rows
+    shapes = [(groups * q_rows, d), (groups * kv_rows, d), (groups * kv_rows, d)]
+    segs = []
+    for g in range(groups):
+        base = g * per_group * d
+        segs.append(wl.Segment(0, g * q_rows * d, q_rows * d, base))
+        segs.append(wl.Segment(1, g * kv_rows * d, kv_rows * d, base + q_rows * d))
+        segs.append(wl.Segment(2, g * kv_rows * d, kv_rows * d, base + (q_rows + kv_rows) * d))
+    lay = wl.Layout(tuple(shapes), 1, groups * per_group * d, 8, tuple(segs))
+    assert mb.muon_layout_validate(mb.make_layout_desc(lay, 2)) == mb.OK
+    W, Wn = _case(mb, shapes, lay, "gqa_qkv")
+    # and against the oracle (two steps were taken; check that the parameters moved and stayed finite)
+    for w, w0 in zip(W, Wn):
+        assert bool(torch.isfinite(w).all()) and not np.array_equal(w.cpu().numpy(), w0)
