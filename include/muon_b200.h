@@ -244,6 +244,8 @@ int muon_shard_apply(muon_ctx_t* ctx, const muon_layout_t* layout, int32_t shard
  *     M <- mu*M + G;  u = G + mu*M (Nesterov) or M;  U = cast(u)
  *     X_0 = U / (||U||_F + eps), run on U^T when rows > cols (transpose-first, Section 6.6)
  *     X_{k+1} = a_k X_k + (b_k A + c_k A^2) X_k,  A = X_k X_k^T,  k = 0..ns_steps-1
+ *       (evaluated as the matrix polynomial it is: X_{k+1} = P_k X_k with P_k = a_k I + b_k A + c_k A^2; in bf16 mode each
+ *        produced matrix -- A, P_k, X_{k+1} -- is rounded once, products accumulate in fp32)
  *     W <- W (1 - lr*wd) - lr * 0.2 sqrt(max(rows, cols)) * X_ns
  *   params, momenta : host arrays [count] of device pointers to fp32 matrices (in/out)
  *   grads           : host array  [count] of device pointers, element type opt.grad_dtype

@@ -493,6 +493,37 @@ def test_per_matrix_coefficient_rows_one_launch_per_product():
     ref.close()
 
 
+def test_per_matrix_coefficient_rows_across_launch_sets():
+    """Rows follow their matrices through the plan's reordering: a small cap forces several launch sets, two core shapes
+    share some of them, and the caller's order interleaves shapes and coefficient classes."""
+    from paper_2609_21594_b200 import binding as mb
+
+    shapes = [(256, 512), (384, 256), (512, 256), (256, 384)] * 5
+    classes = ([3.4445, -4.7750, 2.0315], [3.0, -3.2, 1.2], [1.5, -0.5, 0.0])
+    rows = [classes[(i * 7 + i // 3) % 3] for i in range(len(shapes))]
+    ctx = _ctx(mb, "bf16", "tensor", "bf16", coeffs_per_matrix=1, chunk_elems=1 << 18)
+    nsets, _ = mb.muon_plan_launch_sets(ctx.opt, shapes)
+    assert nsets >= 4
+    ctx.ensure_workspace(shapes)
+    gen = torch.Generator(device="cuda").manual_seed(78)
+    G = [(torch.randn(s, device="cuda", generator=gen) * 1e-3).to(torch.bfloat16) for s in shapes]
+    O = [torch.empty(s, dtype=torch.bfloat16, device="cuda") for s in shapes]
+    ctx.muon_orthogonalize_batched(G, O, shapes, 5, rows)
+    torch.cuda.synchronize()
+    assert ctx.muon_last_device_status() == 0
+    ctx.close()
+    ref = _ctx(mb, "bf16", "tensor", "bf16", chunk_elems=1 << 18)
+    ref.ensure_workspace(shapes)
+    for cls in classes:
+        idx = [i for i in range(len(shapes)) if rows[i] == cls]
+        O2 = [torch.empty(shapes[i], dtype=torch.bfloat16, device="cuda") for i in idx]
+        ref.muon_orthogonalize_batched([G[i] for i in idx], O2, [shapes[i] for i in idx], 5, cls)
+        torch.cuda.synchronize()
+        for j, i in enumerate(idx):
+            assert torch.equal(O2[j].view(torch.int16), O[i].view(torch.int16)), (i, shapes[i])
+    ref.close()
+
+
 def test_plain_momentum_rule_and_eps_option():
     """nesterov = 0 (u = M') and a non-default epsilon are options of the context, not compile-time choices."""
     from paper_2609_21594_b200 import binding as mb
