@@ -601,11 +601,15 @@ void muon_destroy(muon_ctx_t* ctx) {
 int muon_workspace_bytes(const muon_options_t* opt, const muon_shape_t* shapes, int32_t count, size_t* bytes) {
   if (!opt || !bytes || count < 0 || (count > 0 && !shapes)) return MUON_ERR_INVALID_ARG;
   if (!valid_options(*opt)) return MUON_ERR_INVALID_ARG;
-  Plan p;
-  const int st = build_plan(*opt, shapes, count, &p);
+  Plan p, q;
+  int st = build_plan(*opt, shapes, count, &p);
   if (st != MUON_OK) return st;
+  // the host-buffer pipeline packs the same matrices into other launch sets: the workspace covers both plans
+  st = build_plan(*opt, shapes, count, &q, nullptr, kPipeEdgeElems);
+  if (st != MUON_OK) return st;
+  const size_t need = std::max(p.ws_bytes, q.ws_bytes);
   // strided views with an odd pitch form groups of their own; the slack covers the alignment of the extra pieces
-  *bytes = p.ws_bytes ? p.ws_bytes + 4096 * p.chunks.size() : 0;
+  *bytes = need ? need + 4096 * std::max(p.chunks.size(), q.chunks.size()) : 0;
   return MUON_OK;
 }
 
