@@ -39,7 +39,7 @@ NUM_SHARDS = 8
 
 # DRAM bytes (read + write) per launch of the Newton-Schulz product kernel, from ncu captures of the same command
 # line; keyed by (config, layers).  Filled in from the committed summaries under profiles/.
-NS_TRAFFIC = {("llama8b", 32): 1.647e9}
+NS_TRAFFIC = {("llama8b", 32): 1.767e9}
 NS_TRAFFIC_NOTE = ("mean of dram__bytes_read.sum + dram__bytes_write.sum over the 210 product launches of one full-size step "
                    "(one-pass ncu launch list of this command line, summarised under profiles/); algorithmic bytes per launch: 1.27e9")
 
