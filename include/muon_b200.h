@@ -110,7 +110,9 @@ typedef struct {
   int32_t coeffs_per_matrix; /* 1: `coeffs` holds one row per matrix of the call, [count][3] or [count][3*ns_steps]:   */
                            /* matrices of one call may iterate with different polynomials (a per-parameter-group  */
                            /* choice in the pluggable design of Section 6.2); they still share their launches       */
-  int32_t reserved;        /* must be 0 */
+  int32_t launch_per_product; /* 0 (default): a launch set with only a few tiles per product runs its whole Newton-Schulz   */
+                           /* iteration as ONE launch (grid barriers between the products); 1: every product is always   */
+                           /* a launch of its own (15 per set for five steps) -- same tiles, same results                  */
 } muon_options_t;
 
 /* Fills *opt with the defaults: bf16 grads, bf16 NS, Nesterov, constant coefficients, eps 1e-7, cap 2^29. */

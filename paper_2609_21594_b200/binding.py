@@ -54,7 +54,7 @@ class LayoutDesc(C.Structure):
 class Options(C.Structure):
     _fields_ = [("grad_dtype", C.c_int32), ("ns_precision", C.c_int32), ("nesterov", C.c_int32),
                 ("coeffs_per_step", C.c_int32), ("eps", C.c_float), ("engine", C.c_int32),
-                ("chunk_elems", C.c_int64), ("coeffs_per_matrix", C.c_int32), ("reserved", C.c_int32)]
+                ("chunk_elems", C.c_int64), ("coeffs_per_matrix", C.c_int32), ("launch_per_product", C.c_int32)]
 
 
 _vp = C.c_void_p

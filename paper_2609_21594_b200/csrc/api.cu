@@ -29,6 +29,7 @@ bool valid_options(const muon_options_t& o) {
   if (o.nesterov != 0 && o.nesterov != 1) return false;
   if (o.coeffs_per_step != 0 && o.coeffs_per_step != 1) return false;
   if (o.coeffs_per_matrix != 0 && o.coeffs_per_matrix != 1) return false;
+  if (o.launch_per_product != 0 && o.launch_per_product != 1) return false;
   if (!(o.eps >= 0.f) || !std::isfinite(o.eps)) return false;
   if (o.chunk_elems < 0) return false;
   return true;
@@ -204,7 +205,7 @@ int run_set_products(muon_ctx* ctx, const SetRun& sr, const ChunkRun& r, cudaStr
     // Small sets: the whole iteration in ONE cooperative launch, products separated by grid barriers instead of
     // launch boundaries ("per-matrix NS launches starve the device for small matrices", Section 6.6 -- so do
     // per-product launches when a product is a handful of tiles).
-    if (sr.tables->persist && r.ns_steps <= tc::kMaxPersistSteps && ctx->persist_pairs != 0) {
+    if (sr.tables->persist && !ctx->opt.launch_per_product && r.ns_steps <= tc::kMaxPersistSteps && ctx->persist_pairs != 0) {
       if (ctx->persist_pairs < 0) ctx->persist_pairs = std::max(0, tc_pair_max_resident(ctx->device));
       const int pairs = std::min(ctx->persist_pairs, sr.tables->max_tiles);
       if (pairs > 0 && sr.tables->max_tiles <= 2 * ctx->persist_pairs) {
@@ -539,7 +540,7 @@ int muon_default_options(muon_options_t* opt) {
   opt->nesterov = 1;
   opt->coeffs_per_step = 0;
   opt->coeffs_per_matrix = 0;
-  opt->reserved = 0;
+  opt->launch_per_product = 0;
   opt->eps = 1e-7f;
   opt->engine = MUON_ENGINE_TENSOR;
   opt->chunk_elems = int64_t(1) << 29;

@@ -56,7 +56,7 @@ def test_default_options():
     o = mb.muon_default_options()
     assert (o.grad_dtype, o.ns_precision, o.nesterov, o.coeffs_per_step, o.engine) == (0, 0, 1, 0, 0)
     assert o.eps == pytest.approx(1e-7) and o.chunk_elems == 1 << 29
-    assert (o.coeffs_per_matrix, o.reserved) == (0, 0)
+    assert (o.coeffs_per_matrix, o.launch_per_product) == (0, 0)
 
 
 @pytest.mark.parametrize("gen", [wl.layout_per_param, wl.layout_flat_concat])

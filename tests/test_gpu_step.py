@@ -524,6 +524,45 @@ def test_per_matrix_coefficient_rows_across_launch_sets():
     ref.close()
 
 
+@pytest.mark.parametrize("shapes", [
+    [(256, 256)] * 3,
+    [(1408, 2048)] * 2,
+    [(2048, 2048)] * 2 + [(1408, 2048)] * 2,
+    wl.shapes_1b(1),
+    [(4096, 4096)] * 2 + [(1024, 4096)] * 3,
+], ids=["tiny3", "moe2", "two_shapes", "1b_layer", "llama_shapes"])
+def test_whole_iteration_launch_equals_one_launch_per_product_on_a_poisoned_workspace(shapes):
+    """The whole-iteration launch (small sets: grid barriers between the products) against the same tiles run as fifteen
+    launches: bit-identical, three times in a row, with every byte of the workspace set to 0xFF before each call -- a tile that
+    read an operand before its producer had written it would read NaNs, not the (identical) values a previous call left behind.
+    The larger sets run one launch per product either way; for them the test checks run-to-run identity on a poisoned workspace."""
+    from paper_2609_21594_b200 import binding as mb
+
+    def run(launch_per_product, reps):
+        ctx = _ctx(mb, "bf16", "tensor", launch_per_product=launch_per_product)
+        ws = torch.empty(mb.muon_workspace_bytes(ctx.opt, shapes) + 4096, dtype=torch.uint8, device="cuda")
+        ctx.muon_set_workspace(ws)
+        gen = torch.Generator(device="cuda").manual_seed(5)
+        ins = [(torch.randn(s, device="cuda", generator=gen) * 1e-3).to(torch.bfloat16) for s in shapes]
+        outs = [torch.empty_like(t) for t in ins]
+        res = []
+        for _ in range(reps):
+            ws.fill_(0xFF)
+            ctx.muon_orthogonalize_batched(ins, outs, shapes, 5, QUINTIC)
+            torch.cuda.synchronize()
+            res.append([o.clone() for o in outs])
+        assert ctx.muon_last_device_status() == 0
+        ctx.close()
+        return res
+
+    flow = run(0, 3)
+    ref = run(1, 1)[0]
+    for rep in flow:
+        for i, (a, b) in enumerate(zip(rep, ref)):
+            assert bool(torch.isfinite(a.float()).all()), i
+            assert torch.equal(a.view(torch.int16), b.view(torch.int16)), i
+
+
 def test_plain_momentum_rule_and_eps_option():
     """nesterov = 0 (u = M') and a non-default epsilon are options of the context, not compile-time choices."""
     from paper_2609_21594_b200 import binding as mb
@@ -573,8 +612,8 @@ def test_one_launch_per_product_for_all_shape_groups_and_no_encoding_in_steady_s
     encoded again."""
     from paper_2609_21594_b200 import binding as mb
 
-    def run(shapes, name):
-        ctx = _ctx(mb, "bf16", "tensor")
+    def run(shapes, name, **opt):
+        ctx = _ctx(mb, "bf16", "tensor", **opt)
         ctx.ensure_workspace(shapes)
         ins = [bf16_input(wl.grad_np(name, 0, i, s))[0] for i, s in enumerate(shapes)]
         outs = [torch.empty_like(t) for t in ins]
@@ -607,6 +646,9 @@ def test_one_launch_per_product_for_all_shape_groups_and_no_encoding_in_steady_s
     # d=256 layer, two core shapes, a handful of tiles per product: one launch for the whole iteration
     (ns, total), outs, ins = run(wl.shapes_tiny(), "grouped")
     assert ns == 1 and total == 1 + 2 + 1                                      # + stage, norm, apply
+    (ns15, total15), outs15, _ = run(wl.shapes_tiny(), "grouped", launch_per_product=1)
+    assert ns15 == 15 and total15 == 15 + 2 + 1
+    assert all(np.array_equal(a, b) for a, b in zip(outs, outs15))
     ref = orc.newton_schulz(host_f64(ins[4]), 5, QUINTIC, 1e-7, "bf16")
     assert rel(outs[4], ref) <= TOL_BF16
     # one layer of the 1B-class stack: four core shapes in one launch set, too many tiles for the single launch
