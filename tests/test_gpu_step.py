@@ -563,6 +563,35 @@ def test_whole_iteration_launch_equals_one_launch_per_product_on_a_poisoned_work
             assert torch.equal(a.view(torch.int16), b.view(torch.int16)), i
 
 
+@pytest.mark.parametrize("steps", [1, 2, 16, 17])
+def test_step_counts_at_the_edges_of_the_whole_iteration_launch(steps):
+    """One step, two steps, the largest count the whole-iteration launch takes (16) and one more (17: one launch per product):
+    bit-identical to one launch per product, and the singular values end where the quintic's fixed band says (the map is
+    chaotic inside the band, so after many steps only properties can be compared, not elements)."""
+    from paper_2609_21594_b200 import binding as mb
+
+    shapes = wl.shapes_tiny()
+    mats = [wl.grad_np("edges", 0, i, s) for i, s in enumerate(shapes)]
+    ctx = _ctx(mb, "bf16", "tensor")
+    n0 = ctx.muon_launch_count()
+    outs, vals = _ortho(mb, ctx, mats, steps=steps)
+    launches = ctx.muon_launch_count() - n0
+    assert launches == (1 if steps <= 16 else 3 * steps) + 3
+    ctx.close()
+    ref_ctx = _ctx(mb, "bf16", "tensor", launch_per_product=1)
+    ref, _ = _ortho(mb, ref_ctx, mats, steps=steps)
+    ref_ctx.close()
+    for o, r in zip(outs, ref):
+        assert np.array_equal(o, r)
+    if steps <= 2:
+        for o, v in zip(outs, vals):
+            assert rel(o, orc.newton_schulz(v, steps, QUINTIC, 1e-7, "bf16")) <= TOL_SINGLE_STEP * steps
+    else:
+        for o in outs:
+            sv = np.linalg.svd(o, compute_uv=False)
+            assert 0.6 < sv.min() and sv.max() < 1.25, (sv.min(), sv.max())
+
+
 def test_plain_momentum_rule_and_eps_option():
     """nesterov = 0 (u = M') and a non-default epsilon are options of the context, not compile-time choices."""
     from paper_2609_21594_b200 import binding as mb
