@@ -40,6 +40,8 @@ NUM_SHARDS = 8
 # DRAM bytes (read + write) per launch of the Newton-Schulz product kernel, from ncu captures of the same command
 # line; keyed by (config, layers).  Filled in from the committed summaries under profiles/.
 NS_TRAFFIC = {("llama8b", 32): 1.767e9}
+# the same capture by product (70 launches each): A = X X^T, P = aI + bA + cA A^T, X' = P X; algorithmic 1.69e9 / 0.41e9 / 2.20e9
+NS_TRAFFIC_BY_PRODUCT = {("llama8b", 32): {"G1": 2.510e9, "G2": 0.384e9, "G3": 2.408e9}}
 NS_TRAFFIC_NOTE = ("mean of dram__bytes_read.sum + dram__bytes_write.sum over the 210 product launches of one full-size step "
                    "(one-pass ncu launch list of this command line, summarised under profiles/); algorithmic bytes per launch: 1.27e9")
 
@@ -518,6 +520,7 @@ def run_ours(args, world, rank, local):
     roofline = {"bound": "tensor", "kernel": "ns_product_pair_kernel", "achieved": ns.get("tflops_algorithmic_symmetric"),
                 "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": ns.get("frac_of_sustained_peak"),
                 "traffic": NS_TRAFFIC.get((cfg, args.layers)),
+                "traffic_by_product": NS_TRAFFIC_BY_PRODUCT.get((cfg, args.layers)),
                 "traffic_note": NS_TRAFFIC_NOTE if NS_TRAFFIC.get((cfg, args.layers)) else "no capture for this workload",
                 "peak_source": f"bf16_tflops_sustained of {peaks['source']} (kernel timed inside a long step)",
                 "flops_per_launch": wl.ns_flops(shapes)[1] / max(1, ns_launches / args.steps),
