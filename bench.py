@@ -40,7 +40,7 @@ NUM_SHARDS = 8
 # DRAM bytes (read + write) per launch of the Newton-Schulz product kernel, from ncu captures of the same command
 # line; keyed by (config, layers).  Filled in from the committed summaries under profiles/.
 NS_TRAFFIC = {("llama8b", 32): 1.767e9}
-# the same capture by product (70 launches each): A = X X^T, P = aI + bA + cA A^T, X' = P X; algorithmic 1.69e9 / 0.41e9 / 2.20e9
+# the same capture by product (70 launches each): A = X X^T, P = aI + bA + cA A^T, X' = P X; algorithmic 1.21e9 / 0.41e9 / 2.20e9
 NS_TRAFFIC_BY_PRODUCT = {("llama8b", 32): {"G1": 2.510e9, "G2": 0.384e9, "G3": 2.408e9}}
 NS_TRAFFIC_NOTE = ("mean of dram__bytes_read.sum + dram__bytes_write.sum over the 210 product launches of one full-size step "
                    "(one-pass ncu launch list of this command line, summarised under profiles/); algorithmic bytes per launch: 1.27e9")
