@@ -118,6 +118,23 @@ __device__ __forceinline__ BlockPos locate_block(const Args& a) {
   return p;
 }
 
+// Sum of squares of bf16 values, the same bits whichever kernel variant computes it.  A square of a bf16 value is exact in
+// fp32; the squares of one aligned group of 8 consecutive source columns of a row are added in column order with one fp32
+// fused multiply-add each (s = fma(q, q, s), starting from 0), and only the group sums are accumulated in double.  The
+// 8-elements-per-thread kernels hold a group in one thread; here two neighbouring threads hold 4 columns each: the even
+// one runs its half of the chain, hands the result to its neighbour, and the odd one finishes the chain and owns the sum.
+// (Positions beyond the matrix hold 0, which leaves the chain unchanged.)
+__device__ __forceinline__ double sum_of_squares_group(const float (&q)[4], int tx) {
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) s = __fmaf_rn(q[i], q[i], s);
+  float t = __shfl_up_sync(0xffffffffu, s, 1);
+  if ((tx & 1) == 0) return 0.0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) t = __fmaf_rn(q[i], q[i], t);
+  return double(t);
+}
+
 // GT: gradient/input element type; XT: NS element type; MOM: momentum rule on/off.
 // Thread (ty = tid/16, tx = tid%16) handles 4 consecutive columns tx*4.. of rows ty, ty+16, ty+32, ty+48.
 template <typename GT, typename XT, bool MOM, bool FLAT>
@@ -146,6 +163,7 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
     const int rr = ty + pass * 16, cc = tx * 4;
     const int r = r0 + rr, c = c0 + cc;
     float u[4] = {0.f, 0.f, 0.f, 0.f};
+    float sq[4] = {0.f, 0.f, 0.f, 0.f};                   // this thread's rounded values of the row (0 where there is none)
     if (r < d.rows && c < d.cols) {
       const size_t off = cur.at(d, r) + c;
       float g[4], m[4] = {0.f, 0.f, 0.f, 0.f};
@@ -190,8 +208,13 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         xv[i] = XConv<XT>::from(u[i]);
-        const double q = double(XConv<XT>::to(xv[i]));
-        if (i < nv) sum += q * q;
+        const float qf = XConv<XT>::to(xv[i]);
+        if (sizeof(XT) == 2) {
+          if (i < nv) sq[i] = qf;                         // summed below, by the group-of-8 rule
+        } else {
+          const double q = double(qf);
+          if (i < nv) sum += q * q;
+        }
       }
       if (!d.transposed) {
         XT* dst = X + size_t(r) * ldx + c;     // ldx % 8 == 0 and c % 4 == 0: 8/16-byte aligned
@@ -206,6 +229,7 @@ __global__ void __launch_bounds__(256) stage_kernel(StageArgs a) {
         for (int i = 0; i < 4; ++i) tile[rr][cc + i] = xv[i];
       }
     }
+    if (sizeof(XT) == 2) sum += sum_of_squares_group(sq, tx);   // every lane takes part (shuffle inside)
   }
   if (d.transposed) {
     __syncthreads();
@@ -466,14 +490,16 @@ __global__ void __launch_bounds__(256, 6) stage_wide_kernel(StageArgs a) {
             __stcs(reinterpret_cast<float4*>(M + off) + 1, make_float4(m[4], m[5], m[6], m[7]));
           }
           uint32_t pk[4];
+          float grp = 0.f;
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const __nv_bfloat162 b = __floats2bfloat162_rn(g[2 * i], g[2 * i + 1]);
             pk[i] = *reinterpret_cast<const uint32_t*>(&b);
-            const double q0 = double(__uint_as_float(pk[i] << 16)), q1 = double(__uint_as_float(pk[i] & 0xffff0000u));
-            sum += q0 * q0;
-            sum += q1 * q1;
+            const float q0 = __uint_as_float(pk[i] << 16), q1 = __uint_as_float(pk[i] & 0xffff0000u);
+            grp = __fmaf_rn(q0, q0, grp);                          // the group-of-8 rule: see sum_of_squares_group
+            grp = __fmaf_rn(q1, q1, grp);
           }
+          sum += double(grp);
           if (!d.transposed) {
             *reinterpret_cast<uint4*>(X + size_t(r) * ldx + c) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           } else {
